@@ -1,0 +1,153 @@
+/*
+ * gt_attn.h -- C ABI of the B200 (sm_100a) biased graph-attention library.
+ *
+ * The library implements the single-GPU hot path of graph-transformer training that the
+ * MegaGraph paper parallelises: all-to-all node attention with an additive structural
+ * bias (the paper's Eq. 1),
+ *
+ *     Attention(Q,K,V) = Softmax(Q K^T / sqrt(d) + b_attn) V ,
+ *
+ * where b_attn encodes topology via shortest-path distances (Sec. "Preliminaries: Graph
+ * Transformer" and Sec. "Graph-Aware Context Parallelism", item 2).  Here b_attn is never
+ * materialised as floats: it is a uint8 shortest-path-distance (SPD) index matrix shared
+ * by all heads plus a small per-head table, b_attn[h][i][j] = bias[h][spd[i][j]].
+ *
+ * Conventions common to all entry points
+ * --------------------------------------
+ *  - Every pointer is a DEVICE pointer unless marked (host).  The caller owns every
+ *    buffer; the library allocates and frees no device memory.  Scratch comes from a
+ *    caller-provided workspace whose size is obtained from the matching *_workspace()
+ *    query (host function, no GPU work).  Workspace and all tensor base pointers must be
+ *    16-byte aligned.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only
+ *    enqueue work and return; they never synchronise.  Errors detected on the host are
+ *    returned immediately.  Errors detected on the device (a bounded wait that ran out)
+ *    are recorded in a status word at the start of the workspace and are reported by
+ *    gt_check(), which synchronises the stream.
+ *  - Node features are packed: a batch of G graphs with n_g nodes each is stored as
+ *    T = sum n_g consecutive rows; Q, K, V, O and their gradients are bf16 [T, H, d]
+ *    (row-major, d contiguous); graph g owns rows cu_seqlens[g] .. cu_seqlens[g+1]-1 and
+ *    attention is block diagonal (nodes attend only within their graph).  With one graph
+ *    (n_graphs == 1) cu_seqlens and spd_offsets may be NULL.
+ *  - SPD layout: graph g's block starts at byte spd_offsets[g] (int64, device) and holds
+ *    n_g rows of pitch ld_g = round_up(n_g, 16) bytes; spd[i*ld_g + j] is the bucket of the
+ *    ordered pair (i -> j): min(hops, max_dist), or max_dist+1 if j is unreachable from i.
+ *    There are n_buckets = max_dist + 2 buckets.  Values >= n_buckets found in the matrix
+ *    are clamped to n_buckets-1 on the device.  Padding bytes (j >= n_g) are ignored.
+ *  - Supported shapes: head_dim in {32, 64}; 1 <= max_dist <= 254; n_heads >= 1;
+ *    anything else returns GT_ERR_UNSUPPORTED / GT_ERR_INVALID_ARG without launching.
+ */
+#ifndef GT_ATTN_H_
+#define GT_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum gt_status {
+    GT_OK = 0,
+    GT_ERR_INVALID_ARG = 1,    /* NULL required pointer, bad size, misaligned pointer          */
+    GT_ERR_UNSUPPORTED = 2,    /* head_dim not in {32,64}, chunked call on a multi-graph batch */
+    GT_ERR_WORKSPACE = 3,      /* workspace NULL or smaller than the *_workspace() query       */
+    GT_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed (launch, descriptor)       */
+    GT_ERR_DEVICE_TIMEOUT = 5, /* a bounded device-side wait expired (reported by gt_check)    */
+    GT_ERR_NO_DEVICE = 6       /* no sm_100 device is current                                  */
+} gt_status;
+
+/* Packed batch description (host struct; cu_seqlens is a device pointer). */
+typedef struct gt_batch {
+    int32_t n_total;           /* T = sum n_g  (N for a single graph), >= 1              */
+    int32_t n_graphs;          /* G >= 1                                                 */
+    const int32_t* cu_seqlens; /* device int32[G+1], cu[0]=0, cu[G]=T; may be NULL if G==1 */
+    int32_t max_seqlen;        /* max_g n_g (host-known; sizes the launch grid)          */
+} gt_batch;
+
+const char* gt_status_string(gt_status s);
+
+/* Synchronises `stream`, then returns and clears the device status word held in the first
+ * bytes of `workspace` (GT_OK, or GT_ERR_DEVICE_TIMEOUT if a kernel gave up on a wait; the
+ * outputs of that call are then undefined).  `workspace` is one that was passed to any of
+ * the calls below. */
+gt_status gt_check(void* workspace, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * gt_spd_build -- structural-encoding construction (the paper builds b_attn from batch
+ * topology on the CPU during data loading, Sec. "Preliminaries" and the T_stall term of the
+ * latency model; this builds its index form on the GPU).
+ *
+ * Multi-source breadth-first search over a CSR graph.  row_ptr int32[T+1], col_idx
+ * int32[nnz]: row i lists the out-neighbours of packed node i as PACKED node ids; edges
+ * must stay inside a graph.  Self loops and duplicate entries are tolerated.  Writes the
+ * SPD block(s) described above into spd_out (every byte of every row, padding bytes = 255).
+ * The traversal runs to exhaustion, so pairs farther than max_dist (bucket max_dist) stay
+ * distinct from unreachable pairs (bucket max_dist+1).  Bit-exact and deterministic.
+ * Out-of-range col_idx entries are undefined behaviour.
+ * ------------------------------------------------------------------------------------- */
+size_t gt_spd_build_workspace(const gt_batch* batch, int64_t nnz, int32_t max_dist);
+gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx, int64_t nnz,
+                       const gt_batch* batch, int32_t max_dist,
+                       const int64_t* spd_offsets, uint8_t* spd_out,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * gt_biased_attn_fwd -- Eq. 1, forward.  For every graph, head h and query row i:
+ *     S_ij = (q_i . k_j)/sqrt(head_dim) + bias[h][spd_ij]        (all j of the same graph)
+ *     out_i = sum_j softmax_j(S_i)_j v_j,     lse[h][i] = log sum_j exp(S_ij)  (natural log)
+ * computed tile by tile with an online softmax in which the bias is added to the score
+ * before the running max / sum are updated (Sec. GA-CP, item 3).  bf16 inputs, fp32
+ * accumulation and softmax, bf16 `out` [T,H,d], fp32 `lse` [H,T].
+ * bias: fp32 [n_heads, max_dist+2].
+ * ------------------------------------------------------------------------------------- */
+size_t gt_biased_attn_fwd_workspace(const gt_batch* batch, int32_t n_heads, int32_t head_dim);
+gt_status gt_biased_attn_fwd(const void* q, const void* k, const void* v,
+                             const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
+                             const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                             void* out, float* lse,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * gt_biased_attn_bwd -- gradient of Eq. 1 for upstream gradient `dout` (bf16 [T,H,d]).
+ * With P_ij = exp(S_ij - lse_i) recomputed tile by tile:
+ *     Delta_i = dout_i . out_i         dP_ij = dout_i . v_j        dS_ij = P_ij (dP_ij - Delta_i)
+ *     dv_j = sum_i P_ij dout_i         dq_i = sum_j dS_ij k_j / sqrt(d)
+ *     dk_j = sum_i dS_ij q_i / sqrt(d) dbias[h][b] = sum over pairs with spd_ij == b of dS_ij
+ * `out` and `lse` are the forward results.  dq, dk, dv (bf16 [T,H,d]) and dbias
+ * (fp32 [n_heads, max_dist+2], summed over all graphs of the batch) are OVERWRITTEN.
+ * dq and dbias are accumulated with floating-point atomics, so their low-order bits may
+ * differ from run to run.
+ * ------------------------------------------------------------------------------------- */
+size_t gt_biased_attn_bwd_workspace(const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist);
+gt_status gt_biased_attn_bwd(const void* q, const void* k, const void* v, const void* out,
+                             const void* dout, const float* lse,
+                             const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
+                             const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                             void* dq, void* dk, void* dv, float* dbias,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * gt_biased_attn_fwd_chunked -- single-GPU analogue of graph-aware context parallelism
+ * (Sec. GA-CP: ring steps over KV blocks; Eq. 2: the bias columns of each block are taken at
+ * the block's global node indices; item 3: bias folded in before the softmax statistics).
+ * The key/value rows are split into n_kv_chunks contiguous chunks of
+ * w = round_up(ceil(N / n_kv_chunks), 128) rows (the last may be short or empty); each chunk
+ * yields a partial (out_c, lse_c) using spd[i][j] at the GLOBAL column j; partials are then
+ * merged:  lse = log sum_c exp(lse_c),  out = sum_c exp(lse_c - lse) out_c.
+ * Results equal gt_biased_attn_fwd up to rounding.  Single graph only (n_graphs == 1).
+ * lse_chunks: optional fp32 [n_kv_chunks, H, N] receiving lse_c (-inf for empty chunks), or NULL.
+ * ------------------------------------------------------------------------------------- */
+size_t gt_biased_attn_fwd_chunked_workspace(const gt_batch* batch, int32_t n_heads, int32_t head_dim,
+                                            int32_t n_kv_chunks);
+gt_status gt_biased_attn_fwd_chunked(const void* q, const void* k, const void* v,
+                                     const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
+                                     const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                     void* out, float* lse,
+                                     int32_t n_kv_chunks, float* lse_chunks,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GT_ATTN_H_ */

@@ -1,0 +1,198 @@
+"""ctypes binding of libgtattn.so: same names as the C ABI, argument marshalling only.
+
+Every function takes torch CUDA tensors (device memory owned by the caller), passes raw
+pointers and sizes through the C ABI on torch's current stream and raises ``GtError`` on a
+non-zero status.  There is no CPU fallback: if the CUDA library has not been built the
+import of the library fails loudly on first use.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgtattn.so")
+
+GT_OK = 0
+STATUS_NAMES = {0: "GT_OK", 1: "GT_ERR_INVALID_ARG", 2: "GT_ERR_UNSUPPORTED", 3: "GT_ERR_WORKSPACE",
+                4: "GT_ERR_CUDA", 5: "GT_ERR_DEVICE_TIMEOUT", 6: "GT_ERR_NO_DEVICE"}
+
+EXPORTS = ("gt_status_string", "gt_check",
+           "gt_spd_build_workspace", "gt_spd_build",
+           "gt_biased_attn_fwd_workspace", "gt_biased_attn_fwd",
+           "gt_biased_attn_bwd_workspace", "gt_biased_attn_bwd",
+           "gt_biased_attn_fwd_chunked_workspace", "gt_biased_attn_fwd_chunked")
+
+
+class GtError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)}")
+        self.status = status
+
+
+class _GtBatch(ctypes.Structure):
+    _fields_ = [("n_total", ctypes.c_int32), ("n_graphs", ctypes.c_int32),
+                ("cu_seqlens", ctypes.c_void_p), ("max_seqlen", ctypes.c_int32)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libgtattn.so (built in-tree by ``paper_2609_34420_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_34420_b200.build` "
+                              "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+        bp = ctypes.POINTER(_GtBatch)
+        L.gt_status_string.restype = ctypes.c_char_p
+        L.gt_status_string.argtypes = [ctypes.c_int]
+        L.gt_check.restype = ctypes.c_int
+        L.gt_check.argtypes = [vp, vp]
+        L.gt_spd_build_workspace.restype = sz
+        L.gt_spd_build_workspace.argtypes = [bp, i64, i32]
+        L.gt_spd_build.restype = ctypes.c_int
+        L.gt_spd_build.argtypes = [vp, vp, i64, bp, i32, vp, vp, vp, sz, vp]
+        if hasattr(L, "gt_biased_attn_fwd"):
+            L.gt_biased_attn_fwd_workspace.restype = sz
+            L.gt_biased_attn_fwd_workspace.argtypes = [bp, i32, i32]
+            L.gt_biased_attn_fwd.restype = ctypes.c_int
+            L.gt_biased_attn_fwd.argtypes = [vp, vp, vp, vp, vp, vp, bp, i32, i32, i32, vp, vp, vp, sz, vp]
+        if hasattr(L, "gt_biased_attn_bwd"):
+            L.gt_biased_attn_bwd_workspace.restype = sz
+            L.gt_biased_attn_bwd_workspace.argtypes = [bp, i32, i32, i32]
+            L.gt_biased_attn_bwd.restype = ctypes.c_int
+            L.gt_biased_attn_bwd.argtypes = [vp] * 9 + [bp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        if hasattr(L, "gt_biased_attn_fwd_chunked"):
+            L.gt_biased_attn_fwd_chunked_workspace.restype = sz
+            L.gt_biased_attn_fwd_chunked_workspace.argtypes = [bp, i32, i32, i32]
+            L.gt_biased_attn_fwd_chunked.restype = ctypes.c_int
+            L.gt_biased_attn_fwd_chunked.argtypes = [vp, vp, vp, vp, vp, vp, bp, i32, i32, i32, vp, vp, i32, vp, vp, sz, vp]
+        _lib = L
+    return _lib
+
+
+@dataclass
+class Batch:
+    """Packed batch: device ``cu_seqlens`` int32[G+1] and ``spd_offsets`` int64[G+1]
+    (both None for a single graph)."""
+    n_total: int
+    n_graphs: int = 1
+    max_seqlen: Optional[int] = None
+    cu_seqlens: Optional[torch.Tensor] = None
+    spd_offsets: Optional[torch.Tensor] = None
+
+    def c_struct(self) -> _GtBatch:
+        return _GtBatch(self.n_total, self.n_graphs, _ptr(self.cu_seqlens),
+                        self.n_total if self.max_seqlen is None else self.max_seqlen)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _raise(status: int, where: str) -> None:
+    if status != GT_OK:
+        raise GtError(status, where)
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    ws = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    ws[:256].zero_()
+    return ws
+
+
+def gt_check(workspace: torch.Tensor) -> None:
+    """Synchronise the current stream and raise if a kernel recorded a device-side error."""
+    _raise(lib().gt_check(_ptr(workspace), _stream()), "gt_check")
+
+
+# ------------------------------------------------------------------------------------------
+def gt_spd_build_workspace(batch: Batch, nnz: int, max_dist: int) -> int:
+    b = batch.c_struct()
+    return int(lib().gt_spd_build_workspace(ctypes.byref(b), int(nnz), int(max_dist)))
+
+
+def gt_spd_build(row_ptr: torch.Tensor, col_idx: torch.Tensor, batch: Batch, max_dist: int,
+                 spd_out: torch.Tensor, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Enqueue the SPD build; returns the workspace used (pass it to ``gt_check``)."""
+    nnz = int(col_idx.numel())
+    if workspace is None:
+        workspace = _workspace(gt_spd_build_workspace(batch, nnz, max_dist), row_ptr.device)
+    b = batch.c_struct()
+    st = lib().gt_spd_build(_ptr(row_ptr), _ptr(col_idx) if nnz else None, nnz, ctypes.byref(b), int(max_dist),
+                            _ptr(batch.spd_offsets), _ptr(spd_out), _ptr(workspace), workspace.numel(), _stream())
+    _raise(st, "gt_spd_build")
+    return workspace
+
+
+def gt_biased_attn_fwd_workspace(batch: Batch, n_heads: int, head_dim: int) -> int:
+    b = batch.c_struct()
+    return int(lib().gt_biased_attn_fwd_workspace(ctypes.byref(b), n_heads, head_dim))
+
+
+def gt_biased_attn_fwd(q, k, v, spd, bias, batch: Batch, max_dist: int, out, lse,
+                       workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _, H, d = q.shape
+    if workspace is None:
+        workspace = _workspace(gt_biased_attn_fwd_workspace(batch, H, d), q.device)
+    b = batch.c_struct()
+    st = lib().gt_biased_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(spd), _ptr(batch.spd_offsets), _ptr(bias),
+                                  ctypes.byref(b), H, d, int(max_dist), _ptr(out), _ptr(lse),
+                                  _ptr(workspace), workspace.numel(), _stream())
+    _raise(st, "gt_biased_attn_fwd")
+    return workspace
+
+
+def gt_biased_attn_bwd_workspace(batch: Batch, n_heads: int, head_dim: int, max_dist: int) -> int:
+    b = batch.c_struct()
+    return int(lib().gt_biased_attn_bwd_workspace(ctypes.byref(b), n_heads, head_dim, max_dist))
+
+
+def gt_biased_attn_bwd(q, k, v, out, dout, lse, spd, bias, batch: Batch, max_dist: int, dq, dk, dv, dbias,
+                       workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _, H, d = q.shape
+    if workspace is None:
+        workspace = _workspace(gt_biased_attn_bwd_workspace(batch, H, d, max_dist), q.device)
+    b = batch.c_struct()
+    st = lib().gt_biased_attn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(dout), _ptr(lse), _ptr(spd),
+                                  _ptr(batch.spd_offsets), _ptr(bias), ctypes.byref(b), H, d, int(max_dist),
+                                  _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dbias),
+                                  _ptr(workspace), workspace.numel(), _stream())
+    _raise(st, "gt_biased_attn_bwd")
+    return workspace
+
+
+def gt_biased_attn_fwd_chunked_workspace(batch: Batch, n_heads: int, head_dim: int, n_kv_chunks: int) -> int:
+    b = batch.c_struct()
+    return int(lib().gt_biased_attn_fwd_chunked_workspace(ctypes.byref(b), n_heads, head_dim, n_kv_chunks))
+
+
+def gt_biased_attn_fwd_chunked(q, k, v, spd, bias, batch: Batch, max_dist: int, out, lse, n_kv_chunks: int,
+                               lse_chunks: Optional[torch.Tensor] = None,
+                               workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _, H, d = q.shape
+    if workspace is None:
+        workspace = _workspace(gt_biased_attn_fwd_chunked_workspace(batch, H, d, n_kv_chunks), q.device)
+    b = batch.c_struct()
+    st = lib().gt_biased_attn_fwd_chunked(_ptr(q), _ptr(k), _ptr(v), _ptr(spd), _ptr(batch.spd_offsets), _ptr(bias),
+                                          ctypes.byref(b), H, d, int(max_dist), _ptr(out), _ptr(lse),
+                                          int(n_kv_chunks), _ptr(lse_chunks),
+                                          _ptr(workspace), workspace.numel(), _stream())
+    _raise(st, "gt_biased_attn_fwd_chunked")
+    return workspace
