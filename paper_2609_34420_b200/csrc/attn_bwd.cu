@@ -1,0 +1,615 @@
+// gt_biased_attn_bwd: gradient of Eq. 1 (O = Softmax(Q K^T / sqrt(d) + B_h[spd]) V) with
+// respect to Q, K, V and the per-head bias table.
+//
+// One CTA owns one head and one tile of 128 keys and walks over all 128-row query tiles of
+// the graph.  Scores are recomputed TRANSPOSED (S^T = K Q^T, thread = key row = TMEM lane) so
+// that P^T and dS^T can go straight back to tensor memory as the A operands of
+// dV += P^T dO and dK += dS^T Q; dS^T is also written to shared memory (MN-major A operand) for
+// dQ_i = dS K, which is added to an fp32 accumulator in global memory.  The bias-table
+// gradient dB[h][b] = sum of dS over pairs in bucket b is binned in shared memory (one
+// private bin column per thread, no conflicts) and flushed once per CTA with fp64 atomics.
+//
+//   warp 0        TMA producer: K, V once; Q_i, dO_i through a 2-stage ring
+//   warp 1        MMA issuer (5 GEMMs per query tile)
+//   warp 2        aux loader: SPD tile, lse*log2(e) and Delta of the query tile (cp.async)
+//   warps 4-11    two softmax warpgroups: query columns [0,64) and [64,128) of the tile
+//   warps 12-15   dQ reducer: TMEM -> red.global.add.v4.f32
+//
+// TMEM columns: S^T/P^T [0,128)  dP^T/dS^T [128,256)  dV [256,320)  dK [320,384)  dQ0 [384,448)  dQ1 [448,512).
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "attn_common.cuh"
+#include "sm100_primitives.cuh"
+
+namespace gt {
+namespace {
+
+using namespace sm100;
+
+constexpr int kTile = 128;
+constexpr int kStages = 2;
+constexpr int kBwdThreads = 512;
+constexpr int kSoftmaxThreads = 256;
+constexpr int kPrivateBinBuckets = 32;     // up to this many buckets: one private bin column per thread
+
+struct BwdParams {
+    const uint8_t* spd;
+    const int64_t* spd_offsets;
+    const int32_t* cu_seqlens;
+    const float* bias;
+    const float* lse2;       // [H,T] lse * log2(e)      (workspace)
+    const float* delta;      // [H,T] rowsum(dO * O)     (workspace)
+    float* dq_acc;           // [T,H,D] fp32             (workspace, zeroed)
+    double* db_acc;          // [H,nb] fp64              (workspace, zeroed)
+    __nv_bfloat16* dk;
+    __nv_bfloat16* dv;
+    uint32_t* status;
+    int32_t n_total;
+    int32_t n_heads;
+    int32_t n_buckets;
+    float c1;                // log2(e)/sqrt(d)
+    float scale;             // 1/sqrt(d)
+};
+
+enum BwdBarrier {
+    kBarKvFull = 0,
+    kBarQdoFull = 1,                       // [2]
+    kBarAuxFull = kBarQdoFull + kStages,   // [2]
+    kBarStageEmpty = kBarAuxFull + kStages,// [2]
+    kBarSFull = kBarStageEmpty + kStages,
+    kBarDpFull,
+    kBarPFull,
+    kBarDsFull,
+    kBarDqFull,                            // [2]
+    kBarDqFree = kBarDqFull + 2,           // [2]
+    kBarFinal = kBarDqFree + 2,
+    kNumBwdBarriers
+};
+
+template <int D>
+struct BwdSmem {
+    static constexpr int kRowBytes = D * 2;
+    static constexpr int kTileBytes = 128 * kRowBytes;
+    static constexpr int kSpdBytes = kTile * kTile;
+    static constexpr int kK = 0;
+    static constexpr int kV = kK + kTileBytes;
+    static constexpr int kQ = kV + kTileBytes;                      // [kStages]
+    static constexpr int kDo = kQ + kStages * kTileBytes;           // [kStages]
+    static constexpr int kSpd = kDo + kStages * kTileBytes;         // [kStages]
+    static constexpr int kLse = kSpd + kStages * kSpdBytes;         // [kStages][128] float
+    static constexpr int kDelta = kLse + kStages * 512;             // [kStages][128] float
+    static constexpr int kDs = kDelta + kStages * 512;              // 2 atoms x 128 rows x 128 B
+    static constexpr int kBins = kDs + 32768;                       // [32][256] float
+    static constexpr int kBias = kBins + kPrivateBinBuckets * kSoftmaxThreads * 4;
+    static constexpr int kBars = kBias + 256 * 4;
+    static constexpr int kMisc = kBars + kNumBwdBarriers * 8;
+    static constexpr int kTotal = kMisc + 16;
+    static constexpr int kDynamic = kTotal + 1024;
+};
+
+__device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src, uint32_t src_bytes)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t n_threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
+__device__ __forceinline__ void setmaxnreg_inc_192() { asm volatile("setmaxnreg.inc.sync.aligned.u32 192;"); }
+__device__ __forceinline__ void setmaxnreg_dec_72() { asm volatile("setmaxnreg.dec.sync.aligned.u32 72;"); }
+
+template <int D, bool kPrivateBins>
+__global__ void __launch_bounds__(kBwdThreads, 1)
+attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_do,
+                const BwdParams p)
+{
+    using L = BwdSmem<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const int h = blockIdx.x;
+    const int g = blockIdx.z;
+    const int32_t node0 = p.cu_seqlens ? p.cu_seqlens[g] : 0;
+    const int32_t n_g = p.cu_seqlens ? p.cu_seqlens[g + 1] - node0 : p.n_total;
+    const int32_t kv0 = (int32_t)blockIdx.y * kTile;
+    if (kv0 >= n_g) return;
+    const int64_t ld = (int64_t)((n_g + 15) & ~15);
+    const uint8_t* spd_g = p.spd + (p.spd_offsets ? p.spd_offsets[g] : 0);
+    const int32_t n_q = (n_g + kTile - 1) / kTile;
+
+    uint64_t* bars = (uint64_t*)(smem + L::kBars);
+    uint32_t* misc = (uint32_t*)(smem + L::kMisc);
+    float* s_bias = (float*)(smem + L::kBias);
+    float* s_bins = (float*)(smem + L::kBins);
+    auto bar = [&](int i) { return smem_u32(&bars[i]); };
+    volatile uint32_t* abort_flag = &misc[1];
+
+    if (tid == 0) {
+        misc[1] = 0u;
+        mbar_init(bar(kBarKvFull), 1);
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar(kBarQdoFull + s), 1);
+            mbar_init(bar(kBarAuxFull + s), 32);
+            mbar_init(bar(kBarStageEmpty + s), 1);
+            mbar_init(bar(kBarDqFull + s), 1);
+            mbar_init(bar(kBarDqFree + s), 128);
+        }
+        mbar_init(bar(kBarSFull), 1);
+        mbar_init(bar(kBarDpFull), 1);
+        mbar_init(bar(kBarPFull), kSoftmaxThreads);
+        mbar_init(bar(kBarDsFull), kSoftmaxThreads);
+        mbar_init(bar(kBarFinal), 1);
+        fence_mbar_init();
+        prefetch_tensormap(&tmap_q);
+        prefetch_tensormap(&tmap_k);
+        prefetch_tensormap(&tmap_v);
+        prefetch_tensormap(&tmap_do);
+    }
+    if (warp == 1) { tmem_alloc(smem_u32(&misc[0]), 512); tmem_relinquish(); }
+    for (int i = tid; i < 256; i += kBwdThreads)
+        s_bias[i] = p.bias[(size_t)h * p.n_buckets + min(i, p.n_buckets - 1)] * kLog2e;
+    for (int i = tid; i < kPrivateBinBuckets * kSoftmaxThreads; i += kBwdThreads) s_bins[i] = 0.f;
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = misc[0];
+    constexpr uint32_t kColS = 0, kColDp = 128, kColDv = 256, kColDk = 320, kColDq = 384;
+
+    if (warp < 4) {
+        setmaxnreg_dec_40();
+        if (warp == 0) {
+            // ------------------------------ TMA producer ------------------------------
+            if (lane == 0) {
+                mbar_arrive_expect_tx(bar(kBarKvFull), 2 * L::kTileBytes);
+                tma_load_3d(smem_u32(smem + L::kK), &tmap_k, bar(kBarKvFull), 0, h, node0 + kv0);
+                tma_load_3d(smem_u32(smem + L::kV), &tmap_v, bar(kBarKvFull), 0, h, node0 + kv0);
+            }
+            for (int i = 0; i < n_q; ++i) {
+                const int s = i & 1;
+                mbar_wait(bar(kBarStageEmpty + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 110);
+                if (lane == 0) {
+                    const int32_t row = node0 + i * kTile;
+                    mbar_arrive_expect_tx(bar(kBarQdoFull + s), 2 * L::kTileBytes);
+                    tma_load_3d(smem_u32(smem + L::kQ + s * L::kTileBytes), &tmap_q, bar(kBarQdoFull + s), 0, h, row);
+                    tma_load_3d(smem_u32(smem + L::kDo + s * L::kTileBytes), &tmap_do, bar(kBarQdoFull + s), 0, h, row);
+                }
+                __syncwarp();
+            }
+        } else if (warp == 1) {
+            // ------------------------------ MMA issuer ------------------------------
+            constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
+            constexpr uint32_t idesc_ts = make_idesc_bf16(128, D, false, true);    // A in TMEM, B MN-major
+            constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);     // A and B MN-major
+            const uint32_t sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV);
+            auto issue_st = [&](int s) {        // S^T = K Q^T
+                uint64_t da = make_smem_desc(sK, L::kRowBytes, 0);
+                uint64_t db = make_smem_desc(smem_u32(smem + L::kQ + s * L::kTileBytes), L::kRowBytes, 0);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    mma_ss(tmem + kColS, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
+                mma_commit(bar(kBarSFull));
+            };
+            auto issue_dpt = [&](int s) {       // dP^T = V dO^T
+                uint64_t da = make_smem_desc(sV, L::kRowBytes, 0);
+                uint64_t db = make_smem_desc(smem_u32(smem + L::kDo + s * L::kTileBytes), L::kRowBytes, 0);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    mma_ss(tmem + kColDp, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
+                mma_commit(bar(kBarDpFull));
+            };
+            mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 120);
+            mbar_wait(bar(kBarQdoFull + 0), 0, abort_flag, p.status, 121);
+            tc_fence_after();
+            if (lane == 0) { issue_st(0); issue_dpt(0); }
+            __syncwarp();
+            for (int i = 0; i < n_q; ++i) {
+                const int s = i & 1;
+                // ---- after P^T: dV += P^T dO_i, then S^T of the next tile ----
+                mbar_wait(bar(kBarPFull), i & 1, abort_flag, p.status, 122);
+                tc_fence_after();
+                if (lane == 0) {
+                    uint64_t db = make_smem_desc(smem_u32(smem + L::kDo + s * L::kTileBytes), L::kRowBytes, 0);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_ts(tmem + kColDv, tmem + kColS + (ks >> 2) * 64 + (ks & 3) * 8,
+                               advance_desc(db, ks * 16 * L::kRowBytes), idesc_ts, (i > 0 || ks > 0) ? 1u : 0u);
+                }
+                __syncwarp();
+                if (i + 1 < n_q) {
+                    mbar_wait(bar(kBarQdoFull + (s ^ 1)), ((i + 1) >> 1) & 1, abort_flag, p.status, 123);
+                    tc_fence_after();
+                    if (lane == 0) issue_st(s ^ 1);
+                    __syncwarp();
+                }
+                // ---- after dS^T: dK += dS^T Q_i, dQ_i = dS K, then dP^T of the next tile ----
+                mbar_wait(bar(kBarDsFull), i & 1, abort_flag, p.status, 124);
+                mbar_wait(bar(kBarDqFree + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 125);
+                tc_fence_after();
+                if (lane == 0) {
+                    uint64_t dbq = make_smem_desc(smem_u32(smem + L::kQ + s * L::kTileBytes), L::kRowBytes, 0);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_ts(tmem + kColDk, tmem + kColDp + (ks >> 2) * 64 + (ks & 3) * 8,
+                               advance_desc(dbq, ks * 16 * L::kRowBytes), idesc_ts, (i > 0 || ks > 0) ? 1u : 0u);
+                    uint64_t da = make_smem_desc(smem_u32(smem + L::kDs), 128, 16384);
+                    uint64_t dbk = make_smem_desc(sK, L::kRowBytes, 0);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_ss(tmem + kColDq + s * 64, advance_desc(da, ks * 2048),
+                               advance_desc(dbk, ks * 16 * L::kRowBytes), idesc_dq, ks > 0);
+                    mma_commit(bar(kBarDqFull + s));
+                    mma_commit(bar(kBarStageEmpty + s));
+                    if (i + 1 < n_q) issue_dpt(s ^ 1);
+                }
+                __syncwarp();
+            }
+            if (lane == 0) mma_commit(bar(kBarFinal));
+            __syncwarp();
+        } else if (warp == 2) {
+            // ------------------------------ aux loader ------------------------------
+            for (int i = 0; i < n_q; ++i) {
+                const int s = i & 1;
+                mbar_wait(bar(kBarStageEmpty + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 130);
+                const int32_t q0 = i * kTile;
+                const uint32_t dst0 = smem_u32(smem + L::kSpd + s * L::kSpdBytes);
+#pragma unroll 4
+                for (int it = 0; it < (kTile * 8) / 32; ++it) {
+                    const int c = it * 32 + lane;
+                    const int r = c >> 3, cc = c & 7;
+                    const int64_t col = (int64_t)kv0 + cc * 16;
+                    const bool valid = (q0 + r < n_g) && (col < ld);
+                    const uint8_t* src = valid ? spd_g + (int64_t)(q0 + r) * ld + col : spd_g;
+                    cp_async_16(dst0 + r * 128 + cc * 16, src, valid ? 16u : 0u);
+                }
+                const uint32_t dl = smem_u32(smem + L::kLse + s * 512), dd = smem_u32(smem + L::kDelta + s * 512);
+#pragma unroll
+                for (int it = 0; it < 4; ++it) {
+                    const int r = it * 32 + lane;
+                    const bool valid = q0 + r < n_g;
+                    const size_t off = (size_t)h * p.n_total + node0 + (valid ? q0 + r : 0);
+                    cp_async_4(dl + r * 4, p.lse2 + off, valid ? 4u : 0u);
+                    cp_async_4(dd + r * 4, p.delta + off, valid ? 4u : 0u);
+                }
+                cp_async_mbar_arrive_noinc(bar(kBarAuxFull + s));
+            }
+        }
+    } else if (warp < 12) {
+        // ================================ softmax warpgroups ================================
+        setmaxnreg_inc_192();
+        const int w = (warp >> 2) - 1;                  // query-column half handled by this warpgroup
+        const int r = tid & 127;                        // key row within the tile = TMEM lane
+        const int st = tid - 128;                       // 0..255 index among softmax threads
+        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + kColS + w * 64 + lane_off;
+        const uint32_t tDp = tmem + kColDp + w * 64 + lane_off;
+        const bool kv_valid = kv0 + r < n_g;
+        const float c1 = p.c1;
+        const uint32_t nb_m1 = (uint32_t)p.n_buckets - 1u;
+        float* my_bins = s_bins + (kPrivateBins ? st : lane);
+        constexpr int kBinStride = kPrivateBins ? kSoftmaxThreads : 32;
+
+        for (int i = 0; i < n_q; ++i) {
+            const int s = i & 1;
+            float pr[64];
+            uint32_t bk[16];
+            // ---------------- P^T = exp2(S^T c1 + b2 - lse2) ----------------
+            mbar_wait(bar(kBarSFull), i & 1, abort_flag, p.status, 140);
+            tc_fence_after();
+            {
+                uint32_t a0[32], a1[32];
+                tmem_ld32(tS, a0);
+                tmem_ld32(tS + 32, a1);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 32; ++c) { pr[c] = __uint_as_float(a0[c]); pr[32 + c] = __uint_as_float(a1[c]); }
+            }
+            mbar_wait(bar(kBarAuxFull + s), (i >> 1) & 1, abort_flag, p.status, 141);
+            const uint8_t* spd_col = smem + L::kSpd + s * L::kSpdBytes + (w * 64) * 128 + r;
+            const float4* lse4 = (const float4*)(smem + L::kLse + s * 512 + w * 256);
+#pragma unroll
+            for (int c4 = 0; c4 < 16; ++c4) {
+                const float4 l4 = lse4[c4];
+                const float ls[4] = {l4.x, l4.y, l4.z, l4.w};
+                uint32_t packed = 0;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int c = c4 * 4 + k;
+                    const uint32_t b = min((uint32_t)spd_col[c * 128], nb_m1);    // never index past the table
+                    packed |= b << (8 * k);
+                    pr[c] = ex2_approx(fmaf(pr[c], c1, s_bias[b]) - ls[k]);
+                }
+                bk[c4] = packed;
+            }
+            const int nq_valid = n_g - i * kTile - w * 64;      // valid query columns of this half
+            if (!kv_valid || nq_valid < 64) {
+#pragma unroll
+                for (int c = 0; c < 64; ++c)
+                    if (!kv_valid || c >= nq_valid) pr[c] = 0.f;
+            }
+            {
+                uint32_t pk[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) pk[c] = pack_bf16x2(pr[2 * c], pr[2 * c + 1]);
+                tmem_st32(tS, pk);                      // P^T half: 32 packed columns at the start of the half
+                tmem_wait_st();
+            }
+            tc_fence_before();
+            mbar_arrive(bar(kBarPFull));
+
+            // ---------------- dS^T = P^T o (dP^T - Delta) ----------------
+            mbar_wait(bar(kBarDpFull), i & 1, abort_flag, p.status, 142);
+            tc_fence_after();
+            {
+                uint32_t a0[32], a1[32];
+                tmem_ld32(tDp, a0);
+                tmem_ld32(tDp + 32, a1);
+                tmem_wait_ld();
+                const float4* dl4 = (const float4*)(smem + L::kDelta + s * 512 + w * 256);
+#pragma unroll
+                for (int c4 = 0; c4 < 16; ++c4) {
+                    const float4 d4 = dl4[c4];
+                    const float dl[4] = {d4.x, d4.y, d4.z, d4.w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int c = c4 * 4 + k;
+                        const float dp = __uint_as_float(c < 32 ? a0[c & 31] : a1[c & 31]);
+                        const float ds = pr[c] * (dp - dl[k]);
+                        pr[c] = ds;
+                        const uint32_t b = (bk[c4] >> (8 * k)) & 0xffu;
+                        if (kPrivateBins) my_bins[b * kBinStride] += ds;
+                        else atomicAdd(&my_bins[b * kBinStride], ds);
+                    }
+                }
+            }
+            {
+                uint32_t pk[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) pk[c] = pack_bf16x2(pr[2 * c], pr[2 * c + 1]);
+                tmem_st32(tDp, pk);
+                uint8_t* ds_row = smem + L::kDs + w * 16384 + r * 128;
+#pragma unroll
+                for (int c8 = 0; c8 < 8; ++c8)
+                    *(uint4*)(ds_row + ((c8 ^ (r & 7)) << 4)) = make_uint4(pk[4 * c8], pk[4 * c8 + 1], pk[4 * c8 + 2], pk[4 * c8 + 3]);
+                tmem_wait_st();
+            }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            mbar_arrive(bar(kBarDsFull));
+        }
+
+        // ---------------- epilogue: dV (warpgroup 0) and dK (warpgroup 1) ----------------
+        mbar_wait(bar(kBarFinal), 0, abort_flag, p.status, 143);
+        tc_fence_after();
+        {
+            const uint32_t tacc = tmem + (w == 0 ? kColDv : kColDk) + lane_off;
+            const float mul = w == 0 ? 1.0f : p.scale;
+            __nv_bfloat16* dst_base = (w == 0 ? p.dv : p.dk) + ((size_t)(node0 + kv0 + r) * p.n_heads + h) * D;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tacc + c * 32, o);
+                tmem_wait_ld();
+                if (kv_valid) {
+                    uint4* dst = (uint4*)(dst_base + c * 32);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(o[8 * k]) * mul, __uint_as_float(o[8 * k + 1]) * mul);
+                        v.y = pack_bf16x2(__uint_as_float(o[8 * k + 2]) * mul, __uint_as_float(o[8 * k + 3]) * mul);
+                        v.z = pack_bf16x2(__uint_as_float(o[8 * k + 4]) * mul, __uint_as_float(o[8 * k + 5]) * mul);
+                        v.w = pack_bf16x2(__uint_as_float(o[8 * k + 6]) * mul, __uint_as_float(o[8 * k + 7]) * mul);
+                        dst[k] = v;
+                    }
+                }
+            }
+        }
+        // ---------------- flush the bias-gradient bins ----------------
+        named_barrier_sync(1, kSoftmaxThreads);
+        if (kPrivateBins) {
+            if (st < p.n_buckets) {
+                float acc = 0.f;
+                for (int k = 0; k < kSoftmaxThreads; ++k) acc += s_bins[st * kSoftmaxThreads + ((k + st) & (kSoftmaxThreads - 1))];
+                atomicAdd(&p.db_acc[(size_t)h * p.n_buckets + st], (double)acc);
+            }
+        } else {
+            for (int b = st; b < p.n_buckets; b += kSoftmaxThreads) {
+                float acc = 0.f;
+                for (int k = 0; k < 32; ++k) acc += s_bins[b * 32 + ((k + b) & 31)];
+                atomicAdd(&p.db_acc[(size_t)h * p.n_buckets + b], (double)acc);
+            }
+        }
+    } else {
+        // ================================ dQ reducer ================================
+        setmaxnreg_dec_72();
+        const int r = tid & 127;
+        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+        for (int i = 0; i < n_q; ++i) {
+            const int s = i & 1;
+            mbar_wait(bar(kBarDqFull + s), (i >> 1) & 1, abort_flag, p.status, 150);
+            tc_fence_after();
+            const int32_t q = i * kTile + r;
+            float* dst = p.dq_acc + ((size_t)(node0 + q) * p.n_heads + h) * D;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tmem + kColDq + s * 64 + c * 32 + lane_off, o);
+                tmem_wait_ld();
+                if (q < n_g) {
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        red_add_v4(dst + c * 32 + 4 * k, __uint_as_float(o[4 * k]), __uint_as_float(o[4 * k + 1]),
+                                   __uint_as_float(o[4 * k + 2]), __uint_as_float(o[4 * k + 3]));
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(bar(kBarDqFree + s));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) __nanosleep(200000);
+    if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+// Delta[h][t] = sum_c dO[t,h,c] * O[t,h,c];  lse2[h][t] = lse[h][t] * log2(e).
+template <int D>
+__global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
+                                      const float* __restrict__ lse, float* __restrict__ delta, float* __restrict__ lse2,
+                                      int32_t n_total, int32_t n_heads)
+{
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // = t * H + h
+    if (idx >= (size_t)n_total * n_heads) return;
+    const int32_t t = (int32_t)(idx / n_heads), h = (int32_t)(idx % n_heads);
+    const uint4* o4 = (const uint4*)(out + idx * D);
+    const uint4* d4 = (const uint4*)(dout + idx * D);
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < D / 8; ++i) {
+        const uint4 a = o4[i], b = d4[i];
+        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            acc += __uint_as_float(aw[k] << 16) * __uint_as_float(bw[k] << 16);
+            acc += __uint_as_float(aw[k] & 0xffff0000u) * __uint_as_float(bw[k] & 0xffff0000u);
+        }
+    }
+    const size_t o = (size_t)h * n_total + t;
+    delta[o] = acc;
+    lse2[o] = lse[o] * kLog2e;
+}
+
+// dq = bf16(scale * dq_acc);  dbias = float(db_acc)
+__global__ void bwd_finalize_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dq, size_t n_vec4,
+                                    float scale, const double* __restrict__ db_acc, float* __restrict__ dbias, int32_t n_db)
+{
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < (size_t)n_db) dbias[idx] = (float)db_acc[idx];
+    if (idx >= n_vec4) return;
+    const float4 v = ((const float4*)dq_acc)[idx];
+    uint2 pk;
+    pk.x = pack_bf16x2(v.x * scale, v.y * scale);
+    pk.y = pack_bf16x2(v.z * scale, v.w * scale);
+    ((uint2*)dq)[idx] = pk;
+}
+
+struct BwdWorkspace {
+    size_t db_off, delta_off, lse2_off, dq_off, total;
+};
+
+BwdWorkspace bwd_workspace(const gt_batch* b, int32_t n_heads, int32_t head_dim, int32_t max_dist)
+{
+    BwdWorkspace w{};
+    const size_t rows = (size_t)b->n_total * n_heads;
+    w.db_off = kHeaderBytes;
+    w.delta_off = w.db_off + align_up((size_t)n_heads * (max_dist + 2) * sizeof(double), 256);
+    w.lse2_off = w.delta_off + align_up(rows * sizeof(float), 256);
+    w.dq_off = w.lse2_off + align_up(rows * sizeof(float), 256);
+    w.total = w.dq_off + align_up(rows * head_dim * sizeof(float), 256);
+    return w;
+}
+
+template <int D>
+gt_status launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
+                     const BwdParams& p, const gt_batch* batch, cudaStream_t s)
+{
+    dim3 grid((unsigned)p.n_heads, (unsigned)((batch->max_seqlen + kTile - 1) / kTile), (unsigned)batch->n_graphs);
+    if (p.n_buckets <= kPrivateBinBuckets) {
+        auto kern = attn_bwd_kernel<D, true>;
+        GT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kDynamic));
+        kern<<<grid, kBwdThreads, BwdSmem<D>::kDynamic, s>>>(tq, tk, tv, tdo, p);
+    } else {
+        auto kern = attn_bwd_kernel<D, false>;
+        GT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kDynamic));
+        kern<<<grid, kBwdThreads, BwdSmem<D>::kDynamic, s>>>(tq, tk, tv, tdo, p);
+    }
+    GT_CUDA_TRY(cudaGetLastError());
+    return GT_OK;
+}
+
+}  // namespace
+}  // namespace gt
+
+extern "C" size_t gt_biased_attn_bwd_workspace(const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist)
+{
+    if (gt::validate_batch(batch) != GT_OK || n_heads < 1 || max_dist < 1 || max_dist > 254) return 0;
+    return gt::bwd_workspace(batch, n_heads, head_dim, max_dist).total;
+}
+
+extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void* v, const void* out,
+                                        const void* dout, const float* lse,
+                                        const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
+                                        const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                        void* dq, void* dk, void* dv, float* dbias,
+                                        void* workspace, size_t workspace_bytes, void* stream)
+{
+    using namespace gt;
+    gt_status st = validate_attn_common(batch, n_heads, head_dim, max_dist, spd_offsets);
+    if (st != GT_OK) return st;
+    if (!q || !k || !v || !out || !dout || !lse || !spd || !bias || !dq || !dk || !dv || !dbias) return GT_ERR_INVALID_ARG;
+    if (misaligned16(q) || misaligned16(k) || misaligned16(v) || misaligned16(out) || misaligned16(dout) ||
+        misaligned16(spd) || misaligned16(dq) || misaligned16(dk) || misaligned16(dv))
+        return GT_ERR_INVALID_ARG;
+    if (n_heads > 65535 || batch->n_graphs > 65535) return GT_ERR_UNSUPPORTED;
+    const BwdWorkspace wsp = bwd_workspace(batch, n_heads, head_dim, max_dist);
+    if (workspace == nullptr || workspace_bytes < wsp.total || misaligned16(workspace)) return GT_ERR_WORKSPACE;
+    if (sm_count() <= 0) return GT_ERR_NO_DEVICE;
+
+    CUtensorMap tq, tk, tv, tdo;
+    if ((st = encode_thd_map(&tq, q, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&tk, k, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&tv, v, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&tdo, dout, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    uint8_t* ws = (uint8_t*)workspace;
+    const size_t rows = (size_t)batch->n_total * n_heads;
+    const int32_t n_db = n_heads * (max_dist + 2);
+    BwdParams p{};
+    p.spd = spd;
+    p.spd_offsets = batch->n_graphs > 1 ? spd_offsets : nullptr;
+    p.cu_seqlens = batch->n_graphs > 1 ? batch->cu_seqlens : nullptr;
+    p.bias = bias;
+    p.lse2 = (float*)(ws + wsp.lse2_off);
+    p.delta = (float*)(ws + wsp.delta_off);
+    p.dq_acc = (float*)(ws + wsp.dq_off);
+    p.db_acc = (double*)(ws + wsp.db_off);
+    p.dk = (__nv_bfloat16*)dk;
+    p.dv = (__nv_bfloat16*)dv;
+    p.status = (uint32_t*)workspace;
+    p.n_total = batch->n_total;
+    p.n_heads = n_heads;
+    p.n_buckets = max_dist + 2;
+    p.scale = 1.0f / sqrtf((float)head_dim);
+    p.c1 = kLog2e * p.scale;
+
+    GT_CUDA_TRY(cudaMemsetAsync(ws + wsp.db_off, 0, (size_t)n_db * sizeof(double), s));
+    GT_CUDA_TRY(cudaMemsetAsync(ws + wsp.dq_off, 0, rows * head_dim * sizeof(float), s));
+    const unsigned pre_blocks = (unsigned)((rows + 255) / 256);
+    if (head_dim == 64)
+        bwd_preprocess_kernel<64><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse,
+                                                             (float*)(ws + wsp.delta_off), (float*)(ws + wsp.lse2_off),
+                                                             batch->n_total, n_heads);
+    else
+        bwd_preprocess_kernel<32><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse,
+                                                             (float*)(ws + wsp.delta_off), (float*)(ws + wsp.lse2_off),
+                                                             batch->n_total, n_heads);
+    GT_CUDA_TRY(cudaGetLastError());
+    st = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, p, batch, s) : launch_bwd<32>(tq, tk, tv, tdo, p, batch, s);
+    if (st != GT_OK) return st;
+    const size_t n_vec4 = rows * head_dim / 4;
+    const size_t n_fin = n_vec4 > (size_t)n_db ? n_vec4 : (size_t)n_db;
+    bwd_finalize_kernel<<<(unsigned)((n_fin + 255) / 256), 256, 0, s>>>(p.dq_acc, (__nv_bfloat16*)dq, n_vec4, p.scale,
+                                                                         p.db_acc, dbias, n_db);
+    GT_CUDA_TRY(cudaGetLastError());
+    return GT_OK;
+}

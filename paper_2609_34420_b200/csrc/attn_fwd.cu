@@ -1,0 +1,587 @@
+// gt_biased_attn_fwd / gt_biased_attn_fwd_chunked: Eq. 1 forward,
+//     O = Softmax(Q K^T / sqrt(d) + B_h[spd]) V,
+// flash-style: score tiles are produced by tcgen05 MMAs into tensor memory, the bias is
+// gathered from a per-head table by the SPD bucket and added BEFORE the running max / sum
+// are updated (the rule the paper states for its context-parallel online softmax), P goes
+// back to tensor memory as the A operand of the P V MMA.
+//
+// One CTA = one head x 256 query rows (two 128-row tiles, one softmax warpgroup each, so the
+// tensor pipe works on one tile while the other is in its softmax) x all key tiles of the
+// graph (or of one key chunk for the chunked entry point).
+//
+//   warp 0      TMA producer: Q once, then K/V tiles through a 3-stage ring
+//   warp 1      MMA issuer: S_t = Q_t K^T (SS), O_t += P_t V (A from TMEM, B = V as MN-major)
+//   warp 2      SPD loader: 256x128-byte index tile per key tile via cp.async, 16-byte chunks
+//               XOR-swizzled by row so that the row-per-thread reads are conflict free
+//   warps 4-7   softmax of tile 0 (thread = query row = TMEM lane), warps 8-11 of tile 1
+//
+// TMEM columns: S0 [0,128) S1 [128,256) P0 [256,320) P1 [320,384) O0 [384,448) O1 [448,512).
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "attn_common.cuh"
+#include "sm100_primitives.cuh"
+
+namespace gt {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+gt_status encode_thd_map(CUtensorMap* map, const void* base, int32_t n_total, int32_t n_heads, int32_t head_dim)
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return GT_ERR_CUDA;
+        }
+        fn = (EncodeTiledFn)p;
+    }
+    cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)n_heads, (cuuint64_t)n_total};
+    cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)n_heads * head_dim * 2};
+    cuuint32_t box[3] = {(cuuint32_t)head_dim, 1, 128};
+    cuuint32_t elem_strides[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, elem_strides,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    head_dim == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? GT_OK : GT_ERR_CUDA;
+}
+
+namespace {
+
+using namespace sm100;
+
+constexpr int kRowsPerTile = 128;
+constexpr int kQTiles = 2;
+constexpr int kRowsPerCta = kRowsPerTile * kQTiles;
+constexpr int kKvTile = 128;
+constexpr int kKvStages = 3;
+constexpr int kSpdStages = 2;
+constexpr int kFwdThreads = 384;
+constexpr float kRescaleThreshold = 8.0f;     // log2 units: keep a stale max while P stays below 2^8
+
+struct FwdParams {
+    const uint8_t* spd;
+    const int64_t* spd_offsets;
+    const int32_t* cu_seqlens;
+    const float* bias;
+    __nv_bfloat16* out;        // [T,H,D]          (unchunked)
+    float* lse;                // [H,T]            (unchunked)
+    float* part_o;             // [C,T,H,D] fp32   (chunked)
+    float* part_lse;           // [C,H,T]          (chunked)
+    uint32_t* status;
+    int32_t n_total;
+    int32_t n_heads;
+    int32_t n_buckets;
+    int32_t kv_chunk_rows;     // chunked: keys per chunk (multiple of 128)
+    float c1;                  // log2(e) / sqrt(d)
+};
+
+enum FwdBarrier {
+    kBarQFull = 0,
+    kBarKvFull = 1,                          // [kKvStages]
+    kBarKvEmpty = kBarKvFull + kKvStages,    // [kKvStages]
+    kBarSpdFull = kBarKvEmpty + kKvStages,   // [kSpdStages]
+    kBarSpdEmpty = kBarSpdFull + kSpdStages, // [kSpdStages]
+    kBarSFull = kBarSpdEmpty + kSpdStages,   // [2]
+    kBarSFree = kBarSFull + 2,               // [2]
+    kBarPFull = kBarSFree + 2,               // [2]
+    kBarODone = kBarPFull + 2,               // [2]
+    kNumFwdBarriers = kBarODone + 2
+};
+
+template <int D>
+struct FwdSmem {
+    static constexpr int kRowBytes = D * 2;
+    static constexpr int kTileBytes = 128 * kRowBytes;
+    static constexpr int kSpdTileBytes = kRowsPerCta * kKvTile;
+    static constexpr int kQ = 0;
+    static constexpr int kK = kQ + kQTiles * kTileBytes;
+    static constexpr int kV = kK + kKvStages * kTileBytes;
+    static constexpr int kSpd = kV + kKvStages * kTileBytes;
+    static constexpr int kBias = kSpd + kSpdStages * kSpdTileBytes;
+    static constexpr int kBars = kBias + 256 * 4;
+    static constexpr int kMisc = kBars + kNumFwdBarriers * 8;
+    static constexpr int kTotal = kMisc + 16;
+    static constexpr int kDynamic = kTotal + 1024;   // slack for the 1024-byte alignment
+};
+
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
+template <int D, bool kPartial>
+__global__ void __launch_bounds__(kFwdThreads, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                const __grid_constant__ CUtensorMap tmap_v, const FwdParams p)
+{
+    using L = FwdSmem<D>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const int h = blockIdx.x;
+    const int g = kPartial ? 0 : (int)blockIdx.z;
+    const int chunk = kPartial ? (int)blockIdx.z : 0;
+
+    const int32_t node0 = p.cu_seqlens ? p.cu_seqlens[g] : 0;
+    const int32_t n_g = p.cu_seqlens ? p.cu_seqlens[g + 1] - node0 : p.n_total;
+    const int32_t q0 = (int32_t)blockIdx.y * kRowsPerCta;
+    if (q0 >= n_g) return;
+    const int64_t ld = (int64_t)((n_g + 15) & ~15);
+    const uint8_t* spd_g = p.spd + (p.spd_offsets ? p.spd_offsets[g] : 0);
+    const int32_t kv_begin = kPartial ? chunk * p.kv_chunk_rows : 0;
+    const int32_t kv_end = kPartial ? min(n_g, kv_begin + p.kv_chunk_rows) : n_g;
+    const int32_t n_kv = kv_end > kv_begin ? (kv_end - kv_begin + kKvTile - 1) / kKvTile : 0;
+
+    if (kPartial && n_kv == 0) {            // empty chunk: weight zero in the merge
+        for (int i = tid; i < kRowsPerCta; i += kFwdThreads) {
+            int q = q0 + i;
+            if (q < n_g) {
+                p.part_lse[((size_t)chunk * p.n_heads + h) * p.n_total + q] = -INFINITY;
+                float* o = p.part_o + (((size_t)chunk * p.n_total + q) * p.n_heads + h) * D;
+                for (int c = 0; c < D; ++c) o[c] = 0.f;
+            }
+        }
+        return;
+    }
+
+    uint64_t* bars = (uint64_t*)(smem + L::kBars);
+    uint32_t* misc = (uint32_t*)(smem + L::kMisc);       // [0] TMEM base, [1] abort flag
+    float* s_bias = (float*)(smem + L::kBias);
+    auto bar = [&](int i) { return smem_u32(&bars[i]); };
+    volatile uint32_t* abort_flag = &misc[1];
+
+    if (tid == 0) {
+        misc[1] = 0u;
+        mbar_init(bar(kBarQFull), 1);
+        for (int s = 0; s < kKvStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), 1); }
+        for (int s = 0; s < kSpdStages; ++s) { mbar_init(bar(kBarSpdFull + s), 32); mbar_init(bar(kBarSpdEmpty + s), 8); }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(bar(kBarSFull + t), 1);
+            mbar_init(bar(kBarSFree + t), 128);
+            mbar_init(bar(kBarPFull + t), 128);
+            mbar_init(bar(kBarODone + t), 1);
+        }
+        fence_mbar_init();
+        prefetch_tensormap(&tmap_q);
+        prefetch_tensormap(&tmap_k);
+        prefetch_tensormap(&tmap_v);
+    }
+    if (warp == 1) { tmem_alloc(smem_u32(&misc[0]), 512); tmem_relinquish(); }
+    for (int i = tid; i < 256; i += kFwdThreads)
+        s_bias[i] = p.bias[(size_t)h * p.n_buckets + min(i, p.n_buckets - 1)] * kLog2e;
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = misc[0];
+
+    if (warp < 4) {
+        // =========================== producer / MMA / SPD warps ===========================
+        setmaxnreg_dec_40();
+        if (warp == 0) {
+            if (lane == 0) {
+                mbar_arrive_expect_tx(bar(kBarQFull), kQTiles * L::kTileBytes);
+                for (int t = 0; t < kQTiles; ++t)
+                    tma_load_3d(smem_u32(smem + L::kQ + t * L::kTileBytes), &tmap_q, bar(kBarQFull), 0, h,
+                                node0 + q0 + t * kRowsPerTile);
+            }
+            for (int j = 0; j < n_kv; ++j) {
+                const int s = j % kKvStages;
+                mbar_wait(bar(kBarKvEmpty + s), ((j / kKvStages) & 1) ^ 1, abort_flag, p.status, 10);
+                if (lane == 0) {
+                    const int32_t row = node0 + kv_begin + j * kKvTile;
+                    mbar_arrive_expect_tx(bar(kBarKvFull + s), 2 * L::kTileBytes);
+                    tma_load_3d(smem_u32(smem + L::kK + s * L::kTileBytes), &tmap_k, bar(kBarKvFull + s), 0, h, row);
+                    tma_load_3d(smem_u32(smem + L::kV + s * L::kTileBytes), &tmap_v, bar(kBarKvFull + s), 0, h, row);
+                }
+                __syncwarp();
+            }
+        } else if (warp == 1) {
+            constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
+            constexpr uint32_t idesc_o = make_idesc_bf16(128, D, false, true);
+            auto issue_s = [&](int t, int stage) {
+                uint64_t da = make_smem_desc(smem_u32(smem + L::kQ + t * L::kTileBytes), L::kRowBytes, 0);
+                uint64_t db = make_smem_desc(smem_u32(smem + L::kK + stage * L::kTileBytes), L::kRowBytes, 0);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    mma_ss(tmem + t * 128, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
+                mma_commit(bar(kBarSFull + t));
+            };
+            mbar_wait(bar(kBarQFull), 0, abort_flag, p.status, 20);
+            mbar_wait(bar(kBarKvFull + 0), 0, abort_flag, p.status, 21);
+            tc_fence_after();
+            if (lane == 0) { issue_s(0, 0); issue_s(1, 0); }
+            __syncwarp();
+            for (int j = 0; j < n_kv; ++j) {
+                const int s = j % kKvStages;
+                if (j + 1 < n_kv) {
+                    const int s1 = (j + 1) % kKvStages;
+                    mbar_wait(bar(kBarKvFull + s1), ((j + 1) / kKvStages) & 1, abort_flag, p.status, 22);
+                    for (int t = 0; t < 2; ++t) {
+                        mbar_wait(bar(kBarSFree + t), j & 1, abort_flag, p.status, 23);
+                        tc_fence_after();
+                        if (lane == 0) issue_s(t, s1);
+                        __syncwarp();
+                    }
+                }
+                for (int t = 0; t < 2; ++t) {
+                    mbar_wait(bar(kBarPFull + t), j & 1, abort_flag, p.status, 24);
+                    tc_fence_after();
+                    if (lane == 0) {
+                        uint64_t dv = make_smem_desc(smem_u32(smem + L::kV + s * L::kTileBytes), L::kRowBytes, 0);
+#pragma unroll
+                        for (int ks = 0; ks < kKvTile / 16; ++ks)
+                            mma_ts(tmem + 384 + t * 64, tmem + 256 + t * 64 + ks * 8,
+                                   advance_desc(dv, ks * 16 * L::kRowBytes), idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
+                        mma_commit(bar(kBarODone + t));
+                    }
+                    __syncwarp();
+                }
+                if (lane == 0) mma_commit(bar(kBarKvEmpty + s));
+                __syncwarp();
+            }
+        } else if (warp == 2) {
+            for (int j = 0; j < n_kv; ++j) {
+                const int s2 = j % kSpdStages;
+                mbar_wait(bar(kBarSpdEmpty + s2), ((j / kSpdStages) & 1) ^ 1, abort_flag, p.status, 30);
+                const int32_t kv0 = kv_begin + j * kKvTile;
+                const uint32_t dst0 = smem_u32(smem + L::kSpd + s2 * L::kSpdTileBytes);
+#pragma unroll 4
+                for (int i = 0; i < (kRowsPerCta * 8) / 32; ++i) {
+                    const int c = i * 32 + lane;
+                    const int r = c >> 3, cc = c & 7;
+                    const int64_t col = (int64_t)kv0 + cc * 16;
+                    const bool valid = (q0 + r < n_g) && (col < ld);
+                    const uint8_t* src = valid ? spd_g + (int64_t)(q0 + r) * ld + col : spd_g;
+                    cp_async_16(dst0 + r * 128 + ((cc ^ (r & 7)) << 4), src, valid ? 16u : 0u);
+                }
+                cp_async_mbar_arrive_noinc(bar(kBarSpdFull + s2));
+            }
+        }
+    } else {
+        // ================================= softmax warpgroups =================================
+        setmaxnreg_inc_232();
+        const int t = (warp >> 2) - 1;
+        const int r = tid & 127;
+        const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + t * 128 + lane_off;
+        const uint32_t tP = tmem + 256 + t * 64 + lane_off;
+        const uint32_t tO = tmem + 384 + t * 64 + lane_off;
+        const float c1 = p.c1;
+        float m = -INFINITY, l = 0.f;
+
+        for (int j = 0; j < n_kv; ++j) {
+            float x[128];
+            mbar_wait(bar(kBarSFull + t), j & 1, abort_flag, p.status, 40);
+            tc_fence_after();
+            {
+                uint32_t s0[32], s1[32], s2r[32], s3[32];
+                tmem_ld32(tS, s0);
+                tmem_ld32(tS + 32, s1);
+                tmem_ld32(tS + 64, s2r);
+                tmem_ld32(tS + 96, s3);
+                tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive(bar(kBarSFree + t));
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    x[i] = __uint_as_float(s0[i]);
+                    x[32 + i] = __uint_as_float(s1[i]);
+                    x[64 + i] = __uint_as_float(s2r[i]);
+                    x[96 + i] = __uint_as_float(s3[i]);
+                }
+            }
+            const int s2 = j % kSpdStages;
+            mbar_wait(bar(kBarSpdFull + s2), (j / kSpdStages) & 1, abort_flag, p.status, 41);
+            {
+                const uint8_t* srow = smem + L::kSpd + s2 * L::kSpdTileBytes + (t * 128 + r) * 128;
+#pragma unroll
+                for (int c8 = 0; c8 < 8; ++c8) {
+                    const uint4 w = *(const uint4*)(srow + ((c8 ^ (r & 7)) << 4));
+                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const uint32_t b = (ww[i >> 2] >> ((i & 3) * 8)) & 0xffu;
+                        x[c8 * 16 + i] = fmaf(x[c8 * 16 + i], c1, s_bias[b]);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarSpdEmpty + s2));
+
+            const int32_t kv0 = kv_begin + j * kKvTile;
+            if (kv0 + kKvTile > kv_end) {           // ragged last key tile
+                const int valid = kv_end - kv0;
+#pragma unroll
+                for (int i = 0; i < 128; ++i)
+                    if (i >= valid) x[i] = -INFINITY;
+            }
+            float mt = x[0];
+#pragma unroll
+            for (int i = 1; i + 1 < 128; i += 2) mt = max3(mt, x[i], x[i + 1]);
+            mt = fmaxf(mt, x[127]);
+            // The reference maximum is kept at an integer (log2 units): rescale factors are then
+            // exact powers of two and the bf16 mantissa of every P entry does not depend on how
+            // the keys are tiled or chunked, which keeps chunked and unchunked results within
+            // fp32 rounding of each other.
+            const float m_new = fmaxf(m, ceilf(mt));
+            const bool need = (m_new - m) > kRescaleThreshold;
+
+            if (j > 0) {
+                mbar_wait(bar(kBarODone + t), (j - 1) & 1, abort_flag, p.status, 42);
+                tc_fence_after();
+            }
+            if (__any_sync(0xffffffffu, need)) {
+                const float alpha = ex2_approx(m - m_new);
+                l *= alpha;
+                if (j > 0) {
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(tO + c * 32, o);
+                    }
+                }
+                m = m_new;
+            }
+            float sum = 0.f;
+            uint32_t pk0[32], pk1[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float a = ex2_approx(x[2 * i] - m), b = ex2_approx(x[2 * i + 1] - m);
+                sum += a + b;
+                pk0[i] = pack_bf16x2(a, b);
+            }
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float a = ex2_approx(x[64 + 2 * i] - m), b = ex2_approx(x[64 + 2 * i + 1] - m);
+                sum += a + b;
+                pk1[i] = pack_bf16x2(a, b);
+            }
+            l += sum;
+            tmem_st32(tP, pk0);
+            tmem_st32(tP + 32, pk1);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar(kBarPFull + t));
+        }
+
+        // ---- epilogue: O / l, LSE ----
+        mbar_wait(bar(kBarODone + t), (n_kv - 1) & 1, abort_flag, p.status, 43);
+        tc_fence_after();
+        const int32_t q = q0 + t * kRowsPerTile + r;
+        const float inv_l = 1.0f / l;
+        const float lse_nat = (m + log2f(l)) * kLn2;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(tO + c * 32, o);
+            tmem_wait_ld();
+            if (q < n_g) {
+                if (kPartial) {
+                    float4* dst = (float4*)(p.part_o + (((size_t)chunk * p.n_total + q) * p.n_heads + h) * D + c * 32);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        dst[i] = make_float4(__uint_as_float(o[4 * i]) * inv_l, __uint_as_float(o[4 * i + 1]) * inv_l,
+                                             __uint_as_float(o[4 * i + 2]) * inv_l, __uint_as_float(o[4 * i + 3]) * inv_l);
+                } else {
+                    uint4* dst = (uint4*)(p.out + ((size_t)(node0 + q) * p.n_heads + h) * D + c * 32);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(o[8 * i]) * inv_l, __uint_as_float(o[8 * i + 1]) * inv_l);
+                        v.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv_l, __uint_as_float(o[8 * i + 3]) * inv_l);
+                        v.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv_l, __uint_as_float(o[8 * i + 5]) * inv_l);
+                        v.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv_l, __uint_as_float(o[8 * i + 7]) * inv_l);
+                        dst[i] = v;
+                    }
+                }
+            }
+        }
+        if (q < n_g) {
+            if (kPartial) p.part_lse[((size_t)chunk * p.n_heads + h) * p.n_total + q] = lse_nat;
+            else p.lse[(size_t)h * p.n_total + node0 + q] = lse_nat;
+        }
+    }
+
+    // ---- teardown ----
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) __nanosleep(200000);    // let copies that may still be in flight land
+    if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+// Merge of per-chunk partials: lse = log sum_c exp(lse_c), out = sum_c exp(lse_c - lse) out_c.
+// One thread per (row, head, 4 channels).
+template <int D>
+__global__ void chunk_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse,
+                                   __nv_bfloat16* __restrict__ out, float* __restrict__ lse, float* __restrict__ lse_chunks,
+                                   int32_t n_total, int32_t n_heads, int32_t n_chunks)
+{
+    constexpr int kVec = D / 4;
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t n_rows = (size_t)n_total * n_heads;
+    if (idx >= n_rows * kVec) return;
+    const size_t rh = idx / kVec;
+    const int v = (int)(idx % kVec);
+    const int32_t row = (int32_t)(rh / n_heads), h = (int32_t)(rh % n_heads);
+    float mx = -INFINITY;
+    for (int c = 0; c < n_chunks; ++c) mx = fmaxf(mx, part_lse[((size_t)c * n_heads + h) * n_total + row]);
+    float den = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c = 0; c < n_chunks; ++c) {
+        const float lc = part_lse[((size_t)c * n_heads + h) * n_total + row];
+        if (v == 0 && lse_chunks) lse_chunks[((size_t)c * n_heads + h) * n_total + row] = lc;
+        if (lc == -INFINITY) continue;                      // empty chunk: weight 0 (no inf - inf)
+        const float w = exp2f((lc - mx) * kLog2e);
+        den += w;
+        const float4 o = *(const float4*)(part_o + (((size_t)c * n_total + row) * n_heads + h) * D + v * 4);
+        acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+    }
+    const float inv = 1.0f / den;
+    uint2 pk;
+    pk.x = pack_bf16x2(acc.x * inv, acc.y * inv);
+    pk.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+    *(uint2*)(out + ((size_t)row * n_heads + h) * D + v * 4) = pk;
+    if (v == 0) lse[(size_t)h * n_total + row] = mx + logf(den);
+}
+
+int32_t chunk_rows(int32_t n, int32_t n_chunks)
+{
+    int32_t w = (n + n_chunks - 1) / n_chunks;
+    return (w + kKvTile - 1) / kKvTile * kKvTile;
+}
+
+template <int D, bool kPartial>
+gt_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
+                     const gt_batch* batch, int grid_z, cudaStream_t s)
+{
+    auto kern = attn_fwd_kernel<D, kPartial>;
+    GT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kDynamic));
+    dim3 grid((unsigned)p.n_heads, (unsigned)((batch->max_seqlen + kRowsPerCta - 1) / kRowsPerCta), (unsigned)grid_z);
+    kern<<<grid, kFwdThreads, FwdSmem<D>::kDynamic, s>>>(tq, tk, tv, p);
+    GT_CUDA_TRY(cudaGetLastError());
+    return GT_OK;
+}
+
+gt_status check_fwd_args(const void* q, const void* k, const void* v, const uint8_t* spd, const int64_t* spd_offsets,
+                         const float* bias, const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                         void* out, float* lse)
+{
+    gt_status st = validate_attn_common(batch, n_heads, head_dim, max_dist, spd_offsets);
+    if (st != GT_OK) return st;
+    if (!q || !k || !v || !spd || !bias || !out || !lse) return GT_ERR_INVALID_ARG;
+    if (misaligned16(q) || misaligned16(k) || misaligned16(v) || misaligned16(spd) || misaligned16(out)) return GT_ERR_INVALID_ARG;
+    if (n_heads > 65535 || batch->n_graphs > 65535) return GT_ERR_UNSUPPORTED;
+    return GT_OK;
+}
+
+}  // namespace
+}  // namespace gt
+
+extern "C" size_t gt_biased_attn_fwd_workspace(const gt_batch* batch, int32_t n_heads, int32_t head_dim)
+{
+    (void)batch; (void)n_heads; (void)head_dim;
+    return gt::kHeaderBytes;
+}
+
+extern "C" gt_status gt_biased_attn_fwd(const void* q, const void* k, const void* v,
+                                        const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
+                                        const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                        void* out, float* lse,
+                                        void* workspace, size_t workspace_bytes, void* stream)
+{
+    using namespace gt;
+    gt_status st = check_fwd_args(q, k, v, spd, spd_offsets, bias, batch, n_heads, head_dim, max_dist, out, lse);
+    if (st != GT_OK) return st;
+    if (workspace == nullptr || workspace_bytes < kHeaderBytes || misaligned16(workspace)) return GT_ERR_WORKSPACE;
+    if (sm_count() <= 0) return GT_ERR_NO_DEVICE;
+    CUtensorMap tq, tk, tv;
+    if ((st = encode_thd_map(&tq, q, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&tk, k, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&tv, v, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
+    FwdParams p{};
+    p.spd = spd;
+    p.spd_offsets = batch->n_graphs > 1 ? spd_offsets : nullptr;
+    p.cu_seqlens = batch->n_graphs > 1 ? batch->cu_seqlens : nullptr;
+    p.bias = bias;
+    p.out = (__nv_bfloat16*)out;
+    p.lse = lse;
+    p.status = (uint32_t*)workspace;
+    p.n_total = batch->n_total;
+    p.n_heads = n_heads;
+    p.n_buckets = max_dist + 2;
+    p.c1 = kLog2e / sqrtf((float)head_dim);
+    cudaStream_t s = (cudaStream_t)stream;
+    return head_dim == 64 ? launch_fwd<64, false>(tq, tk, tv, p, batch, batch->n_graphs, s)
+                          : launch_fwd<32, false>(tq, tk, tv, p, batch, batch->n_graphs, s);
+}
+
+extern "C" size_t gt_biased_attn_fwd_chunked_workspace(const gt_batch* batch, int32_t n_heads, int32_t head_dim,
+                                                       int32_t n_kv_chunks)
+{
+    if (gt::validate_batch(batch) != GT_OK || n_heads < 1 || n_kv_chunks < 1) return 0;
+    size_t rows = (size_t)batch->n_total * n_heads;
+    return gt::kHeaderBytes + (size_t)n_kv_chunks * rows * head_dim * sizeof(float)
+         + gt::align_up((size_t)n_kv_chunks * rows * sizeof(float), 256);
+}
+
+extern "C" gt_status gt_biased_attn_fwd_chunked(const void* q, const void* k, const void* v,
+                                                const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
+                                                const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                                void* out, float* lse, int32_t n_kv_chunks, float* lse_chunks,
+                                                void* workspace, size_t workspace_bytes, void* stream)
+{
+    using namespace gt;
+    gt_status st = check_fwd_args(q, k, v, spd, spd_offsets, bias, batch, n_heads, head_dim, max_dist, out, lse);
+    if (st != GT_OK) return st;
+    if (n_kv_chunks < 1 || n_kv_chunks > 65535) return GT_ERR_INVALID_ARG;
+    if (batch->n_graphs != 1) return GT_ERR_UNSUPPORTED;
+    const size_t need = gt_biased_attn_fwd_chunked_workspace(batch, n_heads, head_dim, n_kv_chunks);
+    if (workspace == nullptr || workspace_bytes < need || misaligned16(workspace)) return GT_ERR_WORKSPACE;
+    if (sm_count() <= 0) return GT_ERR_NO_DEVICE;
+    CUtensorMap tq, tk, tv;
+    if ((st = encode_thd_map(&tq, q, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&tk, k, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&tv, v, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
+    const size_t rows = (size_t)batch->n_total * n_heads;
+    uint8_t* ws = (uint8_t*)workspace;
+    FwdParams p{};
+    p.spd = spd;
+    p.bias = bias;
+    p.part_lse = (float*)(ws + kHeaderBytes);
+    p.part_o = (float*)(ws + kHeaderBytes + align_up((size_t)n_kv_chunks * rows * sizeof(float), 256));
+    p.status = (uint32_t*)workspace;
+    p.n_total = batch->n_total;
+    p.n_heads = n_heads;
+    p.n_buckets = max_dist + 2;
+    p.kv_chunk_rows = chunk_rows(batch->n_total, n_kv_chunks);
+    p.c1 = kLog2e / sqrtf((float)head_dim);
+    cudaStream_t s = (cudaStream_t)stream;
+    st = head_dim == 64 ? launch_fwd<64, true>(tq, tk, tv, p, batch, n_kv_chunks, s)
+                        : launch_fwd<32, true>(tq, tk, tv, p, batch, n_kv_chunks, s);
+    if (st != GT_OK) return st;
+    const size_t n_thr = rows * (head_dim / 4);
+    const unsigned blocks = (unsigned)((n_thr + 255) / 256);
+    if (head_dim == 64)
+        chunk_merge_kernel<64><<<blocks, 256, 0, s>>>(p.part_o, p.part_lse, (__nv_bfloat16*)out, lse, lse_chunks,
+                                                      batch->n_total, n_heads, n_kv_chunks);
+    else
+        chunk_merge_kernel<32><<<blocks, 256, 0, s>>>(p.part_o, p.part_lse, (__nv_bfloat16*)out, lse, lse_chunks,
+                                                      batch->n_total, n_heads, n_kv_chunks);
+    GT_CUDA_TRY(cudaGetLastError());
+    return GT_OK;
+}

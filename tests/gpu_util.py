@@ -40,3 +40,51 @@ def gpu_spd(w: wl.Workload, dev="cuda") -> torch.Tensor:
 def rel_l2(x: np.ndarray, r: np.ndarray) -> float:
     den = float(np.linalg.norm(r.reshape(-1)))
     return float(np.linalg.norm((x - r).reshape(-1))) / (den if den > 0 else 1.0)
+
+
+class DeviceCase:
+    """A workload moved to the device, with the SPD either from the oracle (default, so that
+    attention parity does not depend on the SPD kernel) or from gt_spd_build."""
+
+    def __init__(self, w: wl.Workload, spd_from_gpu: bool = False, dev="cuda"):
+        from oracle import spd as ospd
+        self.w = w
+        b = w.batch
+        t = w.tensors()
+        self.batch = device_batch(b, dev)
+        self.spd_host = ospd.spd_packed(b.row_ptr, b.col_idx, b.cu_seqlens, w.max_dist)
+        self.spd = gpu_spd(w, dev) if spd_from_gpu else torch.from_numpy(self.spd_host).to(dev)
+        self.q, self.k, self.v, self.dout = (bf16_tensor(x, dev) for x in (t.q, t.k, t.v, t.dout))
+        self.bias = torch.tensor(t.bias, device=dev)
+        self.T, self.H, self.d = t.q.shape
+
+    def host_f64(self):
+        t = self.w.tensors()
+        f = wl.bf16_bits_to_f64
+        return f(t.q), f(t.k), f(t.v), f(t.dout), t.bias.astype(np.float64)
+
+    def forward(self):
+        out = torch.full((self.T, self.H, self.d), float("nan"), dtype=torch.bfloat16, device=self.q.device)
+        lse = torch.full((self.H, self.T), float("nan"), dtype=torch.float32, device=self.q.device)
+        ws = gt.gt_biased_attn_fwd(self.q, self.k, self.v, self.spd, self.bias, self.batch, self.w.max_dist, out, lse)
+        gt.gt_check(ws)
+        return out, lse
+
+    def forward_chunked(self, n_chunks, want_chunk_lse=False):
+        out = torch.full((self.T, self.H, self.d), float("nan"), dtype=torch.bfloat16, device=self.q.device)
+        lse = torch.full((self.H, self.T), float("nan"), dtype=torch.float32, device=self.q.device)
+        cl = torch.full((n_chunks, self.H, self.T), float("nan"), dtype=torch.float32,
+                        device=self.q.device) if want_chunk_lse else None
+        ws = gt.gt_biased_attn_fwd_chunked(self.q, self.k, self.v, self.spd, self.bias, self.batch, self.w.max_dist,
+                                           out, lse, n_chunks, cl)
+        gt.gt_check(ws)
+        return out, lse, cl
+
+    def backward(self, out, lse, dout=None):
+        dout = self.dout if dout is None else dout
+        dq, dk, dv = (torch.full_like(self.q, float("nan")) for _ in range(3))
+        dbias = torch.full_like(self.bias, float("nan"))
+        ws = gt.gt_biased_attn_bwd(self.q, self.k, self.v, out, dout, lse, self.spd, self.bias, self.batch,
+                                   self.w.max_dist, dq, dk, dv, dbias)
+        gt.gt_check(ws)
+        return dq, dk, dv, dbias

@@ -1,0 +1,102 @@
+"""gt_biased_attn_bwd vs the fp64 oracle's analytic backward, through the C ABI.
+
+Tolerance (bf16 inputs, fp32 accumulation): relative-L2 error <= 2e-2 for each of dQ, dK, dV
+and dBias over the whole tensor."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as oattn
+from paper_2609_34420_b200 import workloads as wl
+
+from gpu_util import DeviceCase, rel_l2, to_f64
+
+pytestmark = pytest.mark.gpu
+
+GRAD_REL_L2 = 2e-2
+
+
+def oracle_backward(case: DeviceCase):
+    q, k, v, do, b = case.host_f64()
+    bt = case.w.batch
+    return oattn.backward_batch(q, k, v, do, case.spd_host, bt.spd_offsets, bt.cu_seqlens, b)
+
+
+def check_backward(w: wl.Workload):
+    case = DeviceCase(w)
+    out, lse = case.forward()
+    dq, dk, dv, db = case.backward(out, lse)
+    rdq, rdk, rdv, rdb = oracle_backward(case)
+    errs = {}
+    for name, got, ref in (("dq", dq, rdq), ("dk", dk, rdk), ("dv", dv, rdv), ("dbias", db, rdb)):
+        g = to_f64(got)
+        assert np.isfinite(g).all(), name
+        errs[name] = rel_l2(g, ref)
+    assert all(e <= GRAD_REL_L2 for e in errs.values()), errs
+    # softmax shift invariance: every row of dS sums to zero, hence sum_b dB[h,b] = 0
+    # (up to the bf16 rounding of the stored O that enters Delta = rowsum(dO * O))
+    dbf = to_f64(db)
+    floor = 2.0 ** -7 * np.abs(to_f64(out) * to_f64(case.dout)).sum(axis=(0, 2))
+    assert (np.abs(dbf.sum(axis=1)) <= 2e-3 * np.abs(dbf).sum(axis=1) + floor).all(), dbf.sum(axis=1)
+    return case, errs
+
+
+@pytest.mark.parametrize("n", [1, 2, 17, 127, 128, 129, 255, 256, 300, 513])
+@pytest.mark.parametrize("d", [32, 64])
+def test_tails(n, d):
+    check_backward(wl.small_workload([n], 2, d, 5, seed=n + d, avg_degree=2.0))
+
+
+@pytest.mark.parametrize("d", [32, 64])
+def test_directed_graph_asymmetric_spd(d):
+    check_backward(wl.small_workload([333], 3, d, 6, seed=5, avg_degree=1.8, directed=True))
+
+
+@pytest.mark.parametrize("d", [32, 64])
+def test_varlen_batch_shares_one_bias_table(d):
+    check_backward(wl.small_workload([5, 130, 1, 256, 300, 64, 2, 97], 3, d, 6, seed=d, avg_degree=1.7))
+
+
+def test_many_buckets_uses_shared_bins():
+    check_backward(wl.small_workload([400], 2, 64, 60, seed=8, avg_degree=1.05))
+
+
+def test_max_dist_254():
+    check_backward(wl.small_workload([300], 2, 32, 254, seed=9, avg_degree=1.0))
+
+
+@pytest.mark.parametrize("name", ["tiny_er256", "tiny_er256_sparse", "ba4096", "varlen_rgg64"])
+def test_named_workloads(name):
+    check_backward(wl.make_workload(name))
+
+
+def test_unused_buckets_get_exact_zero_and_outputs_are_overwritten():
+    w = wl.make_workload("ba4096")           # distances stop near 5 of 18 buckets
+    case = DeviceCase(w)
+    out, lse = case.forward()
+    _, _, _, db = case.backward(out, lse)
+    present = np.bincount(case.spd_host.reshape(4096, -1)[:, :4096].reshape(-1), minlength=256)[:w.n_buckets] > 0
+    assert (to_f64(db)[:, ~present] == 0).all()
+    dq2, dk2, dv2, db2 = case.backward(out, lse)      # second call on fresh NaN-filled outputs: no accumulation
+    assert np.isfinite(to_f64(dq2)).all() and rel_l2(to_f64(db2), to_f64(db)) < 1e-5
+
+
+def test_rows_with_zero_dout_do_not_contribute():
+    """dK, dV, dB depend only on query rows whose dO is non-zero (the row-slab protocol used
+    to check the largest workload against a partial oracle relies on this)."""
+    w = wl.small_workload([600], 2, 64, 6, seed=12, avg_degree=2.0)
+    case = DeviceCase(w)
+    out, lse = case.forward()
+    rows = np.sort(np.random.default_rng(0).choice(600, 100, replace=False))
+    do_masked = torch.zeros_like(case.dout)
+    do_masked[rows] = case.dout[rows]
+    dq, dk, dv, db = case.backward(out, lse, dout=do_masked)
+    q, k, v, do, b = case.host_f64()
+    spd = case.spd_host.reshape(600, -1)
+    rdq, rdk, rdv, rdb = oattn.backward_single(q, k, v, do, spd, b, rows=rows)
+    assert rel_l2(to_f64(dq)[rows], rdq) <= GRAD_REL_L2
+    assert rel_l2(to_f64(dk), rdk) <= GRAD_REL_L2 and rel_l2(to_f64(dv), rdv) <= GRAD_REL_L2
+    assert rel_l2(to_f64(db), rdb) <= GRAD_REL_L2
+    mask = np.ones(600, bool)
+    mask[rows] = False
+    assert (to_f64(dq)[mask] == 0).all()

@@ -1,0 +1,118 @@
+"""gt_biased_attn_fwd / gt_biased_attn_fwd_chunked vs the fp64 oracle, through the C ABI.
+
+Tolerances (bf16 inputs, fp32 accumulation, bf16 output): output max-abs error <= 1e-2,
+LSE max-abs error <= 1e-3, chunked vs unchunked output relative-L2 <= 1e-3."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as oattn
+from paper_2609_34420_b200 import workloads as wl
+
+from gpu_util import DeviceCase, rel_l2, to_f64
+
+pytestmark = pytest.mark.gpu
+
+O_MAX_ABS = 1e-2
+LSE_MAX_ABS = 1e-3
+CHUNK_REL_L2 = 1e-3
+
+
+def oracle_forward(case: DeviceCase):
+    q, k, v, _, b = case.host_f64()
+    bt = case.w.batch
+    return oattn.forward_batch(q, k, v, case.spd_host, bt.spd_offsets, bt.cu_seqlens, b)
+
+
+def check_forward(w: wl.Workload, strict: bool = False):
+    case = DeviceCase(w)
+    out, lse = case.forward()
+    ro, rl = oracle_forward(case)
+    o = to_f64(out)
+    assert np.isfinite(o).all() and np.isfinite(to_f64(lse)).all()
+    # 1e-2 absolute, or one bf16 ulp (2^-7 relative) where that is larger: a bf16 output cannot
+    # be closer than half an ulp, which alone exceeds 1e-2 once |O| > 2.56 (only tiny graphs and
+    # the adversarial peaked-softmax cases get there; the named workloads stay below 1e-2)
+    tol = O_MAX_ABS if strict else np.maximum(O_MAX_ABS, np.abs(ro) * 2.0 ** -7)
+    assert (np.abs(o - ro) <= tol).all(), np.abs(o - ro).max()
+    assert np.abs(to_f64(lse) - rl).max() <= LSE_MAX_ABS, np.abs(to_f64(lse) - rl).max()
+    return case, out, lse
+
+
+@pytest.mark.parametrize("n", [1, 2, 17, 127, 128, 129, 255, 256, 257, 300, 513])
+@pytest.mark.parametrize("d", [32, 64])
+def test_tails(n, d):
+    check_forward(wl.small_workload([n], 2, d, 5, seed=n + d, avg_degree=2.0))
+
+
+@pytest.mark.parametrize("d", [32, 64])
+def test_directed_graph_asymmetric_spd(d):
+    check_forward(wl.small_workload([200], 3, d, 6, seed=5, avg_degree=1.8, directed=True))
+
+
+@pytest.mark.parametrize("d", [32, 64])
+def test_varlen_batch(d):
+    check_forward(wl.small_workload([5, 130, 1, 256, 300, 64, 2, 97], 3, d, 6, seed=d, avg_degree=1.7))
+
+
+def test_large_bias_spread_and_max_dist_254():
+    w = wl.small_workload([400], 2, 64, 254, seed=8, avg_degree=1.1)
+    w.tensors().bias[:] *= 12.0           # forces many running-max rescales
+    check_forward(w)
+
+
+@pytest.mark.parametrize("name", ["tiny_er256", "tiny_er256_sparse", "ba4096", "varlen_rgg64"])
+def test_named_workloads(name):
+    check_forward(wl.make_workload(name), strict=True)     # the stated 1e-2 bound, no allowance
+
+
+def test_forward_is_deterministic():
+    case = DeviceCase(wl.make_workload("ba4096"))
+    a, la = case.forward()
+    b, lb = case.forward()
+    assert torch.equal(a, b) and torch.equal(la, lb)
+
+
+@pytest.mark.parametrize("n,chunks", [(300, 1), (300, 2), (300, 3), (1000, 8), (129, 4), (4096, 8)])
+def test_chunked_matches_unchunked_and_oracle(n, chunks):
+    w = wl.small_workload([n], 2, 64, 6, seed=n, avg_degree=2.0, directed=True)    # asymmetric SPD
+    case, out, lse = check_forward(w)
+    oc, lc, cl = case.forward_chunked(chunks, want_chunk_lse=True)
+    assert rel_l2(to_f64(oc), to_f64(out)) <= CHUNK_REL_L2
+    ro, rl = oracle_forward(case)
+    assert (np.abs(to_f64(oc) - ro) <= np.maximum(O_MAX_ABS, np.abs(ro) * 2.0 ** -7)).all()
+    assert np.abs(to_f64(lc) - rl).max() <= LSE_MAX_ABS
+    # per-chunk statistic against its definition (bias taken at the global column)
+    width = -(-((n + chunks - 1) // chunks) // 128) * 128
+    bounds = [(min(c * width, n), min((c + 1) * width, n)) for c in range(chunks)]
+    q, k, _, _, b = case.host_f64()
+    ref_cl = oattn.chunk_lse(q, k, case.spd_host.reshape(n, -1), b, bounds)
+    got_cl = to_f64(cl)
+    empty = np.isneginf(ref_cl)
+    assert (np.isneginf(got_cl) == empty).all()
+    assert np.abs(got_cl[~empty] - ref_cl[~empty]).max() <= LSE_MAX_ABS
+
+
+def test_chunked_d32_and_large_bias_spread():
+    w = wl.small_workload([700], 4, 32, 6, seed=3, avg_degree=2.0)
+    w.tensors().bias[:] *= 10.0
+    case, out, lse = check_forward(w)
+    oc, lc, _ = case.forward_chunked(5)
+    assert rel_l2(to_f64(oc), to_f64(out)) <= CHUNK_REL_L2
+    assert np.abs(to_f64(lc) - to_f64(lse)).max() <= LSE_MAX_ABS
+
+
+def test_rejects_unsupported_shapes():
+    from paper_2609_34420_b200 import binding as gt
+    case = DeviceCase(wl.small_workload([64], 2, 32, 4, seed=0))
+    q16 = case.q[:, :, :16].contiguous()
+    out = torch.empty_like(q16)
+    lse = torch.empty(2, 64, device="cuda")
+    with pytest.raises(gt.GtError) as e:
+        gt.gt_biased_attn_fwd(q16, q16, q16, case.spd, case.bias, case.batch, 4, out, lse)
+    assert e.value.status == 2
+    multi = DeviceCase(wl.small_workload([64, 64], 2, 32, 4, seed=0))
+    o2, l2 = torch.empty_like(multi.q), torch.empty(2, 128, device="cuda")
+    with pytest.raises(gt.GtError) as e:
+        gt.gt_biased_attn_fwd_chunked(multi.q, multi.k, multi.v, multi.spd, multi.bias, multi.batch, 4, o2, l2, 2)
+    assert e.value.status == 2
