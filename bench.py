@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Benchmark of the biased graph-attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step = one pass of the whole hot path over one seeded synthetic batch:
+gt_spd_build -> gt_biased_attn_fwd -> gt_biased_attn_bwd -> gt_biased_attn_fwd_chunked.
+The headline metric is forward+backward attention TFLOP/s (14*H*d*sum n_g^2 FLOPs per step
+divided by the forward+backward time inside the step, CUDA events); the SPD build GB/s, the
+chunked forward and the whole-step time are reported beside it.  With N > 1 (torchrun) every
+rank processes its own batch: weak scaling over independent batches, no data-path collective.
+
+`--impl reference` times the CPU oracle (fp64, host cores) on a bounded row sample of the
+same workload and prints the same JSON line with "impl": "reference".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_34420_b200 import workloads as wl  # noqa: E402
+
+METRIC = "fwd+bwd biased-attention TFLOP/s"
+UNIT = "TFLOP/s"
+DEFAULT_WORKLOAD = "powerlaw64k"
+ORACLE_SAMPLE_ROWS = 256
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the backward kernel, from the ncu
+# capture summarised under profiles/ (captured on a smaller graph and scaled by N^2); None until measured.
+BWD_KERNEL_DRAM_BYTES_PER_N2 = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return json.load(fh), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def host_cores() -> int:
+    return len(os.sched_getaffinity(0))
+
+
+# --------------------------------------------------------------------------------------
+# CPU oracle arm (also the cpu_baseline of the CUDA arm)
+# --------------------------------------------------------------------------------------
+def oracle_sample(w: wl.Workload, n_rows: int, seed: int = 123):
+    """Time the oracle (BFS rows + fp64 forward + analytic backward) on `n_rows` seeded
+    query rows of graph 0 of the workload.  Returns (seconds, flops_equivalent, spd_seconds)."""
+    from oracle import attention as oattn
+    from oracle import spd as ospd
+
+    rp, ci = w.batch.graph_csr(0)
+    n = len(rp) - 1
+    t = w.tensors()
+    a, b = int(w.batch.cu_seqlens[0]), int(w.batch.cu_seqlens[1])
+    f = wl.bf16_bits_to_f64
+    q, k, v, do = f(t.q[a:b]), f(t.k[a:b]), f(t.v[a:b]), f(t.dout[a:b])
+    bias = t.bias.astype(np.float64)
+    rows = np.sort(np.random.default_rng(seed).choice(n, size=min(n_rows, n), replace=False))
+    ospd.spd_rows(rp, ci, w.max_dist, rows[:1])                 # build/load the C library outside the timing
+    t0 = time.perf_counter()
+    spd = ospd.spd_rows(rp, ci, w.max_dist, rows)
+    t1 = time.perf_counter()
+    oattn.forward_single(q, k, v, spd, bias, rows=rows, compact_spd=True)
+    oattn.backward_single(q, k, v, do, spd, bias, rows=rows, compact_spd=True)
+    t2 = time.perf_counter()
+    flops = 14.0 * w.n_heads * w.head_dim * len(rows) * n
+    return t2 - t1, flops, t1 - t0, len(rows), n
+
+
+def run_reference(args) -> int:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    w = wl.make_workload(args.workload)
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(w, 32)
+    times, flops = [], 0.0
+    for _ in range(args.steps):
+        sec, flops, spd_sec, n_rows, n = oracle_sample(w, ORACLE_SAMPLE_ROWS)
+        times.append(sec)
+    ms = 1e3 * sum(times) / len(times)
+    value = flops / (ms * 1e-3) / 1e12
+    sample = f"{n_rows} seeded query rows of {n} (full key range), fp64 forward + analytic backward per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "note": w.note, "n_heads": w.n_heads, "head_dim": w.head_dim,
+                   "max_dist": w.max_dist, "n_total": w.batch.n_total},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_cores(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# --------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_uuid: str):
+        self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={device_uuid}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.tmp.close()
+        os.unlink(self.tmp.name)
+        busy = [x for x in sm if x > 0]
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------
+# CUDA arm
+# --------------------------------------------------------------------------------------
+def run_cuda(args) -> int:
+    import torch
+
+    from paper_2609_34420_b200 import binding as gt
+    from paper_2609_34420_b200 import dist_util
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
+    rank, local_rank, world = dist_util.env_world()
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    dist_util.init_process_group("nccl")
+    gt.lib()
+
+    w = wl.make_workload(args.workload, seed=dist_util.shard_seed(0, rank))
+    b, t = w.batch, w.tensors()
+    T, H, d, D = b.n_total, w.n_heads, w.head_dim, w.max_dist
+    single = b.n_graphs == 1
+    n_chunks = w.n_kv_chunks if single else 1
+
+    def dev_bf16(bits):
+        return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    # ---- device-resident inputs ----
+    rp = torch.from_numpy(b.row_ptr).to(dev)
+    ci = torch.from_numpy(b.col_idx).to(dev)
+    batch = gt.Batch(T, b.n_graphs, b.max_seqlen,
+                     None if single else torch.from_numpy(b.cu_seqlens).to(dev),
+                     None if single else torch.from_numpy(b.spd_offsets).to(dev))
+    q, k, v, do = dev_bf16(t.q), dev_bf16(t.k), dev_bf16(t.v), dev_bf16(t.dout)
+    bias = torch.from_numpy(t.bias).to(dev)
+    spd = torch.empty(b.spd_bytes, dtype=torch.uint8, device=dev)
+    out, dq, dk, dv = (torch.empty_like(q) for _ in range(4))
+    out_c = torch.empty_like(q)
+    lse = torch.empty(H, T, dtype=torch.float32, device=dev)
+    lse_c = torch.empty_like(lse)
+    dbias = torch.empty_like(bias)
+    ws_spd = gt._workspace(gt.gt_spd_build_workspace(batch, ci.numel(), D), dev)
+    ws_fwd = gt._workspace(gt.gt_biased_attn_fwd_workspace(batch, H, d), dev)
+    ws_bwd = gt._workspace(gt.gt_biased_attn_bwd_workspace(batch, H, d, D), dev)
+    ws_chk = gt._workspace(gt.gt_biased_attn_fwd_chunked_workspace(batch, H, d, n_chunks), dev) if single else None
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def step(marks=None):
+        if marks is not None:
+            marks[0].record()
+        gt.gt_spd_build(rp, ci, batch, D, spd, ws_spd)
+        if marks is not None:
+            marks[1].record()
+        gt.gt_biased_attn_fwd(q, k, v, spd, bias, batch, D, out, lse, ws_fwd)
+        if marks is not None:
+            marks[2].record()
+        gt.gt_biased_attn_bwd(q, k, v, out, do, lse, spd, bias, batch, D, dq, dk, dv, dbias, ws_bwd)
+        if marks is not None:
+            marks[3].record()
+        if single:
+            gt.gt_biased_attn_fwd_chunked(q, k, v, spd, bias, batch, D, out_c, lse_c, n_chunks, None, ws_chk)
+        if marks is not None:
+            marks[4].record()
+
+    kernels_per_step = 2 + 1 + 3 + (2 if single else 0)     # spd(setup,bfs) fwd bwd(pre,main,finalize) chunked(partial,merge)
+
+    for _ in range(max(args.warmup, 0)):
+        step()
+    torch.cuda.synchronize()
+    for wsx in (ws_spd, ws_fwd, ws_bwd) + ((ws_chk,) if single else ()):
+        gt.gt_check(wsx)
+
+    # ---- timed region ----
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid)) if rank == 0 else None
+    marks = [[ev() for _ in range(5)] for _ in range(args.steps)]
+    e0, e1 = ev(), ev()
+    dist_util.barrier(dev)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(args.steps):
+        step(marks[i])
+    e1.record()
+    torch.cuda.synchronize()
+    dist_util.barrier(dev)
+    clocks = sampler.stop() if sampler else None
+    for wsx in (ws_spd, ws_fwd, ws_bwd) + ((ws_chk,) if single else ()):
+        gt.gt_check(wsx)
+
+    total_ms = e0.elapsed_time(e1)
+    ph = np.array([[m[j].elapsed_time(m[j + 1]) for j in range(4)] for m in marks])       # [K, 4]
+    spd_ms, fwd_ms, bwd_ms, chk_ms = (float(x) for x in ph.mean(axis=0))
+    f_fwd, f_bwd = w.attn_flops()
+    ms_step, _ = dist_util.aggregate(total_ms / args.steps, 0.0, dev)
+    fb_ms, flops_all = dist_util.aggregate(fwd_ms + bwd_ms, f_fwd + f_bwd, dev)
+    value = flops_all / (fb_ms * 1e-3) / 1e12
+    spd_alg_bytes = float(b.spd_bytes + 4 * (T + 1) + 4 * ci.numel())
+
+    # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region ----
+    host_in = {name: x.cpu().pin_memory() for name, x in
+               (("q", q), ("k", k), ("v", v), ("do", do), ("bias", bias), ("rp", rp), ("ci", ci))}
+    host_out = {name: torch.empty_like(x, device="cpu").pin_memory() for name, x in
+                (("out", out), ("lse", lse), ("dq", dq), ("dk", dk), ("dv", dv), ("dbias", dbias))}
+    h2d = sum(x.numel() * x.element_size() for x in host_in.values())
+    d2h = sum(x.numel() * x.element_size() for x in host_out.values())
+
+    def e2e_step():
+        q.copy_(host_in["q"], non_blocking=True)
+        k.copy_(host_in["k"], non_blocking=True)
+        v.copy_(host_in["v"], non_blocking=True)
+        do.copy_(host_in["do"], non_blocking=True)
+        bias.copy_(host_in["bias"], non_blocking=True)
+        rp.copy_(host_in["rp"], non_blocking=True)
+        ci.copy_(host_in["ci"], non_blocking=True)
+        gt.gt_spd_build(rp, ci, batch, D, spd, ws_spd)
+        gt.gt_biased_attn_fwd(q, k, v, spd, bias, batch, D, out, lse, ws_fwd)
+        gt.gt_biased_attn_bwd(q, k, v, out, do, lse, spd, bias, batch, D, dq, dk, dv, dbias, ws_bwd)
+        for name, src in (("out", out), ("lse", lse), ("dq", dq), ("dk", dk), ("dv", dv), ("dbias", dbias)):
+            host_out[name].copy_(src, non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize()
+    n_e2e = max(1, min(args.steps, 3))
+    dist_util.barrier(dev)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(n_e2e):
+        e2e_step()
+    e1.record()
+    torch.cuda.synchronize()
+    dist_util.barrier(dev)
+    e2e_ms, e2e_flops = dist_util.aggregate(e0.elapsed_time(e1) / n_e2e, f_fwd + f_bwd, dev)
+    e2e_value = e2e_flops / (e2e_ms * 1e-3) / 1e12
+
+    if rank != 0:
+        return 0
+
+    peaks, peak_kind = load_peaks()
+    bwd_tflops = f_bwd / (bwd_ms * 1e-3) / 1e12
+    peak_tf = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    sum_n2 = float(b.sum_n2)
+    roofline = {
+        "kernel": "attn_bwd_kernel", "bound": "tensor", "achieved": bwd_tflops, "peak": peak_tf, "unit": "TFLOP/s",
+        "frac": bwd_tflops / peak_tf, "peak_kind": f"bf16_tflops_sustained of {peak_kind} (kernel timed inside a long step)",
+        "frac_of_burst_peak": bwd_tflops / float(peaks["bf16_tflops"]),
+        "traffic": None if BWD_KERNEL_DRAM_BYTES_PER_N2 is None else BWD_KERNEL_DRAM_BYTES_PER_N2 * sum_n2,
+        "flops_per_launch": f_bwd, "ms_per_launch": bwd_ms,
+    }
+    roofline_spd = {
+        "kernel": "spd_bfs_kernel", "bound": "hbm", "achieved": spd_alg_bytes / (spd_ms * 1e-3) / 1e9,
+        "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
+        "frac": spd_alg_bytes / (spd_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"]), "peak_kind": f"hbm_gbs of {peak_kind}",
+        "bytes_per_launch": spd_alg_bytes, "ms_per_launch": spd_ms, "traffic": None,
+    }
+
+    cpu_baseline = None
+    if world == 1:
+        sec, o_flops, spd_sec, n_rows, n0 = oracle_sample(w, ORACLE_SAMPLE_ROWS)
+        cpu_baseline = {"value": o_flops / sec / 1e12, "unit": UNIT, "cores": host_cores(), "kind": "oracle",
+                        "sample": f"{n_rows} seeded query rows of {n0} (full key range): fp64 forward + analytic backward "
+                                  f"in {sec:.2f} s; BFS rows of the same sources in {spd_sec:.3f} s (BLAS steps threaded, "
+                                  "elementwise steps single-threaded numpy)"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "note": w.note, "n_total": T, "n_graphs": b.n_graphs, "n_heads": H,
+                   "head_dim": d, "max_dist": D, "n_kv_chunks": n_chunks, "nnz": int(ci.numel()),
+                   "step": "spd_build + fwd + bwd + chunked fwd", "parallelism": f"dp{world} (independent batches)",
+                   "l2": "inputs larger than L2: the SPD matrix (%.2f GB) is rebuilt and re-streamed every step" % (b.spd_bytes / 1e9)},
+        "phases_ms": {"spd_build": spd_ms, "fwd": fwd_ms, "bwd": bwd_ms, "fwd_chunked": chk_ms if single else None},
+        "fwd_tflops": f_fwd / (fwd_ms * 1e-3) / 1e12, "bwd_tflops": bwd_tflops,
+        "fwd_chunked_tflops": (f_fwd / (chk_ms * 1e-3) / 1e12) if single else None,
+        "spd_build_gbs": roofline_spd["achieved"],
+        "pct_of_bf16_peak": {"burst": 100 * value / world / float(peaks["bf16_tflops"]),
+                             "sustained": 100 * value / world / peak_tf, "nominal_2250": 100 * value / world / 2250.0},
+        "roofline": roofline, "roofline_spd": roofline_spd, "cpu_baseline": cpu_baseline,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "ms_per_step": e2e_ms, "steps": n_e2e, "includes": "H2D of Q,K,V,dO,bias,CSR; spd_build+fwd+bwd; D2H of O,LSE,dQ,dK,dV,dBias"},
+        "gpu_launches": kernels_per_step * args.steps, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main() -> int:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(wl.WORKLOAD_NAMES) + ["tiny_er256_sparse"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_cuda(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

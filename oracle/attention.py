@@ -56,16 +56,17 @@ def _softmax_rows(s: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
 
 
 def forward_single(q: np.ndarray, k: np.ndarray, v: np.ndarray, spd: np.ndarray, bias: np.ndarray,
-                   rows: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray]:
+                   rows: Optional[np.ndarray] = None, compact_spd: bool = False) -> Tuple[np.ndarray, np.ndarray]:
     """One graph.  q,k,v fp64 [n,H,d]; spd uint8 [n, >=n]; bias fp64 [H,nb].
-    Returns O fp64 [r,H,d] and LSE fp64 [H,r] for the selected query rows (default all)."""
+    Returns O fp64 [r,H,d] and LSE fp64 [H,r] for the selected query rows (default all).
+    With compact_spd, spd holds only the selected rows: spd[i] is the SPD row of rows[i]."""
     n, H, d = q.shape
     rows = np.arange(n) if rows is None else np.asarray(rows)
     out = np.zeros((len(rows), H, d))
     lse = np.zeros((H, len(rows)))
     for r0 in range(0, len(rows), ROW_BLOCK):
         rr = rows[r0:r0 + ROW_BLOCK]
-        spd_rows = spd[rr, :n]
+        spd_rows = spd[r0:r0 + len(rr), :n] if compact_spd else spd[rr, :n]
         for h in range(H):
             p, l = _softmax_rows(_scores(q[rr, h, :], k[:, h, :], spd_rows, bias[h]))
             out[r0:r0 + len(rr), h, :] = p @ v[:, h, :]
@@ -74,7 +75,7 @@ def forward_single(q: np.ndarray, k: np.ndarray, v: np.ndarray, spd: np.ndarray,
 
 
 def backward_single(q: np.ndarray, k: np.ndarray, v: np.ndarray, dout: np.ndarray, spd: np.ndarray,
-                    bias: np.ndarray, rows: Optional[np.ndarray] = None):
+                    bias: np.ndarray, rows: Optional[np.ndarray] = None, compact_spd: bool = False):
     """One graph.  dout fp64 [n,H,d] (only the selected rows are read).  Returns
     (dQ [r,H,d] for the selected rows, dK [n,H,d], dV [n,H,d], dB [H,nb]) where dK, dV, dB
     are the sums over the selected query rows only (all rows by default)."""
@@ -88,7 +89,7 @@ def backward_single(q: np.ndarray, k: np.ndarray, v: np.ndarray, dout: np.ndarra
     inv_sqrt_d = 1.0 / np.sqrt(float(d))
     for r0 in range(0, len(rows), ROW_BLOCK):
         rr = rows[r0:r0 + ROW_BLOCK]
-        spd_rows = spd[rr, :n]
+        spd_rows = spd[r0:r0 + len(rr), :n] if compact_spd else spd[rr, :n]
         idx = spd_rows.astype(np.int64).reshape(-1)
         for h in range(H):
             p, _ = _softmax_rows(_scores(q[rr, h, :], k[:, h, :], spd_rows, bias[h]))

@@ -38,6 +38,9 @@ def _load():
         lib.oracle_spd_bfs.restype = ctypes.c_int
         lib.oracle_spd_bfs.argtypes = [ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p,
                                        ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p]
+        lib.oracle_spd_bfs_sources.restype = ctypes.c_int
+        lib.oracle_spd_bfs_sources.argtypes = [ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
+                                               ctypes.c_int64, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -58,6 +61,23 @@ def spd_matrix(row_ptr: np.ndarray, col_idx: np.ndarray, max_dist: int, ld: int 
     rc = _load().oracle_spd_bfs(n, rp.ctypes.data, ci.ctypes.data, int(max_dist), int(ld), out.ctypes.data)
     if rc != 0:
         raise RuntimeError(f"oracle_spd_bfs failed with code {rc}")
+    return out
+
+
+def spd_rows(row_ptr: np.ndarray, col_idx: np.ndarray, max_dist: int, sources: np.ndarray) -> np.ndarray:
+    """uint8 [len(sources), ld]: the SPD rows of the listed sources only (BFS from each)."""
+    n = len(row_ptr) - 1
+    ld = (n + 15) // 16 * 16
+    rp = np.ascontiguousarray(row_ptr, dtype=np.int32)
+    ci = np.ascontiguousarray(col_idx, dtype=np.int32)
+    if ci.size == 0:
+        ci = np.zeros(1, np.int32)
+    src = np.ascontiguousarray(sources, dtype=np.int32)
+    out = np.empty((len(src), ld), dtype=np.uint8)
+    rc = _load().oracle_spd_bfs_sources(n, rp.ctypes.data, ci.ctypes.data, int(max_dist), int(ld),
+                                        len(src), src.ctypes.data, out.ctypes.data)
+    if rc != 0:
+        raise RuntimeError(f"oracle_spd_bfs_sources failed with code {rc}")
     return out
 
 

@@ -21,10 +21,13 @@
 #include <stdlib.h>
 #include <string.h>
 
-int oracle_spd_bfs(int32_t n, const int32_t* row_ptr, const int32_t* col_idx,
-                   int32_t max_dist, int64_t ld, uint8_t* spd)
+/* Rows of the SPD matrix for the listed sources only: row i of `spd` (pitch ld) is the full
+ * distance row of source sources[i].  sources == NULL means all n sources in order. */
+int oracle_spd_bfs_sources(int32_t n, const int32_t* row_ptr, const int32_t* col_idx,
+                           int32_t max_dist, int64_t ld, int32_t n_sources, const int32_t* sources,
+                           uint8_t* spd)
 {
-    if (n < 0 || max_dist < 1 || max_dist > 254 || ld < n) return 1;
+    if (n < 0 || max_dist < 1 || max_dist > 254 || ld < n || n_sources < 0) return 1;
     int fail = 0;
 #pragma omp parallel
     {
@@ -35,7 +38,8 @@ int oracle_spd_bfs(int32_t n, const int32_t* row_ptr, const int32_t* col_idx,
             fail = 1;
         } else {
 #pragma omp for schedule(dynamic, 16)
-            for (int32_t s = 0; s < n; ++s) {
+            for (int32_t si = 0; si < n_sources; ++si) {
+                const int32_t s = sources ? sources[si] : si;
                 for (int32_t t = 0; t < n; ++t) dist[t] = -1;
                 int32_t head = 0, tail = 0;
                 dist[s] = 0;
@@ -50,7 +54,7 @@ int oracle_spd_bfs(int32_t n, const int32_t* row_ptr, const int32_t* col_idx,
                         }
                     }
                 }
-                uint8_t* row = spd + (int64_t)s * ld;
+                uint8_t* row = spd + (int64_t)si * ld;
                 for (int32_t t = 0; t < n; ++t) {
                     int32_t dd = dist[t];
                     row[t] = (uint8_t)(dd < 0 ? max_dist + 1 : (dd > max_dist ? max_dist : dd));
@@ -62,4 +66,10 @@ int oracle_spd_bfs(int32_t n, const int32_t* row_ptr, const int32_t* col_idx,
         free(queue);
     }
     return fail ? 2 : 0;
+}
+
+int oracle_spd_bfs(int32_t n, const int32_t* row_ptr, const int32_t* col_idx,
+                   int32_t max_dist, int64_t ld, uint8_t* spd)
+{
+    return oracle_spd_bfs_sources(n, row_ptr, col_idx, max_dist, ld, n, (const int32_t*)0, spd);
 }

@@ -250,3 +250,15 @@ def test_bias_after_max_update_would_be_wrong():
         wrong_den += np.exp(blk).sum(1, keepdims=True)
     wrong = wrong_num / wrong_den
     assert np.abs(wrong - o[:, 0]).max() > 1e-2
+
+
+def test_compact_spd_rows_match_full():
+    q, k, v, do, spd, b = make_case(110, 2, 32, 4, seed=23, directed=True)
+    rows = np.array([100, 3, 57])
+    a = oattn.forward_single(q, k, v, spd, b, rows=rows)
+    c = oattn.forward_single(q, k, v, np.ascontiguousarray(spd[rows]), b, rows=rows, compact_spd=True)
+    np.testing.assert_array_equal(a[0], c[0])
+    ga = oattn.backward_single(q, k, v, do, spd, b, rows=rows)
+    gc = oattn.backward_single(q, k, v, do, np.ascontiguousarray(spd[rows]), b, rows=rows, compact_spd=True)
+    for x, y in zip(ga, gc):
+        np.testing.assert_array_equal(x, y)

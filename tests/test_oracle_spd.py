@@ -184,3 +184,10 @@ def test_packed_batch_layout():
         ld = int(b.spd_ld[g])
         blk = flat[int(b.spd_offsets[g]):int(b.spd_offsets[g]) + n_g * ld].reshape(n_g, ld)
         np.testing.assert_array_equal(blk[:, :n_g], floyd_warshall_spd(b.graph_csr(g), w.max_dist))
+
+
+def test_source_subset_equals_full_rows():
+    csr = wl.random_directed(90, 1.6, 2)
+    full = ospd.spd_matrix(*csr, 7)
+    rows = np.array([5, 0, 89, 33, 33])
+    np.testing.assert_array_equal(ospd.spd_rows(*csr, 7, rows), full[rows])
