@@ -15,7 +15,7 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libgtattn.so")
+LIB_PATH = os.environ.get("GT_ATTN_LIB", os.path.join(_HERE, "libgtattn.so"))
 
 GT_OK = 0
 STATUS_NAMES = {0: "GT_OK", 1: "GT_ERR_INVALID_ARG", 2: "GT_ERR_UNSUPPORTED", 3: "GT_ERR_WORKSPACE",

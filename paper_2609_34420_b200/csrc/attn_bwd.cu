@@ -96,10 +96,6 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
-__device__ __forceinline__ void named_barrier_sync(uint32_t id, uint32_t n_threads)
-{
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
-}
 __device__ __forceinline__ void setmaxnreg_inc_192() { asm volatile("setmaxnreg.inc.sync.aligned.u32 192;"); }
 __device__ __forceinline__ void setmaxnreg_dec_72() { asm volatile("setmaxnreg.dec.sync.aligned.u32 72;"); }
 
@@ -191,32 +187,38 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);     // A and B MN-major
             const uint32_t sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV);
             auto issue_st = [&](int s) {        // S^T = K Q^T
-                uint64_t da = make_smem_desc(sK, L::kRowBytes, 0);
-                uint64_t db = make_smem_desc(smem_u32(smem + L::kQ + s * L::kTileBytes), L::kRowBytes, 0);
+                if (elect_one()) {
+                    uint64_t da = make_smem_desc(sK, L::kRowBytes, 0);
+                    uint64_t db = make_smem_desc(smem_u32(smem + L::kQ + s * L::kTileBytes), L::kRowBytes, 0);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ss(tmem + kColS, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
-                mma_commit(bar(kBarSFull));
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        mma_ss(tmem + kColS, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
+                    mma_commit(bar(kBarSFull));
+                }
+                __syncwarp();
             };
             auto issue_dpt = [&](int s) {       // dP^T = V dO^T
-                uint64_t da = make_smem_desc(sV, L::kRowBytes, 0);
-                uint64_t db = make_smem_desc(smem_u32(smem + L::kDo + s * L::kTileBytes), L::kRowBytes, 0);
+                if (elect_one()) {
+                    uint64_t da = make_smem_desc(sV, L::kRowBytes, 0);
+                    uint64_t db = make_smem_desc(smem_u32(smem + L::kDo + s * L::kTileBytes), L::kRowBytes, 0);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ss(tmem + kColDp, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
-                mma_commit(bar(kBarDpFull));
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        mma_ss(tmem + kColDp, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
+                    mma_commit(bar(kBarDpFull));
+                }
+                __syncwarp();
             };
             mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 120);
             mbar_wait(bar(kBarQdoFull + 0), 0, abort_flag, p.status, 121);
             tc_fence_after();
-            if (lane == 0) { issue_st(0); issue_dpt(0); }
-            __syncwarp();
+            issue_st(0);
+            issue_dpt(0);
             for (int i = 0; i < n_q; ++i) {
                 const int s = i & 1;
                 // ---- after P^T: dV += P^T dO_i, then S^T of the next tile ----
                 mbar_wait(bar(kBarPFull), i & 1, abort_flag, p.status, 122);
                 tc_fence_after();
-                if (lane == 0) {
+                if (elect_one()) {
                     uint64_t db = make_smem_desc(smem_u32(smem + L::kDo + s * L::kTileBytes), L::kRowBytes, 0);
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
@@ -227,14 +229,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 if (i + 1 < n_q) {
                     mbar_wait(bar(kBarQdoFull + (s ^ 1)), ((i + 1) >> 1) & 1, abort_flag, p.status, 123);
                     tc_fence_after();
-                    if (lane == 0) issue_st(s ^ 1);
-                    __syncwarp();
+                    issue_st(s ^ 1);
                 }
                 // ---- after dS^T: dK += dS^T Q_i, dQ_i = dS K, then dP^T of the next tile ----
                 mbar_wait(bar(kBarDsFull), i & 1, abort_flag, p.status, 124);
                 mbar_wait(bar(kBarDqFree + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 125);
                 tc_fence_after();
-                if (lane == 0) {
+                if (elect_one()) {
                     uint64_t dbq = make_smem_desc(smem_u32(smem + L::kQ + s * L::kTileBytes), L::kRowBytes, 0);
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks)
@@ -248,11 +249,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                                advance_desc(dbk, ks * 16 * L::kRowBytes), idesc_dq, ks > 0);
                     mma_commit(bar(kBarDqFull + s));
                     mma_commit(bar(kBarStageEmpty + s));
-                    if (i + 1 < n_q) issue_dpt(s ^ 1);
                 }
                 __syncwarp();
+                if (i + 1 < n_q) issue_dpt(s ^ 1);
             }
-            if (lane == 0) mma_commit(bar(kBarFinal));
+            if (elect_one()) mma_commit(bar(kBarFinal));
             __syncwarp();
         } else if (warp == 2) {
             // ------------------------------ aux loader ------------------------------

@@ -9,10 +9,10 @@
 // tensor pipe works on one tile while the other is in its softmax) x all key tiles of the
 // graph (or of one key chunk for the chunked entry point).
 //
-//   warp 0      TMA producer: Q once, then K/V tiles through a 3-stage ring
+//   warp 0      TMA producer: Q once, then K/V tiles through a 2-stage ring
 //   warp 1      MMA issuer: S_t = Q_t K^T (SS), O_t += P_t V (A from TMEM, B = V as MN-major)
-//   warp 2      SPD loader: 256x128-byte index tile per key tile via cp.async, 16-byte chunks
-//               XOR-swizzled by row so that the row-per-thread reads are conflict free
+//   warps 2-3   SPD loaders: 256x128-byte index tile per key tile via cp.async (3-stage ring),
+//               16-byte chunks XOR-swizzled by row so that the row-per-thread reads are conflict free
 //   warps 4-7   softmax of tile 0 (thread = query row = TMEM lane), warps 8-11 of tile 1
 //
 // TMEM columns: S0 [0,128) S1 [128,256) P0 [256,320) P1 [320,384) O0 [384,448) O1 [448,512).
@@ -59,8 +59,8 @@ constexpr int kRowsPerTile = 128;
 constexpr int kQTiles = 2;
 constexpr int kRowsPerCta = kRowsPerTile * kQTiles;
 constexpr int kKvTile = 128;
-constexpr int kKvStages = 3;
-constexpr int kSpdStages = 2;
+constexpr int kKvStages = 2;
+constexpr int kSpdStages = 3;
 constexpr int kFwdThreads = 384;
 constexpr float kRescaleThreshold = 8.0f;     // log2 units: keep a stale max while P stays below 2^8
 
@@ -117,7 +117,7 @@ __device__ __forceinline__ float max3(float a, float b, float c)
     return r;
 }
 
-template <int D, bool kPartial>
+template <int D, bool kPartial, bool kShflBias>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const FwdParams p)
@@ -165,7 +165,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         misc[1] = 0u;
         mbar_init(bar(kBarQFull), 1);
         for (int s = 0; s < kKvStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), 1); }
-        for (int s = 0; s < kSpdStages; ++s) { mbar_init(bar(kBarSpdFull + s), 32); mbar_init(bar(kBarSpdEmpty + s), 8); }
+        for (int s = 0; s < kSpdStages; ++s) { mbar_init(bar(kBarSpdFull + s), 64); mbar_init(bar(kBarSpdEmpty + s), 8); }
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar(kBarSFull + t), 1);
             mbar_init(bar(kBarSFree + t), 128);
@@ -187,7 +187,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 
     if (warp < 4) {
         // =========================== producer / MMA / SPD warps ===========================
-        setmaxnreg_dec_40();
+        setmaxnreg_dec_56();
         if (warp == 0) {
             if (lane == 0) {
                 mbar_arrive_expect_tx(bar(kBarQFull), kQTiles * L::kTileBytes);
@@ -207,61 +207,73 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 __syncwarp();
             }
         } else if (warp == 1) {
+            // The warp stays converged around the waits; one elected lane issues each group of MMAs.
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
             constexpr uint32_t idesc_o = make_idesc_bf16(128, D, false, true);
+            const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+            const uint64_t desc_q0 = make_smem_desc(smem_u32(smem + L::kQ), L::kRowBytes, 0);
+            const uint64_t desc_k0 = make_smem_desc(smem_u32(smem + L::kK), L::kRowBytes, 0);
+            const uint64_t desc_v0 = make_smem_desc(smem_u32(smem + L::kV), L::kRowBytes, 0);
             auto issue_s = [&](int t, int stage) {
-                uint64_t da = make_smem_desc(smem_u32(smem + L::kQ + t * L::kTileBytes), L::kRowBytes, 0);
-                uint64_t db = make_smem_desc(smem_u32(smem + L::kK + stage * L::kTileBytes), L::kRowBytes, 0);
+                if (elect_one()) {
+                    const uint64_t da = advance_desc(desc_q0, t * L::kTileBytes);
+                    const uint64_t db = advance_desc(desc_k0, stage * L::kTileBytes);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ss(tmem + t * 128, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
-                mma_commit(bar(kBarSFull + t));
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        mma_ss(tm + t * 128, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
+                    mma_commit(bar(kBarSFull + t));
+                }
+                __syncwarp();
             };
             mbar_wait(bar(kBarQFull), 0, abort_flag, p.status, 20);
             mbar_wait(bar(kBarKvFull + 0), 0, abort_flag, p.status, 21);
             tc_fence_after();
-            if (lane == 0) { issue_s(0, 0); issue_s(1, 0); }
-            __syncwarp();
+            issue_s(0, 0);
+            issue_s(1, 0);
             for (int j = 0; j < n_kv; ++j) {
                 const int s = j % kKvStages;
                 if (j + 1 < n_kv) {
                     const int s1 = (j + 1) % kKvStages;
                     mbar_wait(bar(kBarKvFull + s1), ((j + 1) / kKvStages) & 1, abort_flag, p.status, 22);
+#pragma unroll
                     for (int t = 0; t < 2; ++t) {
                         mbar_wait(bar(kBarSFree + t), j & 1, abort_flag, p.status, 23);
                         tc_fence_after();
-                        if (lane == 0) issue_s(t, s1);
-                        __syncwarp();
+                        issue_s(t, s1);
                     }
                 }
+                const uint64_t dv = advance_desc(desc_v0, s * L::kTileBytes);
+                const uint32_t acc0 = j > 0 ? 1u : 0u;
+#pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     mbar_wait(bar(kBarPFull + t), j & 1, abort_flag, p.status, 24);
                     tc_fence_after();
-                    if (lane == 0) {
-                        uint64_t dv = make_smem_desc(smem_u32(smem + L::kV + s * L::kTileBytes), L::kRowBytes, 0);
+                    if (elect_one()) {
 #pragma unroll
                         for (int ks = 0; ks < kKvTile / 16; ++ks)
-                            mma_ts(tmem + 384 + t * 64, tmem + 256 + t * 64 + ks * 8,
-                                   advance_desc(dv, ks * 16 * L::kRowBytes), idesc_o, (j > 0 || ks > 0) ? 1u : 0u);
+                            mma_ts(tm + 384 + t * 64, tm + 256 + t * 64 + ks * 8,
+                                   advance_desc(dv, ks * 16 * L::kRowBytes), idesc_o, ks > 0 ? 1u : acc0);
                         mma_commit(bar(kBarODone + t));
+                        if (t == 1) mma_commit(bar(kBarKvEmpty + s));
                     }
                     __syncwarp();
                 }
-                if (lane == 0) mma_commit(bar(kBarKvEmpty + s));
-                __syncwarp();
             }
-        } else if (warp == 2) {
+        } else {
+            // warps 2 and 3: SPD tile loader, 128 of the 256 rows each
+            const int half = warp - 2;
             for (int j = 0; j < n_kv; ++j) {
                 const int s2 = j % kSpdStages;
                 mbar_wait(bar(kBarSpdEmpty + s2), ((j / kSpdStages) & 1) ^ 1, abort_flag, p.status, 30);
                 const int32_t kv0 = kv_begin + j * kKvTile;
                 const uint32_t dst0 = smem_u32(smem + L::kSpd + s2 * L::kSpdTileBytes);
+                const int cc = lane & 7;
+                const int64_t col = (int64_t)kv0 + cc * 16;
+                const bool col_ok = col < ld;
 #pragma unroll 4
-                for (int i = 0; i < (kRowsPerCta * 8) / 32; ++i) {
-                    const int c = i * 32 + lane;
-                    const int r = c >> 3, cc = c & 7;
-                    const int64_t col = (int64_t)kv0 + cc * 16;
-                    const bool valid = (q0 + r < n_g) && (col < ld);
+                for (int i = 0; i < 32; ++i) {
+                    const int r = half * 128 + i * 4 + (lane >> 3);
+                    const bool valid = col_ok && (q0 + r < n_g);
                     const uint8_t* src = valid ? spd_g + (int64_t)(q0 + r) * ld + col : spd_g;
                     cp_async_16(dst0 + r * 128 + ((cc ^ (r & 7)) << 4), src, valid ? 16u : 0u);
                 }
@@ -270,7 +282,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
     } else {
         // ================================= softmax warpgroups =================================
-        setmaxnreg_inc_232();
+        setmaxnreg_inc_224();
         const int t = (warp >> 2) - 1;
         const int r = tid & 127;
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
@@ -280,56 +292,115 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const float c1 = p.c1;
         float m = -INFINITY, l = 0.f;
 
-        for (int j = 0; j < n_kv; ++j) {
-            float x[128];
+        // lane b of every softmax warp keeps table entry b (scaled by log2 e); entries past the
+        // table repeat the last one.  With at most 32 buckets a score's bias is fetched by a
+        // warp shuffle whose source lane is the raw SPD byte (only its low 5 bits select).
+        const float tbl = s_bias[lane];
+        const uint64_t c1c1 = pack_f32x2(c1, c1);
+
+        // The two softmax warpgroups take turns in the exponential phase (it saturates the
+        // special-function unit; the other group meanwhile runs its lookup / max phase on the
+        // other pipes).  Barrier 2+t lets group t in; the other group arrives on it when it leaves.
+        if (t == 1) named_barrier_arrive(2, 256);
+
+        // Software-pipelined over key tiles: the first 64 score columns and the SPD row of tile
+        // j+1 are fetched at the end of tile j, so their latency hides behind the P store.
+        uint32_t sa[32], sb[32];                // score chunks of 32 columns, alternating
+        uint4 wa[2], wb[2];                     // SPD bytes of those chunks (2 x 16 bytes each)
+        auto spd_row = [&](int j) {
+            return smem + L::kSpd + (j % kSpdStages) * L::kSpdTileBytes + (t * 128 + r) * 128;
+        };
+        auto prefetch = [&](int j) {
             mbar_wait(bar(kBarSFull + t), j & 1, abort_flag, p.status, 40);
             tc_fence_after();
-            {
-                uint32_t s0[32], s1[32], s2r[32], s3[32];
-                tmem_ld32(tS, s0);
-                tmem_ld32(tS + 32, s1);
-                tmem_ld32(tS + 64, s2r);
-                tmem_ld32(tS + 96, s3);
-                tmem_wait_ld();
-                tc_fence_before();
-                mbar_arrive(bar(kBarSFree + t));
+            tmem_ld32(tS, sa);
+            mbar_wait(bar(kBarSpdFull + (j % kSpdStages)), (j / kSpdStages) & 1, abort_flag, p.status, 41);
+            const uint8_t* srow = spd_row(j);
+            wa[0] = *(const uint4*)(srow + ((0 ^ (r & 7)) << 4));
+            wa[1] = *(const uint4*)(srow + ((1 ^ (r & 7)) << 4));
+        };
+        prefetch(0);
+
+        for (int j = 0; j < n_kv; ++j) {
+            uint64_t xp[64];                       // 128 scores of this row as f32x2 pairs
+            // one chunk = 32 columns: two rounds of (16 bias lookups, then 8 packed FMAs  x = s c1 + bias)
+            auto chunk = [&](int c, const uint32_t (&sr)[32], const uint4 (&ws)[2]) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    x[i] = __uint_as_float(s0[i]);
-                    x[32 + i] = __uint_as_float(s1[i]);
-                    x[64 + i] = __uint_as_float(s2r[i]);
-                    x[96 + i] = __uint_as_float(s3[i]);
-                }
-            }
-            const int s2 = j % kSpdStages;
-            mbar_wait(bar(kBarSpdFull + s2), (j / kSpdStages) & 1, abort_flag, p.status, 41);
-            {
-                const uint8_t* srow = smem + L::kSpd + s2 * L::kSpdTileBytes + (t * 128 + r) * 128;
+                for (int hh = 0; hh < 2; ++hh) {
+                    float bb[16];
+                    const uint32_t words[4] = {ws[hh].x, ws[hh].y, ws[hh].z, ws[hh].w};
 #pragma unroll
-                for (int c8 = 0; c8 < 8; ++c8) {
-                    const uint4 w = *(const uint4*)(srow + ((c8 ^ (r & 7)) << 4));
-                    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) {
-                        const uint32_t b = (ww[i >> 2] >> ((i & 3) * 8)) & 0xffu;
-                        x[c8 * 16 + i] = fmaf(x[c8 * 16 + i], c1, s_bias[b]);
+                    for (int k = 0; k < 4; ++k) {
+                        if (kShflBias) {
+                            bb[4 * k + 0] = __shfl_sync(0xffffffffu, tbl, words[k]);
+                            bb[4 * k + 1] = __shfl_sync(0xffffffffu, tbl, words[k] >> 8);
+                            bb[4 * k + 2] = __shfl_sync(0xffffffffu, tbl, words[k] >> 16);
+                            bb[4 * k + 3] = __shfl_sync(0xffffffffu, tbl, words[k] >> 24);
+                        } else {
+                            bb[4 * k + 0] = s_bias[words[k] & 0xffu];
+                            bb[4 * k + 1] = s_bias[(words[k] >> 8) & 0xffu];
+                            bb[4 * k + 2] = s_bias[(words[k] >> 16) & 0xffu];
+                            bb[4 * k + 3] = s_bias[words[k] >> 24];
+                        }
                     }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        xp[c * 16 + hh * 8 + i] = fma_f32x2(pack_u32x2(sr[hh * 16 + 2 * i], sr[hh * 16 + 2 * i + 1]), c1c1,
+                                                            pack_f32x2(bb[2 * i], bb[2 * i + 1]));
                 }
-            }
+            };
+            const uint8_t* srow = spd_row(j);
+            auto lds_words = [&](int c, uint4 (&ws)[2]) {
+                ws[0] = *(const uint4*)(srow + (((2 * c) ^ (r & 7)) << 4));
+                ws[1] = *(const uint4*)(srow + (((2 * c + 1) ^ (r & 7)) << 4));
+            };
+            tmem_wait_ld();                        // chunk 0 (prefetched at the end of the previous tile)
+            tmem_ld32(tS + 32, sb);
+            lds_words(1, wb);
+            chunk(0, sa, wa);
+            tmem_wait_ld();
+            tmem_ld32(tS + 64, sa);
+            lds_words(2, wa);
+            chunk(1, sb, wb);
+            tmem_wait_ld();
+            tmem_ld32(tS + 96, sb);
+            lds_words(3, wb);
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(kBarSpdEmpty + s2));
+            if (lane == 0) mbar_arrive(bar(kBarSpdEmpty + (j % kSpdStages)));
+            chunk(2, sa, wa);
+            tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive(bar(kBarSFree + t));
+            chunk(3, sb, wb);
 
             const int32_t kv0 = kv_begin + j * kKvTile;
             if (kv0 + kKvTile > kv_end) {           // ragged last key tile
                 const int valid = kv_end - kv0;
 #pragma unroll
-                for (int i = 0; i < 128; ++i)
-                    if (i >= valid) x[i] = -INFINITY;
+                for (int i = 0; i < 64; ++i) {
+                    float lo, hi;
+                    unpack_f32x2(xp[i], lo, hi);
+                    if (2 * i >= valid) lo = -INFINITY;
+                    if (2 * i + 1 >= valid) hi = -INFINITY;
+                    xp[i] = pack_f32x2(lo, hi);
+                }
             }
-            float mt = x[0];
+            float mt0, mt1;
+            unpack_f32x2(xp[0], mt0, mt1);
 #pragma unroll
-            for (int i = 1; i + 1 < 128; i += 2) mt = max3(mt, x[i], x[i + 1]);
-            mt = fmaxf(mt, x[127]);
+            for (int i = 1; i < 64; i += 2) {
+                float a, b, c, d2;
+                unpack_f32x2(xp[i], a, b);
+                if (i + 1 < 64) {
+                    unpack_f32x2(xp[i + 1], c, d2);
+                    mt0 = max3(mt0, a, c);
+                    mt1 = max3(mt1, b, d2);
+                } else {
+                    mt0 = fmaxf(mt0, a);
+                    mt1 = fmaxf(mt1, b);
+                }
+            }
+            const float mt = fmaxf(mt0, mt1);
             // The reference maximum is kept at an integer (log2 units): rescale factors are then
             // exact powers of two and the bf16 mantissa of every P entry does not depend on how
             // the keys are tiled or chunked, which keeps chunked and unchunked results within
@@ -357,23 +428,41 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 }
                 m = m_new;
             }
-            float sum = 0.f;
+
+            // ---- exponential phase: the MUFU results are consumed kExpLag pairs after they are
+            // issued so that the in-order pipeline never waits on a result it has just asked for.
+            named_barrier_sync(2 + t, 256);
+            const uint64_t neg_m = pack_f32x2(-m, -m);
+#pragma unroll
+            for (int i = 0; i < 64; ++i) xp[i] = add_f32x2(xp[i], neg_m);
+            uint64_t sum2 = pack_f32x2(0.f, 0.f);
             uint32_t pk0[32], pk1[32];
+            constexpr int kExpLag = 6;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const float a = ex2_approx(x[2 * i] - m), b = ex2_approx(x[2 * i + 1] - m);
-                sum += a + b;
-                pk0[i] = pack_bf16x2(a, b);
+            for (int i = 0; i < 64 + kExpLag; ++i) {
+                if (i < 64) {
+                    float lo, hi;
+                    unpack_f32x2(xp[i], lo, hi);
+                    xp[i] = pack_f32x2(ex2_approx(lo), ex2_approx(hi));
+                }
+                if (i >= kExpLag) {
+                    const int k = i - kExpLag;
+                    float lo, hi;
+                    unpack_f32x2(xp[k], lo, hi);
+                    sum2 = add_f32x2(sum2, xp[k]);
+                    if (k < 32) pk0[k] = pack_bf16x2(lo, hi);
+                    else pk1[k - 32] = pack_bf16x2(lo, hi);
+                }
             }
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const float a = ex2_approx(x[64 + 2 * i] - m), b = ex2_approx(x[64 + 2 * i + 1] - m);
-                sum += a + b;
-                pk1[i] = pack_bf16x2(a, b);
+            named_barrier_arrive(2 + (t ^ 1), 256);
+            {
+                float lo, hi;
+                unpack_f32x2(sum2, lo, hi);
+                l += lo + hi;
             }
-            l += sum;
             tmem_st32(tP, pk0);
             tmem_st32(tP + 32, pk1);
+            if (j + 1 < n_kv) prefetch(j + 1);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar(kBarPFull + t));
@@ -469,7 +558,7 @@ template <int D, bool kPartial>
 gt_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
                      const gt_batch* batch, int grid_z, cudaStream_t s)
 {
-    auto kern = attn_fwd_kernel<D, kPartial>;
+    auto kern = p.n_buckets <= 32 ? attn_fwd_kernel<D, kPartial, true> : attn_fwd_kernel<D, kPartial, false>;
     GT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kDynamic));
     dim3 grid((unsigned)p.n_heads, (unsigned)((batch->max_seqlen + kRowsPerCta - 1) / kRowsPerCta), (unsigned)grid_z);
     kern<<<grid, kFwdThreads, FwdSmem<D>::kDynamic, s>>>(tq, tk, tv, p);
