@@ -9,11 +9,15 @@
 // gradient dB[h][b] = sum of dS over pairs in bucket b is binned in shared memory (one
 // private bin column per thread, no conflicts) and flushed once per CTA with fp64 atomics.
 //
-//   warp 0        TMA producer: K, V once; Q_i, dO_i through a 2-stage ring
-//   warp 1        MMA issuer (5 GEMMs per query tile)
-//   warp 2        aux loader: SPD tile, lse*log2(e) and Delta of the query tile (cp.async)
-//   warps 4-11    two softmax warpgroups: query columns [0,64) and [64,128) of the tile
-//   warps 12-15   dQ reducer: TMEM -> red.global.add.v4.f32
+//   warp 0        TMA producer: K, V once; Q_i, dO_i and (single graph) the SPD tile, 2-stage ring
+//   warp 1        aux loader: lse*log2(e) and Delta of the query tile; SPD tile for packed batches
+//   warps 4-19    sixteen softmax warps = four groups of 128 threads; group g owns query columns
+//                 [32g, 32g+32) of the tile (32 score elements per thread).  Many warps rather than
+//                 long rows per thread: the per-element work is a chain of dependent shared-memory
+//                 lookups, which only thread-level parallelism hides.  Two of these warps also issue
+//                 the MMAs (after a barrier of all softmax threads): a separate MMA warp would be
+//                 starved of issue slots by the busy warps on its scheduler.
+//   warps 20-23   dQ reducer: TMEM -> red.global.add.v4.f32
 //
 // TMEM columns: S^T/P^T [0,128)  dP^T/dS^T [128,256)  dV [256,320)  dK [320,384)  dQ0 [384,448)  dQ1 [448,512).
 #include <cuda_bf16.h>
@@ -29,9 +33,10 @@ using namespace sm100;
 
 constexpr int kTile = 128;
 constexpr int kStages = 2;
-constexpr int kBwdThreads = 512;
-constexpr int kSoftmaxThreads = 256;
-constexpr int kPrivateBinBuckets = 32;     // up to this many buckets: one private bin column per thread
+constexpr int kBwdThreads = 768;
+constexpr int kSoftmaxThreads = 512;
+constexpr int kColsPerThread = 32;
+constexpr int kMaxPrivateBinBuckets = 28;   // 2 KB of shared memory per bucket
 
 struct BwdParams {
     const uint8_t* spd;
@@ -48,6 +53,7 @@ struct BwdParams {
     int32_t n_total;
     int32_t n_heads;
     int32_t n_buckets;
+    int32_t spd_tma;         // 1: single graph, SPD tiles come by TMA
     float c1;                // log2(e)/sqrt(d)
     float scale;             // 1/sqrt(d)
 };
@@ -55,17 +61,17 @@ struct BwdParams {
 enum BwdBarrier {
     kBarKvFull = 0,
     kBarQdoFull = 1,                       // [2]
-    kBarAuxFull = kBarQdoFull + kStages,   // [2]
-    kBarStageEmpty = kBarAuxFull + kStages,// [2]
-    kBarSFull = kBarStageEmpty + kStages,
+    kBarAuxFull = kBarQdoFull + kStages,   // [2]  SPD tile + lse2 + Delta
+    kBarStageEmpty = kBarAuxFull + kStages,// [2]  one arrive: the dQ reducer, after its TMA reduce has read the stage
+    kBarDvDone = kBarStageEmpty + kStages, // [2]  commit after dV += P^T dO_i (dO_i no longer read)
+    kBarSFull = kBarDvDone + kStages,
     kBarDpFull,
-    kBarPFull,
-    kBarDsFull,
     kBarDqFull,                            // [2]
     kBarDqFree = kBarDqFull + 2,           // [2]
-    kBarFinal = kBarDqFree + 2,
+    kBarFinal = kBarDqFree + 2,            //      two commits
     kNumBwdBarriers
 };
+enum BwdNamedBarrier { kNbFlush = 1, kNbPStored = 2, kNbDsStored = 3, kNbDqStaged = 4 };
 
 template <int D>
 struct BwdSmem {
@@ -74,18 +80,18 @@ struct BwdSmem {
     static constexpr int kSpdBytes = kTile * kTile;
     static constexpr int kK = 0;
     static constexpr int kV = kK + kTileBytes;
-    static constexpr int kQ = kV + kTileBytes;                      // [kStages]
-    static constexpr int kDo = kQ + kStages * kTileBytes;           // [kStages]
-    static constexpr int kSpd = kDo + kStages * kTileBytes;         // [kStages]
+    static constexpr int kStageBytes = 2 * kTileBytes;              // Q_i then dO_i; later the dQ_i staging area
+    static constexpr int kQ = kV + kTileBytes;                      // [kStages] at stride kStageBytes
+    static constexpr int kDo = kQ + kTileBytes;                     // [kStages] at stride kStageBytes
+    static constexpr int kSpd = kQ + kStages * kStageBytes;         // [kStages]
     static constexpr int kLse = kSpd + kStages * kSpdBytes;         // [kStages][128] float
     static constexpr int kDelta = kLse + kStages * 512;             // [kStages][128] float
     static constexpr int kDs = kDelta + kStages * 512;              // 2 atoms x 128 rows x 128 B
-    static constexpr int kBins = kDs + 32768;                       // [32][256] float
-    static constexpr int kBias = kBins + kPrivateBinBuckets * kSoftmaxThreads * 4;
+    static constexpr int kBias = kDs + 32768;
     static constexpr int kBars = kBias + 256 * 4;
     static constexpr int kMisc = kBars + kNumBwdBarriers * 8;
-    static constexpr int kTotal = kMisc + 16;
-    static constexpr int kDynamic = kTotal + 1024;
+    static constexpr int kBins = (kMisc + 16 + 127) & ~127;         // [n_bins][512] float (private) or [nb][32]
+    static size_t dynamic_bytes(int bin_floats) { return (size_t)kBins + (size_t)bin_floats * 4 + 1024; }
 };
 
 __device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src, uint32_t src_bytes)
@@ -96,18 +102,23 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 {
     asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
-__device__ __forceinline__ void setmaxnreg_inc_192() { asm volatile("setmaxnreg.inc.sync.aligned.u32 192;"); }
-__device__ __forceinline__ void setmaxnreg_dec_72() { asm volatile("setmaxnreg.dec.sync.aligned.u32 72;"); }
+// register budget: the CTA is launched with 768 x 80 registers; after the re-split it holds
+// 128 x 40 + 512 x 96 + 128 x 48 = 60416 <= 61440 (an increase can only draw on what the CTA owns)
+__device__ __forceinline__ void setmaxnreg_inc_96() { asm volatile("setmaxnreg.inc.sync.aligned.u32 96;"); }
+__device__ __forceinline__ void setmaxnreg_dec_48() { asm volatile("setmaxnreg.dec.sync.aligned.u32 48;"); }
 
-template <int D, bool kPrivateBins>
+template <int D, bool kPrivateBins, bool kShflBias>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_do,
+                const __grid_constant__ CUtensorMap tmap_spd, const __grid_constant__ CUtensorMap tmap_dq,
                 const BwdParams p)
 {
     using L = BwdSmem<D>;
     extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    // 1024-byte alignment by pointer arithmetic on the __shared__ array itself, so that every derived
+    // pointer keeps its shared address space (integer round trips would turn the accesses generic)
+    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -128,32 +139,34 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     float* s_bins = (float*)(smem + L::kBins);
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     volatile uint32_t* abort_flag = &misc[1];
+    const int n_bin_floats = kPrivateBins ? p.n_buckets * kSoftmaxThreads : p.n_buckets * 32;
 
     if (tid == 0) {
         misc[1] = 0u;
         mbar_init(bar(kBarKvFull), 1);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar(kBarQdoFull + s), 1);
-            mbar_init(bar(kBarAuxFull + s), 32);
+            mbar_init(bar(kBarAuxFull + s), p.spd_tma ? 33 : 32);
             mbar_init(bar(kBarStageEmpty + s), 1);
+            mbar_init(bar(kBarDvDone + s), 1);
             mbar_init(bar(kBarDqFull + s), 1);
             mbar_init(bar(kBarDqFree + s), 128);
         }
         mbar_init(bar(kBarSFull), 1);
         mbar_init(bar(kBarDpFull), 1);
-        mbar_init(bar(kBarPFull), kSoftmaxThreads);
-        mbar_init(bar(kBarDsFull), kSoftmaxThreads);
-        mbar_init(bar(kBarFinal), 1);
+        mbar_init(bar(kBarFinal), 2);
         fence_mbar_init();
         prefetch_tensormap(&tmap_q);
         prefetch_tensormap(&tmap_k);
         prefetch_tensormap(&tmap_v);
         prefetch_tensormap(&tmap_do);
+        prefetch_tensormap(&tmap_dq);
+        if (p.spd_tma) prefetch_tensormap(&tmap_spd);
     }
-    if (warp == 1) { tmem_alloc(smem_u32(&misc[0]), 512); tmem_relinquish(); }
+    if (warp == 2) { tmem_alloc(smem_u32(&misc[0]), 512); tmem_relinquish(); }
     for (int i = tid; i < 256; i += kBwdThreads)
         s_bias[i] = p.bias[(size_t)h * p.n_buckets + min(i, p.n_buckets - 1)] * kLog2e;
-    for (int i = tid; i < kPrivateBinBuckets * kSoftmaxThreads; i += kBwdThreads) s_bins[i] = 0.f;
+    for (int i = tid; i < n_bin_floats; i += kBwdThreads) s_bins[i] = 0.f;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -175,101 +188,33 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 if (lane == 0) {
                     const int32_t row = node0 + i * kTile;
                     mbar_arrive_expect_tx(bar(kBarQdoFull + s), 2 * L::kTileBytes);
-                    tma_load_3d(smem_u32(smem + L::kQ + s * L::kTileBytes), &tmap_q, bar(kBarQdoFull + s), 0, h, row);
-                    tma_load_3d(smem_u32(smem + L::kDo + s * L::kTileBytes), &tmap_do, bar(kBarQdoFull + s), 0, h, row);
+                    tma_load_3d(smem_u32(smem + L::kQ + s * L::kStageBytes), &tmap_q, bar(kBarQdoFull + s), 0, h, row);
+                    tma_load_3d(smem_u32(smem + L::kDo + s * L::kStageBytes), &tmap_do, bar(kBarQdoFull + s), 0, h, row);
+                    if (p.spd_tma) {
+                        mbar_arrive_expect_tx(bar(kBarAuxFull + s), L::kSpdBytes);
+                        tma_load_2d(smem_u32(smem + L::kSpd + s * L::kSpdBytes), &tmap_spd, bar(kBarAuxFull + s), kv0, i * kTile);
+                    }
                 }
                 __syncwarp();
             }
         } else if (warp == 1) {
-            // ------------------------------ MMA issuer ------------------------------
-            constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
-            constexpr uint32_t idesc_ts = make_idesc_bf16(128, D, false, true);    // A in TMEM, B MN-major
-            constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);     // A and B MN-major
-            const uint32_t sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV);
-            auto issue_st = [&](int s) {        // S^T = K Q^T
-                if (elect_one()) {
-                    uint64_t da = make_smem_desc(sK, L::kRowBytes, 0);
-                    uint64_t db = make_smem_desc(smem_u32(smem + L::kQ + s * L::kTileBytes), L::kRowBytes, 0);
-#pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)
-                        mma_ss(tmem + kColS, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
-                    mma_commit(bar(kBarSFull));
-                }
-                __syncwarp();
-            };
-            auto issue_dpt = [&](int s) {       // dP^T = V dO^T
-                if (elect_one()) {
-                    uint64_t da = make_smem_desc(sV, L::kRowBytes, 0);
-                    uint64_t db = make_smem_desc(smem_u32(smem + L::kDo + s * L::kTileBytes), L::kRowBytes, 0);
-#pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)
-                        mma_ss(tmem + kColDp, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
-                    mma_commit(bar(kBarDpFull));
-                }
-                __syncwarp();
-            };
-            mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 120);
-            mbar_wait(bar(kBarQdoFull + 0), 0, abort_flag, p.status, 121);
-            tc_fence_after();
-            issue_st(0);
-            issue_dpt(0);
-            for (int i = 0; i < n_q; ++i) {
-                const int s = i & 1;
-                // ---- after P^T: dV += P^T dO_i, then S^T of the next tile ----
-                mbar_wait(bar(kBarPFull), i & 1, abort_flag, p.status, 122);
-                tc_fence_after();
-                if (elect_one()) {
-                    uint64_t db = make_smem_desc(smem_u32(smem + L::kDo + s * L::kTileBytes), L::kRowBytes, 0);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        mma_ts(tmem + kColDv, tmem + kColS + (ks >> 2) * 64 + (ks & 3) * 8,
-                               advance_desc(db, ks * 16 * L::kRowBytes), idesc_ts, (i > 0 || ks > 0) ? 1u : 0u);
-                }
-                __syncwarp();
-                if (i + 1 < n_q) {
-                    mbar_wait(bar(kBarQdoFull + (s ^ 1)), ((i + 1) >> 1) & 1, abort_flag, p.status, 123);
-                    tc_fence_after();
-                    issue_st(s ^ 1);
-                }
-                // ---- after dS^T: dK += dS^T Q_i, dQ_i = dS K, then dP^T of the next tile ----
-                mbar_wait(bar(kBarDsFull), i & 1, abort_flag, p.status, 124);
-                mbar_wait(bar(kBarDqFree + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 125);
-                tc_fence_after();
-                if (elect_one()) {
-                    uint64_t dbq = make_smem_desc(smem_u32(smem + L::kQ + s * L::kTileBytes), L::kRowBytes, 0);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        mma_ts(tmem + kColDk, tmem + kColDp + (ks >> 2) * 64 + (ks & 3) * 8,
-                               advance_desc(dbq, ks * 16 * L::kRowBytes), idesc_ts, (i > 0 || ks > 0) ? 1u : 0u);
-                    uint64_t da = make_smem_desc(smem_u32(smem + L::kDs), 128, 16384);
-                    uint64_t dbk = make_smem_desc(sK, L::kRowBytes, 0);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        mma_ss(tmem + kColDq + s * 64, advance_desc(da, ks * 2048),
-                               advance_desc(dbk, ks * 16 * L::kRowBytes), idesc_dq, ks > 0);
-                    mma_commit(bar(kBarDqFull + s));
-                    mma_commit(bar(kBarStageEmpty + s));
-                }
-                __syncwarp();
-                if (i + 1 < n_q) issue_dpt(s ^ 1);
-            }
-            if (elect_one()) mma_commit(bar(kBarFinal));
-            __syncwarp();
-        } else if (warp == 2) {
             // ------------------------------ aux loader ------------------------------
             for (int i = 0; i < n_q; ++i) {
                 const int s = i & 1;
                 mbar_wait(bar(kBarStageEmpty + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 130);
                 const int32_t q0 = i * kTile;
-                const uint32_t dst0 = smem_u32(smem + L::kSpd + s * L::kSpdBytes);
+                if (!p.spd_tma) {
+                    // same layout as the TMA 128-byte swizzle: 16-byte chunk c of row r at chunk c ^ (r & 7)
+                    const uint32_t dst0 = smem_u32(smem + L::kSpd + s * L::kSpdBytes);
 #pragma unroll 4
-                for (int it = 0; it < (kTile * 8) / 32; ++it) {
-                    const int c = it * 32 + lane;
-                    const int r = c >> 3, cc = c & 7;
-                    const int64_t col = (int64_t)kv0 + cc * 16;
-                    const bool valid = (q0 + r < n_g) && (col < ld);
-                    const uint8_t* src = valid ? spd_g + (int64_t)(q0 + r) * ld + col : spd_g;
-                    cp_async_16(dst0 + r * 128 + cc * 16, src, valid ? 16u : 0u);
+                    for (int it = 0; it < (kTile * 8) / 32; ++it) {
+                        const int c = it * 32 + lane;
+                        const int r = c >> 3, cc = c & 7;
+                        const int64_t col = (int64_t)kv0 + cc * 16;
+                        const bool valid = (q0 + r < n_g) && (col < ld);
+                        const uint8_t* src = valid ? spd_g + (int64_t)(q0 + r) * ld + col : spd_g;
+                        cp_async_16(dst0 + r * 128 + ((cc ^ (r & 7)) << 4), src, valid ? 16u : 0u);
+                    }
                 }
                 const uint32_t dl = smem_u32(smem + L::kLse + s * 512), dd = smem_u32(smem + L::kDelta + s * 512);
 #pragma unroll
@@ -283,117 +228,201 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 cp_async_mbar_arrive_noinc(bar(kBarAuxFull + s));
             }
         }
-    } else if (warp < 12) {
-        // ================================ softmax warpgroups ================================
-        setmaxnreg_inc_192();
-        const int w = (warp >> 2) - 1;                  // query-column half handled by this warpgroup
-        const int r = tid & 127;                        // key row within the tile = TMEM lane
-        const int st = tid - 128;                       // 0..255 index among softmax threads
+    } else if (warp < 20) {
+        // ================================ softmax warps ================================
+        setmaxnreg_inc_96();
+        const int grp = (warp - 4) >> 2;                // query-column group: columns [32 grp, 32 grp + 32)
+        const int r = ((warp & 3) << 5) | lane;         // key row within the tile = TMEM lane
+        const int st = tid - 128;                       // 0..511 index among softmax threads
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + kColS + w * 64 + lane_off;
-        const uint32_t tDp = tmem + kColDp + w * 64 + lane_off;
+        const uint32_t tS = tmem + kColS + grp * 32 + lane_off;
+        const uint32_t tDp = tmem + kColDp + grp * 32 + lane_off;
         const bool kv_valid = kv0 + r < n_g;
         const float c1 = p.c1;
         const uint32_t nb_m1 = (uint32_t)p.n_buckets - 1u;
+        const float tbl = s_bias[lane];
         float* my_bins = s_bins + (kPrivateBins ? st : lane);
         constexpr int kBinStride = kPrivateBins ? kSoftmaxThreads : 32;
+        // byte (q, r) of the swizzled SPD tile sits at q*128 + (((r>>4) ^ (q&7)) << 4) + (r&15); q&7 == c&7
+        uint32_t spd_off[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) spd_off[k] = (grp * 32) * 128 + ((((uint32_t)r >> 4) ^ k) << 4) + (r & 15);
+
+        // ---- MMA issue duty (after the barriers of all softmax threads) ----
+        const bool issuer_a = warp == 4;                // dV, S^T
+        const bool issuer_b = warp == 9;                // dK, dQ, dP^T
+        constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
+        constexpr uint32_t idesc_ts = make_idesc_bf16(128, D, false, true);    // A in TMEM, B MN-major
+        constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);     // A and B MN-major
+        const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+        const uint32_t sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV);
+        auto issue_st = [&](int i) {                    // S^T = K Q_i^T
+            const int s = i & 1;
+            mbar_wait(bar(kBarQdoFull + s), (i >> 1) & 1, abort_flag, p.status, 120);
+            tc_fence_after();
+            if (elect_one()) {
+                const uint64_t da = make_smem_desc(sK, L::kRowBytes, 0);
+                const uint64_t db = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes), L::kRowBytes, 0);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    mma_ss(tm + kColS, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
+                mma_commit(bar(kBarSFull));
+            }
+            __syncwarp();
+        };
+        auto issue_dpt = [&](int i) {                   // dP^T = V dO_i^T
+            const int s = i & 1;
+            mbar_wait(bar(kBarQdoFull + s), (i >> 1) & 1, abort_flag, p.status, 121);
+            tc_fence_after();
+            if (elect_one()) {
+                const uint64_t da = make_smem_desc(sV, L::kRowBytes, 0);
+                const uint64_t db = make_smem_desc(smem_u32(smem + L::kDo + s * L::kStageBytes), L::kRowBytes, 0);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    mma_ss(tm + kColDp, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
+                mma_commit(bar(kBarDpFull));
+            }
+            __syncwarp();
+        };
+        if (issuer_a) { mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 122); issue_st(0); }
+        if (issuer_b) { mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 123); issue_dpt(0); }
 
         for (int i = 0; i < n_q; ++i) {
             const int s = i & 1;
-            float pr[64];
-            uint32_t bk[16];
+            float pr[kColsPerThread];
+            uint32_t bkp[kColsPerThread / 4];       // the 32 bucket bytes of this thread's elements, clamped
             // ---------------- P^T = exp2(S^T c1 + b2 - lse2) ----------------
             mbar_wait(bar(kBarSFull), i & 1, abort_flag, p.status, 140);
             tc_fence_after();
-            {
-                uint32_t a0[32], a1[32];
-                tmem_ld32(tS, a0);
-                tmem_ld32(tS + 32, a1);
-                tmem_wait_ld();
-#pragma unroll
-                for (int c = 0; c < 32; ++c) { pr[c] = __uint_as_float(a0[c]); pr[32 + c] = __uint_as_float(a1[c]); }
-            }
+            uint32_t acc[32];
+            tmem_ld32(tS, acc);
             mbar_wait(bar(kBarAuxFull + s), (i >> 1) & 1, abort_flag, p.status, 141);
-            const uint8_t* spd_col = smem + L::kSpd + s * L::kSpdBytes + (w * 64) * 128 + r;
-            const float4* lse4 = (const float4*)(smem + L::kLse + s * 512 + w * 256);
+            const uint8_t* spd_tile = smem + L::kSpd + s * L::kSpdBytes;
+            const float4* lse4 = (const float4*)(smem + L::kLse + s * 512 + grp * 128);
+            tmem_wait_ld();
 #pragma unroll
-            for (int c4 = 0; c4 < 16; ++c4) {
-                const float4 l4 = lse4[c4];
-                const float ls[4] = {l4.x, l4.y, l4.z, l4.w};
-                uint32_t packed = 0;
+            for (int rnd = 0; rnd < 2; ++rnd) {             // 16 elements per round: lookups first, math after
+                float bb[16], ls[16];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int c = c4 * 4 + k;
-                    const uint32_t b = min((uint32_t)spd_col[c * 128], nb_m1);    // never index past the table
-                    packed |= b << (8 * k);
-                    pr[c] = ex2_approx(fmaf(pr[c], c1, s_bias[b]) - ls[k]);
+                for (int k = 0; k < 16; ++k) {
+                    const int c = rnd * 16 + k;
+                    const uint32_t b = min((uint32_t)spd_tile[spd_off[c & 7] + c * 128], nb_m1);   // never index past the bins
+                    bb[k] = kShflBias ? __shfl_sync(0xffffffffu, tbl, b) : s_bias[b];
+                    bkp[c >> 2] = (c & 3) == 0 ? b : (bkp[c >> 2] | (b << (8 * (c & 3))));
                 }
-                bk[c4] = packed;
-            }
-            const int nq_valid = n_g - i * kTile - w * 64;      // valid query columns of this half
-            if (!kv_valid || nq_valid < 64) {
 #pragma unroll
-                for (int c = 0; c < 64; ++c)
+                for (int k4 = 0; k4 < 4; ++k4) {
+                    const float4 l4 = lse4[rnd * 4 + k4];
+                    ls[4 * k4] = l4.x; ls[4 * k4 + 1] = l4.y; ls[4 * k4 + 2] = l4.z; ls[4 * k4 + 3] = l4.w;
+                }
+#pragma unroll
+                for (int k = 0; k < 16; ++k) {
+                    const int c = rnd * 16 + k;
+                    pr[c] = ex2_approx(fmaf(__uint_as_float(acc[c]), c1, bb[k]) - ls[k]);
+                }
+            }
+            const int nq_valid = n_g - i * kTile - grp * 32;      // valid query columns of this group
+            if (!kv_valid || nq_valid < 32) {
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
                     if (!kv_valid || c >= nq_valid) pr[c] = 0.f;
             }
             {
-                uint32_t pk[32];
+                uint32_t pk[16];
 #pragma unroll
-                for (int c = 0; c < 32; ++c) pk[c] = pack_bf16x2(pr[2 * c], pr[2 * c + 1]);
-                tmem_st32(tS, pk);                      // P^T half: 32 packed columns at the start of the half
+                for (int c = 0; c < 16; ++c) pk[c] = pack_bf16x2(pr[2 * c], pr[2 * c + 1]);
+                tmem_st16(tS, pk);                      // P^T of this group: 16 packed columns at the start of its range
                 tmem_wait_st();
             }
             tc_fence_before();
-            mbar_arrive(bar(kBarPFull));
+            named_barrier_sync(kNbPStored, kSoftmaxThreads);
+            if (issuer_a) {
+                tc_fence_after();
+                if (elect_one()) {                      // dV += P^T dO_i
+                    const uint64_t db = make_smem_desc(smem_u32(smem + L::kDo + s * L::kStageBytes), L::kRowBytes, 0);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_ts(tm + kColDv, tm + kColS + (ks >> 1) * 32 + (ks & 1) * 8,
+                               advance_desc(db, ks * 16 * L::kRowBytes), idesc_ts, (i > 0 || ks > 0) ? 1u : 0u);
+                    mma_commit(bar(kBarDvDone + s));
+                    if (i + 1 == n_q) mma_commit(bar(kBarFinal));
+                }
+                __syncwarp();
+                if (i + 1 < n_q) issue_st(i + 1);
+            }
 
             // ---------------- dS^T = P^T o (dP^T - Delta) ----------------
             mbar_wait(bar(kBarDpFull), i & 1, abort_flag, p.status, 142);
             tc_fence_after();
-            {
-                uint32_t a0[32], a1[32];
-                tmem_ld32(tDp, a0);
-                tmem_ld32(tDp + 32, a1);
-                tmem_wait_ld();
-                const float4* dl4 = (const float4*)(smem + L::kDelta + s * 512 + w * 256);
+            tmem_ld32(tDp, acc);
+            const float4* dl4 = (const float4*)(smem + L::kDelta + s * 512 + grp * 128);
+            tmem_wait_ld();
 #pragma unroll
-                for (int c4 = 0; c4 < 16; ++c4) {
-                    const float4 d4 = dl4[c4];
-                    const float dl[4] = {d4.x, d4.y, d4.z, d4.w};
+            for (int rnd = 0; rnd < 2; ++rnd) {
+                float dl[16];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const int c = c4 * 4 + k;
-                        const float dp = __uint_as_float(c < 32 ? a0[c & 31] : a1[c & 31]);
-                        const float ds = pr[c] * (dp - dl[k]);
-                        pr[c] = ds;
-                        const uint32_t b = (bk[c4] >> (8 * k)) & 0xffu;
-                        if (kPrivateBins) my_bins[b * kBinStride] += ds;
-                        else atomicAdd(&my_bins[b * kBinStride], ds);
-                    }
+                for (int k4 = 0; k4 < 4; ++k4) {
+                    const float4 d4 = dl4[rnd * 4 + k4];
+                    dl[4 * k4] = d4.x; dl[4 * k4 + 1] = d4.y; dl[4 * k4 + 2] = d4.z; dl[4 * k4 + 3] = d4.w;
+                }
+#pragma unroll
+                for (int k = 0; k < 16; ++k) {
+                    const int c = rnd * 16 + k;
+                    pr[c] = pr[c] * (__uint_as_float(acc[c]) - dl[k]);
+                }
+#pragma unroll
+                for (int k = 0; k < 16; ++k) {
+                    const int c = rnd * 16 + k;
+                    const uint32_t b = (bkp[c >> 2] >> (8 * (c & 3))) & 0xffu;
+                    if (kPrivateBins) my_bins[b * kBinStride] += pr[c];
+                    else atomicAdd(&my_bins[b * kBinStride], pr[c]);
                 }
             }
             {
-                uint32_t pk[32];
+                uint32_t pk[16];
 #pragma unroll
-                for (int c = 0; c < 32; ++c) pk[c] = pack_bf16x2(pr[2 * c], pr[2 * c + 1]);
-                tmem_st32(tDp, pk);
-                uint8_t* ds_row = smem + L::kDs + w * 16384 + r * 128;
+                for (int c = 0; c < 16; ++c) pk[c] = pack_bf16x2(pr[2 * c], pr[2 * c + 1]);
+                tmem_st16(tDp, pk);
+                uint8_t* ds_row = smem + L::kDs + (grp >> 1) * 16384 + r * 128;
 #pragma unroll
-                for (int c8 = 0; c8 < 8; ++c8)
-                    *(uint4*)(ds_row + ((c8 ^ (r & 7)) << 4)) = make_uint4(pk[4 * c8], pk[4 * c8 + 1], pk[4 * c8 + 2], pk[4 * c8 + 3]);
+                for (int c8 = 0; c8 < 4; ++c8)
+                    *(uint4*)(ds_row + ((((grp & 1) * 4 + c8) ^ (r & 7)) << 4)) =
+                        make_uint4(pk[4 * c8], pk[4 * c8 + 1], pk[4 * c8 + 2], pk[4 * c8 + 3]);
                 tmem_wait_st();
             }
             fence_proxy_async_smem();
             tc_fence_before();
-            mbar_arrive(bar(kBarDsFull));
+            named_barrier_sync(kNbDsStored, kSoftmaxThreads);
+            if (issuer_b) {
+                mbar_wait(bar(kBarDqFree + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 125);
+                tc_fence_after();
+                if (elect_one()) {                      // dK += dS^T Q_i ;  dQ_i = dS K
+                    const uint64_t dbq = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes), L::kRowBytes, 0);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_ts(tm + kColDk, tm + kColDp + (ks >> 1) * 32 + (ks & 1) * 8,
+                               advance_desc(dbq, ks * 16 * L::kRowBytes), idesc_ts, (i > 0 || ks > 0) ? 1u : 0u);
+                    const uint64_t da = make_smem_desc(smem_u32(smem + L::kDs), 128, 16384);
+                    const uint64_t dbk = make_smem_desc(sK, L::kRowBytes, 0);
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_ss(tm + kColDq + s * 64, advance_desc(da, ks * 2048),
+                               advance_desc(dbk, ks * 16 * L::kRowBytes), idesc_dq, ks > 0);
+                    mma_commit(bar(kBarDqFull + s));
+                    if (i + 1 == n_q) mma_commit(bar(kBarFinal));
+                }
+                __syncwarp();
+                if (i + 1 < n_q) issue_dpt(i + 1);
+            }
         }
 
-        // ---------------- epilogue: dV (warpgroup 0) and dK (warpgroup 1) ----------------
-        mbar_wait(bar(kBarFinal), 0, abort_flag, p.status, 143);
-        tc_fence_after();
-        {
-            const uint32_t tacc = tmem + (w == 0 ? kColDv : kColDk) + lane_off;
-            const float mul = w == 0 ? 1.0f : p.scale;
-            __nv_bfloat16* dst_base = (w == 0 ? p.dv : p.dk) + ((size_t)(node0 + kv0 + r) * p.n_heads + h) * D;
+        // ---------------- epilogue: dV (group 0) and dK (group 1) ----------------
+        if (grp < 2) {
+            mbar_wait(bar(kBarFinal), 0, abort_flag, p.status, 143);
+            tc_fence_after();
+            const uint32_t tacc = tmem + (grp == 0 ? kColDv : kColDk) + lane_off;
+            const float mul = grp == 0 ? 1.0f : p.scale;
+            __nv_bfloat16* dst_base = (grp == 0 ? p.dv : p.dk) + ((size_t)(node0 + kv0 + r) * p.n_heads + h) * D;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t o[32];
@@ -414,52 +443,68 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             }
         }
         // ---------------- flush the bias-gradient bins ----------------
-        named_barrier_sync(1, kSoftmaxThreads);
+        named_barrier_sync(kNbFlush, kSoftmaxThreads);
         if (kPrivateBins) {
             if (st < p.n_buckets) {
-                float acc = 0.f;
-                for (int k = 0; k < kSoftmaxThreads; ++k) acc += s_bins[st * kSoftmaxThreads + ((k + st) & (kSoftmaxThreads - 1))];
-                atomicAdd(&p.db_acc[(size_t)h * p.n_buckets + st], (double)acc);
+                float a = 0.f;
+                for (int k = 0; k < kSoftmaxThreads; ++k) a += s_bins[st * kSoftmaxThreads + ((k + st) & (kSoftmaxThreads - 1))];
+                atomicAdd(&p.db_acc[(size_t)h * p.n_buckets + st], (double)a);
             }
         } else {
             for (int b = st; b < p.n_buckets; b += kSoftmaxThreads) {
-                float acc = 0.f;
-                for (int k = 0; k < 32; ++k) acc += s_bins[b * 32 + ((k + b) & 31)];
-                atomicAdd(&p.db_acc[(size_t)h * p.n_buckets + b], (double)acc);
+                float a = 0.f;
+                for (int k = 0; k < 32; ++k) a += s_bins[b * 32 + ((k + b) & 31)];
+                atomicAdd(&p.db_acc[(size_t)h * p.n_buckets + b], (double)a);
             }
         }
     } else {
         // ================================ dQ reducer ================================
-        setmaxnreg_dec_72();
-        const int r = tid & 127;
+        // dQ_i (fp32, 128 x D) goes TMEM -> registers -> the shared-memory area of this stage's Q_i and
+        // dO_i (both dead once dK and dV of this tile are done) in 128-byte-swizzled rows of 32
+        // floats, and from there to the global fp32 accumulator with TMA reduce-add: full lines
+        // to L2 instead of 16-byte scattered atomics.  Only then is the stage handed back.
+        setmaxnreg_dec_48();
+        const int r = ((warp & 3) << 5) | lane;
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
         for (int i = 0; i < n_q; ++i) {
             const int s = i & 1;
             mbar_wait(bar(kBarDqFull + s), (i >> 1) & 1, abort_flag, p.status, 150);
+            mbar_wait(bar(kBarDvDone + s), (i >> 1) & 1, abort_flag, p.status, 151);
             tc_fence_after();
-            const int32_t q = i * kTile + r;
-            float* dst = p.dq_acc + ((size_t)(node0 + q) * p.n_heads + h) * D;
+            uint8_t* stage = smem + L::kQ + s * L::kStageBytes;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t o[32];
                 tmem_ld32(tmem + kColDq + s * 64 + c * 32 + lane_off, o);
                 tmem_wait_ld();
-                if (q < n_g) {
+                uint8_t* row = stage + c * 16384 + r * 128;
 #pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        red_add_v4(dst + c * 32 + 4 * k, __uint_as_float(o[4 * k]), __uint_as_float(o[4 * k + 1]),
-                                   __uint_as_float(o[4 * k + 2]), __uint_as_float(o[4 * k + 3]));
-                }
+                for (int k = 0; k < 8; ++k)
+                    *(uint4*)(row + ((k ^ (r & 7)) << 4)) = make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
             }
             tc_fence_before();
             mbar_arrive(bar(kBarDqFree + s));
+            fence_proxy_async_smem();
+            named_barrier_sync(kNbDqStaged, 128);
+            if (warp == 20) {
+                if (elect_one()) {
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c)
+                        tma_reduce_add_2d(&tmap_dq, smem_u32(stage + c * 16384), h * D + c * 32, node0 + i * kTile);
+                    bulk_commit_group();
+                    bulk_wait_group_read0();
+                    mbar_arrive(bar(kBarStageEmpty + s));
+                    if (i + 1 == n_q) bulk_wait_group0();      // all adds have landed before the CTA retires
+                }
+                __syncwarp();
+            }
         }
     }
 
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) __nanosleep(200000);
-    if (warp == 1) tmem_dealloc(tmem, 512);
+    if (warp == 2) tmem_dealloc(tmem, 512);
 }
 
 // Delta[h][t] = sum_c dO[t,h,c] * O[t,h,c];  lse2[h][t] = lse[h][t] * log2(e).
@@ -521,18 +566,18 @@ BwdWorkspace bwd_workspace(const gt_batch* b, int32_t n_heads, int32_t head_dim,
 
 template <int D>
 gt_status launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
-                     const BwdParams& p, const gt_batch* batch, cudaStream_t s)
+                     const CUtensorMap& tspd, const BwdParams& p, const gt_batch* batch, cudaStream_t s)
 {
     dim3 grid((unsigned)p.n_heads, (unsigned)((batch->max_seqlen + kTile - 1) / kTile), (unsigned)batch->n_graphs);
-    if (p.n_buckets <= kPrivateBinBuckets) {
-        auto kern = attn_bwd_kernel<D, true>;
-        GT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kDynamic));
-        kern<<<grid, kBwdThreads, BwdSmem<D>::kDynamic, s>>>(tq, tk, tv, tdo, p);
-    } else {
-        auto kern = attn_bwd_kernel<D, false>;
-        GT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<D>::kDynamic));
-        kern<<<grid, kBwdThreads, BwdSmem<D>::kDynamic, s>>>(tq, tk, tv, tdo, p);
-    }
+    CUtensorMap tdq;
+    gt_status st_map = encode_dq_map(&tdq, p.dq_acc, p.n_total, p.n_heads, D);
+    if (st_map != GT_OK) return st_map;
+    const bool priv = p.n_buckets <= kMaxPrivateBinBuckets;
+    const size_t smem = BwdSmem<D>::dynamic_bytes(priv ? p.n_buckets * kSoftmaxThreads : p.n_buckets * 32);
+    auto kern = priv ? (p.n_buckets <= 32 ? attn_bwd_kernel<D, true, true> : attn_bwd_kernel<D, true, false>)
+                     : (p.n_buckets <= 32 ? attn_bwd_kernel<D, false, true> : attn_bwd_kernel<D, false, false>);
+    GT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kern<<<grid, kBwdThreads, smem, s>>>(tq, tk, tv, tdo, tspd, tdq, p);
     GT_CUDA_TRY(cudaGetLastError());
     return GT_OK;
 }
@@ -575,7 +620,10 @@ extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void
     uint8_t* ws = (uint8_t*)workspace;
     const size_t rows = (size_t)batch->n_total * n_heads;
     const int32_t n_db = n_heads * (max_dist + 2);
+    CUtensorMap tspd = tq;                       // placeholder when the cp.async loader is used
     BwdParams p{};
+    p.spd_tma = batch->n_graphs == 1 ? 1 : 0;
+    if (p.spd_tma && (st = encode_spd_map(&tspd, spd, batch->n_total, 128)) != GT_OK) return st;
     p.spd = spd;
     p.spd_offsets = batch->n_graphs > 1 ? spd_offsets : nullptr;
     p.cu_seqlens = batch->n_graphs > 1 ? batch->cu_seqlens : nullptr;
@@ -605,7 +653,7 @@ extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void
                                                              (float*)(ws + wsp.delta_off), (float*)(ws + wsp.lse2_off),
                                                              batch->n_total, n_heads);
     GT_CUDA_TRY(cudaGetLastError());
-    st = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, p, batch, s) : launch_bwd<32>(tq, tk, tv, tdo, p, batch, s);
+    st = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, tspd, p, batch, s) : launch_bwd<32>(tq, tk, tv, tdo, tspd, p, batch, s);
     if (st != GT_OK) return st;
     const size_t n_vec4 = rows * head_dim / 4;
     const size_t n_fin = n_vec4 > (size_t)n_db ? n_vec4 : (size_t)n_db;

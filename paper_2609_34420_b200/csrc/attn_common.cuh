@@ -16,6 +16,15 @@ constexpr float kLn2 = 0.6931471805599453f;
 // swizzle mode that matches the row length (128B for d=64, 64B for d=32).
 gt_status encode_thd_map(CUtensorMap* map, const void* base, int32_t n_total, int32_t n_heads, int32_t head_dim);
 
+// 2-D tensor map over the uint8 SPD matrix of a single graph (n rows of pitch round_up(n,16));
+// one box = box_rows rows x 128 key columns, written with the 128-byte swizzle (16-byte chunk c
+// of row r lands at chunk c ^ (r & 7)); out-of-range rows / columns are zero-filled.
+gt_status encode_spd_map(CUtensorMap* map, const uint8_t* spd, int32_t n, int32_t box_rows);
+
+// 2-D tensor map over the fp32 dQ accumulator [T, H*d]; one box = 128 rows x 32 floats of one
+// head, 128-byte swizzle (target of the backward kernel's TMA reduce-add).
+gt_status encode_dq_map(CUtensorMap* map, const float* dq_acc, int32_t n_total, int32_t n_heads, int32_t head_dim);
+
 struct AttnArgsCheck {
     const void* ptrs[12];
     int n_ptrs;
