@@ -9,8 +9,14 @@
 // gradient dB[h][b] = sum of dS over pairs in bucket b is binned in shared memory (one
 // private bin column per thread, no conflicts) and flushed once per CTA with fp64 atomics.
 //
-//   warp 0        TMA producer: K, V once; Q_i, dO_i and (single graph) the SPD tile, 2-stage ring
-//   warp 1        aux loader: lse*log2(e) and Delta of the query tile; SPD tile for packed batches
+// Because the scores are transposed, a thread walks along QUERY indices for a fixed key, i.e.
+// down a column of the SPD matrix.  A pre-pass therefore writes a transposed copy of the SPD
+// matrix into the workspace (values clamped to the last bucket on the way), so that the kernel
+// reads each thread's 32 bucket bytes as two 16-byte words instead of 32 byte loads.
+//
+//   warp 0        TMA producer: K, V once; Q_i, dO_i and (single graph) the SPD^T tile, 2-stage ring
+//   warp 1        aux loader: lse*log2(e) and Delta of the query tile; SPD^T tile for packed batches
+//   warp 2        issues S^T = K Q_i^T of the next query tile (not urgent, so it can live in a helper warp)
 //   warps 4-19    sixteen softmax warps = four groups of 128 threads; group g owns query columns
 //                 [32g, 32g+32) of the tile (32 score elements per thread).  Many warps rather than
 //                 long rows per thread: the per-element work is a chain of dependent shared-memory
@@ -39,7 +45,7 @@ constexpr int kColsPerThread = 32;
 constexpr int kMaxPrivateBinBuckets = 28;   // 2 KB of shared memory per bucket
 
 struct BwdParams {
-    const uint8_t* spd;
+    const uint8_t* spd_t;    // transposed, clamped copy of the SPD blocks (workspace)
     const int64_t* spd_offsets;
     const int32_t* cu_seqlens;
     const float* bias;
@@ -130,7 +136,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     const int32_t kv0 = (int32_t)blockIdx.y * kTile;
     if (kv0 >= n_g) return;
     const int64_t ld = (int64_t)((n_g + 15) & ~15);
-    const uint8_t* spd_g = p.spd + (p.spd_offsets ? p.spd_offsets[g] : 0);
+    const uint8_t* spd_g = p.spd_t + (p.spd_offsets ? p.spd_offsets[g] : 0);
     const int32_t n_q = (n_g + kTile - 1) / kTile;
 
     uint64_t* bars = (uint64_t*)(smem + L::kBars);
@@ -192,8 +198,31 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     tma_load_3d(smem_u32(smem + L::kDo + s * L::kStageBytes), &tmap_do, bar(kBarQdoFull + s), 0, h, row);
                     if (p.spd_tma) {
                         mbar_arrive_expect_tx(bar(kBarAuxFull + s), L::kSpdBytes);
-                        tma_load_2d(smem_u32(smem + L::kSpd + s * L::kSpdBytes), &tmap_spd, bar(kBarAuxFull + s), kv0, i * kTile);
+                        tma_load_2d(smem_u32(smem + L::kSpd + s * L::kSpdBytes), &tmap_spd, bar(kBarAuxFull + s), i * kTile, kv0);
                     }
+                }
+                __syncwarp();
+            }
+        } else if (warp == 2) {
+            // ------------------------------ S^T issuer ------------------------------
+            // S^T of the NEXT query tile is not urgent (it is consumed a whole tile later), so it is
+            // issued from this otherwise idle warp as soon as Q_{i} has landed and dV of the previous
+            // tile (which reads P^T from the same TMEM columns) has completed; no softmax warp waits.
+            constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
+            const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+            mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 160);
+            for (int i = 0; i < n_q; ++i) {
+                const int s = i & 1;
+                mbar_wait(bar(kBarQdoFull + s), (i >> 1) & 1, abort_flag, p.status, 161);
+                if (i > 0) mbar_wait(bar(kBarDvDone + (s ^ 1)), ((i - 1) >> 1) & 1, abort_flag, p.status, 162);
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint64_t da = make_smem_desc(smem_u32(smem + L::kK), L::kRowBytes, 0);
+                    const uint64_t db = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes), L::kRowBytes, 0);
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        mma_ss(tm + kColS, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
+                    mma_commit(bar(kBarSFull));
                 }
                 __syncwarp();
             }
@@ -210,9 +239,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     for (int it = 0; it < (kTile * 8) / 32; ++it) {
                         const int c = it * 32 + lane;
                         const int r = c >> 3, cc = c & 7;
-                        const int64_t col = (int64_t)kv0 + cc * 16;
-                        const bool valid = (q0 + r < n_g) && (col < ld);
-                        const uint8_t* src = valid ? spd_g + (int64_t)(q0 + r) * ld + col : spd_g;
+                        const int64_t col = (int64_t)q0 + cc * 16;
+                        const bool valid = (kv0 + r < n_g) && (col < ld);
+                        const uint8_t* src = valid ? spd_g + (int64_t)(kv0 + r) * ld + col : spd_g;
                         cp_async_16(dst0 + r * 128 + ((cc ^ (r & 7)) << 4), src, valid ? 16u : 0u);
                     }
                 }
@@ -239,37 +268,21 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const uint32_t tDp = tmem + kColDp + grp * 32 + lane_off;
         const bool kv_valid = kv0 + r < n_g;
         const float c1 = p.c1;
-        const uint32_t nb_m1 = (uint32_t)p.n_buckets - 1u;
         const float tbl = s_bias[lane];
         float* my_bins = s_bins + (kPrivateBins ? st : lane);
         constexpr int kBinStride = kPrivateBins ? kSoftmaxThreads : 32;
-        // byte (q, r) of the swizzled SPD tile sits at q*128 + (((r>>4) ^ (q&7)) << 4) + (r&15); q&7 == c&7
-        uint32_t spd_off[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) spd_off[k] = (grp * 32) * 128 + ((((uint32_t)r >> 4) ^ k) << 4) + (r & 15);
+        // the thread's 32 bucket bytes: row r of the SPD^T tile, 16-byte chunks 2 grp and 2 grp + 1 (swizzled by r & 7)
+        const uint32_t spd_off0 = r * 128 + (((2 * grp) ^ (r & 7)) << 4), spd_off1 = r * 128 + (((2 * grp + 1) ^ (r & 7)) << 4);
+        const uint32_t bins_base = smem_u32(my_bins);
 
         // ---- MMA issue duty (after the barriers of all softmax threads) ----
-        const bool issuer_a = warp == 4;                // dV, S^T
+        const bool issuer_a = warp == 4;                // dV
         const bool issuer_b = warp == 9;                // dK, dQ, dP^T
         constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
         constexpr uint32_t idesc_ts = make_idesc_bf16(128, D, false, true);    // A in TMEM, B MN-major
         constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);     // A and B MN-major
         const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
         const uint32_t sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV);
-        auto issue_st = [&](int i) {                    // S^T = K Q_i^T
-            const int s = i & 1;
-            mbar_wait(bar(kBarQdoFull + s), (i >> 1) & 1, abort_flag, p.status, 120);
-            tc_fence_after();
-            if (elect_one()) {
-                const uint64_t da = make_smem_desc(sK, L::kRowBytes, 0);
-                const uint64_t db = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes), L::kRowBytes, 0);
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ss(tm + kColS, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
-                mma_commit(bar(kBarSFull));
-            }
-            __syncwarp();
-        };
         auto issue_dpt = [&](int i) {                   // dP^T = V dO_i^T
             const int s = i & 1;
             mbar_wait(bar(kBarQdoFull + s), (i >> 1) & 1, abort_flag, p.status, 121);
@@ -284,13 +297,11 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             }
             __syncwarp();
         };
-        if (issuer_a) { mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 122); issue_st(0); }
         if (issuer_b) { mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 123); issue_dpt(0); }
 
         for (int i = 0; i < n_q; ++i) {
             const int s = i & 1;
             float pr[kColsPerThread];
-            uint32_t bkp[kColsPerThread / 4];       // the 32 bucket bytes of this thread's elements, clamped
             // ---------------- P^T = exp2(S^T c1 + b2 - lse2) ----------------
             mbar_wait(bar(kBarSFull), i & 1, abort_flag, p.status, 140);
             tc_fence_after();
@@ -298,6 +309,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             tmem_ld32(tS, acc);
             mbar_wait(bar(kBarAuxFull + s), (i >> 1) & 1, abort_flag, p.status, 141);
             const uint8_t* spd_tile = smem + L::kSpd + s * L::kSpdBytes;
+            const uint4 w0 = *(const uint4*)(spd_tile + spd_off0), w1 = *(const uint4*)(spd_tile + spd_off1);
+            const uint32_t bw[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};   // bucket bytes, already clamped
             const float4* lse4 = (const float4*)(smem + L::kLse + s * 512 + grp * 128);
             tmem_wait_ld();
 #pragma unroll
@@ -306,9 +319,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 #pragma unroll
                 for (int k = 0; k < 16; ++k) {
                     const int c = rnd * 16 + k;
-                    const uint32_t b = min((uint32_t)spd_tile[spd_off[c & 7] + c * 128], nb_m1);   // never index past the bins
-                    bb[k] = kShflBias ? __shfl_sync(0xffffffffu, tbl, b) : s_bias[b];
-                    bkp[c >> 2] = (c & 3) == 0 ? b : (bkp[c >> 2] | (b << (8 * (c & 3))));
+                    const uint32_t sh = bw[c >> 2] >> (8 * (c & 3));         // the shuffle only looks at the low 5 bits
+                    bb[k] = kShflBias ? __shfl_sync(0xffffffffu, tbl, sh) : s_bias[sh & 0xffu];
                 }
 #pragma unroll
                 for (int k4 = 0; k4 < 4; ++k4) {
@@ -348,7 +360,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     if (i + 1 == n_q) mma_commit(bar(kBarFinal));
                 }
                 __syncwarp();
-                if (i + 1 < n_q) issue_st(i + 1);
             }
 
             // ---------------- dS^T = P^T o (dP^T - Delta) ----------------
@@ -373,9 +384,18 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 #pragma unroll
                 for (int k = 0; k < 16; ++k) {
                     const int c = rnd * 16 + k;
-                    const uint32_t b = (bkp[c >> 2] >> (8 * (c & 3))) & 0xffu;
-                    if (kPrivateBins) my_bins[b * kBinStride] += pr[c];
-                    else atomicAdd(&my_bins[b * kBinStride], pr[c]);
+                    // byte offset of bin b: b * stride * 4, formed by one funnel shift and one mask
+                    constexpr int kLog = kPrivateBins ? 11 : 7;               // log2(kBinStride * 4)
+                    const int sh = 8 * (c & 3) - kLog;
+                    const uint32_t off = (sh >= 0 ? (bw[c >> 2] >> (sh >= 0 ? sh : 0)) : (bw[c >> 2] << (sh < 0 ? -sh : 0))) & (0xffu << kLog);
+                    if (kPrivateBins) {
+                        float v;
+                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(bins_base + off));
+                        v += pr[c];
+                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(bins_base + off), "f"(v));
+                    } else {
+                        atomicAdd((float*)((uint8_t*)my_bins + off), pr[c]);
+                    }
                 }
             }
             {
@@ -507,6 +527,42 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     if (warp == 2) tmem_dealloc(tmem, 512);
 }
 
+// spd_t[j][i] = min(spd[i][j], n_buckets - 1) for every graph block (same offsets and pitch as the
+// source).  64 x 64 byte tiles through shared memory; reads and writes are both coalesced.
+__global__ void __launch_bounds__(256) spd_transpose_clamp_kernel(const uint8_t* __restrict__ spd, uint8_t* __restrict__ spd_t,
+                                                                  const int64_t* __restrict__ spd_offsets,
+                                                                  const int32_t* __restrict__ cu_seqlens, int32_t n_total,
+                                                                  uint32_t last_bucket)
+{
+    __shared__ uint8_t tile[64][64 + 4];
+    const int g = blockIdx.z;
+    const int32_t n_g = cu_seqlens ? cu_seqlens[g + 1] - cu_seqlens[g] : n_total;
+    const int32_t i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
+    if (i0 >= n_g || j0 >= n_g) return;
+    const int64_t ld = (int64_t)((n_g + 15) & ~15);
+    const int64_t base = spd_offsets ? spd_offsets[g] : 0;
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;          // 16 x 16 threads, 4 bytes x 4 rows each
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int i = i0 + ty * 4 + k, j = j0 + tx * 4;
+        uint32_t w = 0;
+        if (i < n_g && j < ld) w = *(const uint32_t*)(spd + base + (int64_t)i * ld + j);
+#pragma unroll
+        for (int b = 0; b < 4; ++b) tile[ty * 4 + k][tx * 4 + b] = (uint8_t)min((w >> (8 * b)) & 0xffu, last_bucket);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int j = j0 + ty * 4 + k, i = i0 + tx * 4;               // output row j (old column), columns i..i+3
+        if (j < n_g && i < ld) {
+            uint32_t w = 0;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) w |= (uint32_t)tile[tx * 4 + b][ty * 4 + k] << (8 * b);
+            *(uint32_t*)(spd_t + base + (int64_t)j * ld + i) = w;
+        }
+    }
+}
+
 // Delta[h][t] = sum_c dO[t,h,c] * O[t,h,c];  lse2[h][t] = lse[h][t] * log2(e).
 template <int D>
 __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
@@ -549,7 +605,7 @@ __global__ void bwd_finalize_kernel(const float* __restrict__ dq_acc, __nv_bfloa
 }
 
 struct BwdWorkspace {
-    size_t db_off, delta_off, lse2_off, dq_off, total;
+    size_t db_off, delta_off, lse2_off, dq_off, spdt_off, total;
 };
 
 BwdWorkspace bwd_workspace(const gt_batch* b, int32_t n_heads, int32_t head_dim, int32_t max_dist)
@@ -560,7 +616,9 @@ BwdWorkspace bwd_workspace(const gt_batch* b, int32_t n_heads, int32_t head_dim,
     w.delta_off = w.db_off + align_up((size_t)n_heads * (max_dist + 2) * sizeof(double), 256);
     w.lse2_off = w.delta_off + align_up(rows * sizeof(float), 256);
     w.dq_off = w.lse2_off + align_up(rows * sizeof(float), 256);
-    w.total = w.dq_off + align_up(rows * head_dim * sizeof(float), 256);
+    w.spdt_off = w.dq_off + align_up(rows * head_dim * sizeof(float), 256);
+    // transposed SPD copy: at most sum n_g * round_up(n_g,16) <= n_total * round_up(max_seqlen,16) bytes
+    w.total = w.spdt_off + align_up((size_t)b->n_total * (size_t)((b->max_seqlen + 15) & ~15), 256);
     return w;
 }
 
@@ -623,8 +681,9 @@ extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void
     CUtensorMap tspd = tq;                       // placeholder when the cp.async loader is used
     BwdParams p{};
     p.spd_tma = batch->n_graphs == 1 ? 1 : 0;
-    if (p.spd_tma && (st = encode_spd_map(&tspd, spd, batch->n_total, 128)) != GT_OK) return st;
-    p.spd = spd;
+    uint8_t* spd_t = ws + wsp.spdt_off;
+    if (p.spd_tma && (st = encode_spd_map(&tspd, spd_t, batch->n_total, 128)) != GT_OK) return st;
+    p.spd_t = spd_t;
     p.spd_offsets = batch->n_graphs > 1 ? spd_offsets : nullptr;
     p.cu_seqlens = batch->n_graphs > 1 ? batch->cu_seqlens : nullptr;
     p.bias = bias;
@@ -643,6 +702,13 @@ extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void
 
     GT_CUDA_TRY(cudaMemsetAsync(ws + wsp.db_off, 0, (size_t)n_db * sizeof(double), s));
     GT_CUDA_TRY(cudaMemsetAsync(ws + wsp.dq_off, 0, rows * head_dim * sizeof(float), s));
+    {
+        const unsigned tiles = (unsigned)((batch->max_seqlen + 63) / 64);
+        dim3 tgrid(tiles, tiles, (unsigned)batch->n_graphs);
+        spd_transpose_clamp_kernel<<<tgrid, 256, 0, s>>>(spd, spd_t, p.spd_offsets, p.cu_seqlens, batch->n_total,
+                                                         (uint32_t)(max_dist + 1));
+        GT_CUDA_TRY(cudaGetLastError());
+    }
     const unsigned pre_blocks = (unsigned)((rows + 255) / 256);
     if (head_dim == 64)
         bwd_preprocess_kernel<64><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse,
