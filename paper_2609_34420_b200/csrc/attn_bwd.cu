@@ -104,10 +104,6 @@ __device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src, uint32
 {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d)
-{
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
 // register budget: the CTA is launched with 768 x 80 registers; after the re-split it holds
 // 128 x 40 + 512 x 96 + 128 x 48 = 60416 <= 61440 (an increase can only draw on what the CTA owns)
 __device__ __forceinline__ void setmaxnreg_inc_96() { asm volatile("setmaxnreg.inc.sync.aligned.u32 96;"); }
@@ -270,7 +266,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const float c1 = p.c1;
         const float tbl = s_bias[lane];
         float* my_bins = s_bins + (kPrivateBins ? st : lane);
-        constexpr int kBinStride = kPrivateBins ? kSoftmaxThreads : 32;
         // the thread's 32 bucket bytes: row r of the SPD^T tile, 16-byte chunks 2 grp and 2 grp + 1 (swizzled by r & 7)
         const uint32_t spd_off0 = r * 128 + (((2 * grp) ^ (r & 7)) << 4), spd_off1 = r * 128 + (((2 * grp + 1) ^ (r & 7)) << 4);
         const uint32_t bins_base = smem_u32(my_bins);
