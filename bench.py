@@ -37,8 +37,8 @@ DEFAULT_WORKLOAD = "powerlaw64k"
 ORACLE_SAMPLE_ROWS = 256
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the backward kernel, from the ncu
-# capture summarised under profiles/ (captured on a smaller graph and scaled by N^2); None until measured.
-BWD_KERNEL_DRAM_BYTES_PER_N2 = None
+# capture summarised in profiles/attn_bwd_kernel_powerlaw16k.md (16 384-node graph, scaled by N^2).
+BWD_KERNEL_DRAM_BYTES_PER_N2 = 1013.9e6 / (16384.0 ** 2)
 
 
 def load_peaks():
@@ -222,7 +222,7 @@ def run_cuda(args) -> int:
         if marks is not None:
             marks[4].record()
 
-    kernels_per_step = 2 + 1 + 3 + (2 if single else 0)     # spd(setup,bfs) fwd bwd(pre,main,finalize) chunked(partial,merge)
+    kernels_per_step = 2 + 1 + 4 + (2 if single else 0)     # spd(setup,bfs) fwd bwd(transpose,pre,main,finalize) chunked(partial,merge)
 
     for _ in range(max(args.warmup, 0)):
         step()

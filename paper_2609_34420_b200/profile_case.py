@@ -1,0 +1,81 @@
+"""Run the hot path a few times on one named workload and print CUDA-event timings.
+
+    python -m paper_2609_34420_b200.profile_case WORKLOAD [REPS] [spd|fwd|bwd|chunked|all]
+
+WORKLOAD is one of the named workloads (tiny_er256, ba4096, powerlaw16k, powerlaw64k,
+varlen_rgg64) or plN for a power-law graph of N nodes (H=8, d=64, max_dist=24).  It is the small,
+self-contained target used for the ncu captures summarised under profiles/.
+"""
+from __future__ import annotations
+
+import sys
+
+import torch
+
+from . import binding as gt
+from . import workloads as wl
+
+
+def main(argv) -> int:
+    name = argv[1] if len(argv) > 1 else "powerlaw16k"
+    reps = int(argv[2]) if len(argv) > 2 else 1
+    what = argv[3] if len(argv) > 3 else "all"
+    if name.startswith("pl") and name[2:].isdigit():
+        w = wl.Workload(name, wl.pack_graphs([wl.chung_lu_power_law(int(name[2:]), 12.0, 2.1, 0)]), 8, 64, 24)
+    else:
+        w = wl.make_workload(name)
+    b = w.batch
+    T, H, d, D = b.n_total, w.n_heads, w.head_dim, w.max_dist
+    dev = torch.device("cuda", 0)
+    single = b.n_graphs == 1
+    batch = gt.Batch(T, b.n_graphs, b.max_seqlen,
+                     None if single else torch.from_numpy(b.cu_seqlens).to(dev),
+                     None if single else torch.from_numpy(b.spd_offsets).to(dev))
+    rp, ci = torch.from_numpy(b.row_ptr).to(dev), torch.from_numpy(b.col_idx).to(dev)
+    g = torch.Generator(device=dev).manual_seed(1)
+    q, k, v, do = (torch.randn(T, H, d, device=dev, generator=g).bfloat16() for _ in range(4))
+    bias = torch.randn(H, D + 2, device=dev, generator=g) * 0.5
+    spd = torch.empty(b.spd_bytes, dtype=torch.uint8, device=dev)
+    out, dq, dk, dv, out_c = (torch.empty_like(q) for _ in range(5))
+    lse, lse_c = torch.empty(H, T, device=dev), torch.empty(H, T, device=dev)
+    dbias = torch.empty_like(bias)
+    ws_spd = gt.gt_spd_build(rp, ci, batch, D, spd)
+    ws_fwd = gt.gt_biased_attn_fwd(q, k, v, spd, bias, batch, D, out, lse)
+    ws_bwd = gt.gt_biased_attn_bwd(q, k, v, out, do, lse, spd, bias, batch, D, dq, dk, dv, dbias)
+    for ws in (ws_spd, ws_fwd, ws_bwd):
+        gt.gt_check(ws)
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    f_fwd, f_bwd = w.attn_flops()
+    if what in ("all", "spd"):
+        ms = timed(lambda: gt.gt_spd_build(rp, ci, batch, D, spd, ws_spd))
+        print(f"spd_build {ms:.3f} ms  {b.spd_bytes / ms / 1e6:.1f} GB/s")
+    if what in ("all", "fwd"):
+        ms = timed(lambda: gt.gt_biased_attn_fwd(q, k, v, spd, bias, batch, D, out, lse, ws_fwd))
+        print(f"fwd {ms:.3f} ms  {f_fwd / ms / 1e9:.1f} TFLOP/s")
+    if what in ("all", "bwd"):
+        ms = timed(lambda: gt.gt_biased_attn_bwd(q, k, v, out, do, lse, spd, bias, batch, D, dq, dk, dv, dbias, ws_bwd))
+        print(f"bwd {ms:.3f} ms  {f_bwd / ms / 1e9:.1f} TFLOP/s")
+    if what in ("all", "chunked") and single:
+        ws_c = gt.gt_biased_attn_fwd_chunked(q, k, v, spd, bias, batch, D, out_c, lse_c, max(w.n_kv_chunks, 2))
+        ms = timed(lambda: gt.gt_biased_attn_fwd_chunked(q, k, v, spd, bias, batch, D, out_c, lse_c,
+                                                         max(w.n_kv_chunks, 2), None, ws_c))
+        print(f"fwd_chunked {ms:.3f} ms  {f_fwd / ms / 1e9:.1f} TFLOP/s")
+        gt.gt_check(ws_c)
+    for ws in (ws_spd, ws_fwd, ws_bwd):
+        gt.gt_check(ws)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main(sys.argv))

@@ -1,0 +1,85 @@
+"""Parity at the full sizes the benchmark times (same entry points, same launch configuration).
+
+The fp64 oracle cannot materialise 65536^2 scores per head in test time, so attention is checked
+with the row-slab protocol: the oracle computes full rows for a seeded subset R of query rows
+(forward O, LSE and dQ on R); the GPU backward is run with dO zeroed outside R, which makes dK, dV
+and dBias depend on the rows of R only, so they are compared with the oracle's sums over R.
+The SPD matrix is compared in full (bit-exact)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention as oattn
+from oracle import spd as ospd
+from paper_2609_34420_b200 import binding as gt
+from paper_2609_34420_b200 import workloads as wl
+
+from gpu_util import bf16_tensor, device_batch, device_csr, rel_l2, to_f64
+
+pytestmark = pytest.mark.gpu
+
+O_MAX_ABS, LSE_MAX_ABS, GRAD_REL_L2, CHUNK_REL_L2 = 1e-2, 1e-3, 2e-2, 1e-3
+
+
+def run_large(name: str, n_slab: int, full_spd_oracle: bool):
+    w = wl.make_workload(name)
+    b, t = w.batch, w.tensors()
+    n, H, d, D = b.n_total, w.n_heads, w.head_dim, w.max_dist
+    dev = "cuda"
+    bt = device_batch(b, dev)
+    rp, ci = device_csr(b, dev)
+
+    # ---- SPD: GPU build, bit-exact against the BFS oracle ----
+    spd = torch.empty(b.spd_bytes, dtype=torch.uint8, device=dev)
+    gt.gt_check(gt.gt_spd_build(rp, ci, bt, D, spd))
+    rows = np.sort(np.random.default_rng(2024).choice(n, size=n_slab, replace=False))
+    ld = int(b.spd_ld[0])
+    if full_spd_oracle:
+        ref = ospd.spd_matrix(b.row_ptr, b.col_idx, D)
+        got = spd.cpu().numpy().reshape(n, ld)
+        assert np.array_equal(got, ref)
+        spd_rows = np.ascontiguousarray(ref[rows])
+        del ref, got
+    else:
+        spd_rows = ospd.spd_rows(b.row_ptr, b.col_idx, D, rows)
+        got_rows = spd.view(n, ld)[torch.from_numpy(rows).to(dev)].cpu().numpy()
+        assert np.array_equal(got_rows, spd_rows)
+
+    # ---- forward (unchunked and chunked) ----
+    q, k, v, do = (bf16_tensor(x, dev) for x in (t.q, t.k, t.v, t.dout))
+    bias = torch.tensor(t.bias, device=dev)
+    out, out_c = torch.empty_like(q), torch.empty_like(q)
+    lse, lse_c = torch.empty(H, n, device=dev), torch.empty(H, n, device=dev)
+    gt.gt_check(gt.gt_biased_attn_fwd(q, k, v, spd, bias, bt, D, out, lse))
+    gt.gt_check(gt.gt_biased_attn_fwd_chunked(q, k, v, spd, bias, bt, D, out_c, lse_c, max(w.n_kv_chunks, 2)))
+    assert rel_l2(to_f64(out_c), to_f64(out)) <= CHUNK_REL_L2
+    assert (lse_c - lse).abs().max().item() <= LSE_MAX_ABS
+
+    f = wl.bf16_bits_to_f64
+    qf, kf, vf, dof, bf = f(t.q), f(t.k), f(t.v), f(t.dout), t.bias.astype(np.float64)
+    ro, rl = oattn.forward_single(qf, kf, vf, spd_rows, bf, rows=rows, compact_spd=True)
+    rows_t = torch.from_numpy(rows).to(dev)
+    assert np.abs(to_f64(out[rows_t]) - ro).max() <= O_MAX_ABS
+    assert np.abs(to_f64(lse[:, rows_t]) - rl).max() <= LSE_MAX_ABS
+
+    # ---- backward with dO restricted to the slab ----
+    do_masked = torch.zeros_like(do)
+    do_masked[rows_t] = do[rows_t]
+    dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+    dbias = torch.empty_like(bias)
+    gt.gt_check(gt.gt_biased_attn_bwd(q, k, v, out, do_masked, lse, spd, bias, bt, D, dq, dk, dv, dbias))
+    rdq, rdk, rdv, rdb = oattn.backward_single(qf, kf, vf, dof, spd_rows, bf, rows=rows, compact_spd=True)
+    errs = {"dq": rel_l2(to_f64(dq[rows_t]), rdq), "dk": rel_l2(to_f64(dk), rdk),
+            "dv": rel_l2(to_f64(dv), rdv), "dbias": rel_l2(to_f64(dbias), rdb)}
+    assert all(e <= GRAD_REL_L2 for e in errs.values()), errs
+    mask = torch.ones(n, dtype=torch.bool, device=dev)
+    mask[rows_t] = False
+    assert (dq[mask].float().abs().max().item() == 0.0)
+
+
+def test_powerlaw16k_full_spd_and_row_slab_attention():
+    run_large("powerlaw16k", n_slab=384, full_spd_oracle=True)
+
+
+def test_powerlaw64k_full_spd_and_row_slab_attention():
+    run_large("powerlaw64k", n_slab=128, full_spd_oracle=True)
