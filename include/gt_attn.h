@@ -93,6 +93,35 @@ gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx, int64_t n
                        void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------
+ * gt_spd_build_static -- gt_spd_build without a workspace argument.  (No counterpart in the
+ * paper: it exists for the way this library is embedded, not for the method.)
+ *
+ * Some callers cannot hand over scratch memory because they may not allocate on the device at
+ * all: a plug-in running inside a host application that owns the GPU allocator, a latency-critical
+ * loop in which a device allocation would stall every stream, or code that runs after the process
+ * has pinned its memory budget.  For them the scratch of the SPD build lives inside the library,
+ * in a fixed array of gt_spd_build_static_limit() bytes (1 MiB) that every GPU loading the library
+ * holds until the process exits.  The call itself allocates and frees nothing.
+ *
+ * Same arguments, results and error codes as gt_spd_build, minus the workspace, with these rules:
+ *  - Size limit: the batch must satisfy gt_spd_build_workspace(batch, nnz, max_dist) <=
+ *    gt_spd_build_static_limit(); in practice every graph of the batch has at most 17 066 nodes
+ *    (larger graphs keep their traversal state in the workspace and need far more).  Otherwise
+ *    GT_ERR_WORKSPACE is returned and nothing is launched.
+ *  - First call per device: the first call made with a given device current looks up the
+ *    device address of the built-in array (a one-off set-up step).  Make that first call outside
+ *    any stream capture.
+ *  - One array per device, shared by all calls: it still holds what the previous call left (the
+ *    call clears the words that must start at zero), and two calls whose GPU work overlaps --
+ *    different streams, or different host threads -- race on it.  Serialise them, or give the
+ *    concurrent ones their own workspace through gt_spd_build.
+ * ------------------------------------------------------------------------------------- */
+size_t gt_spd_build_static_limit(void);
+gt_status gt_spd_build_static(const int32_t* row_ptr, const int32_t* col_idx, int64_t nnz,
+                              const gt_batch* batch, int32_t max_dist,
+                              const int64_t* spd_offsets, uint8_t* spd_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------
  * gt_biased_attn_fwd -- Eq. 1, forward.  For every graph, head h and query row i:
  *     S_ij = (q_i . k_j)/sqrt(head_dim) + bias[h][spd_ij]        (all j of the same graph)
  *     out_i = sum_j softmax_j(S_i)_j v_j,     lse[h][i] = log sum_j exp(S_ij)  (natural log)

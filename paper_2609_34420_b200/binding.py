@@ -22,7 +22,7 @@ STATUS_NAMES = {0: "GT_OK", 1: "GT_ERR_INVALID_ARG", 2: "GT_ERR_UNSUPPORTED", 3:
                 4: "GT_ERR_CUDA", 5: "GT_ERR_DEVICE_TIMEOUT", 6: "GT_ERR_NO_DEVICE"}
 
 EXPORTS = ("gt_status_string", "gt_check",
-           "gt_spd_build_workspace", "gt_spd_build",
+           "gt_spd_build_workspace", "gt_spd_build", "gt_spd_build_static_limit", "gt_spd_build_static",
            "gt_biased_attn_fwd_workspace", "gt_biased_attn_fwd",
            "gt_biased_attn_bwd_workspace", "gt_biased_attn_bwd",
            "gt_biased_attn_fwd_chunked_workspace", "gt_biased_attn_fwd_chunked")
@@ -60,6 +60,11 @@ def lib() -> ctypes.CDLL:
         L.gt_spd_build_workspace.argtypes = [bp, i64, i32]
         L.gt_spd_build.restype = ctypes.c_int
         L.gt_spd_build.argtypes = [vp, vp, i64, bp, i32, vp, vp, vp, sz, vp]
+        if hasattr(L, "gt_spd_build_static"):
+            L.gt_spd_build_static_limit.restype = sz
+            L.gt_spd_build_static_limit.argtypes = []
+            L.gt_spd_build_static.restype = ctypes.c_int
+            L.gt_spd_build_static.argtypes = [vp, vp, i64, bp, i32, vp, vp, vp]
         if hasattr(L, "gt_biased_attn_fwd"):
             L.gt_biased_attn_fwd_workspace.restype = sz
             L.gt_biased_attn_fwd_workspace.argtypes = [bp, i32, i32]
@@ -139,6 +144,22 @@ def gt_spd_build(row_ptr: torch.Tensor, col_idx: torch.Tensor, batch: Batch, max
                             _ptr(batch.spd_offsets), _ptr(spd_out), _ptr(workspace), workspace.numel(), _stream())
     _raise(st, "gt_spd_build")
     return workspace
+
+
+def gt_spd_build_static_limit() -> int:
+    return int(lib().gt_spd_build_static_limit())
+
+
+def gt_spd_build_static(row_ptr: torch.Tensor, col_idx: torch.Tensor, batch: Batch, max_dist: int,
+                        spd_out: torch.Tensor) -> None:
+    """SPD build for callers that must not allocate: the scratch is a fixed array inside the
+    library (one per device, shared by every call, so calls that overlap on the GPU race).
+    Raises GtError(GT_ERR_WORKSPACE) when the batch needs more than gt_spd_build_static_limit()."""
+    nnz = int(col_idx.numel())
+    b = batch.c_struct()
+    st = lib().gt_spd_build_static(_ptr(row_ptr), _ptr(col_idx) if nnz else None, nnz, ctypes.byref(b), int(max_dist),
+                                   _ptr(batch.spd_offsets), _ptr(spd_out), _stream())
+    _raise(st, "gt_spd_build_static")
 
 
 def gt_biased_attn_fwd_workspace(batch: Batch, n_heads: int, head_dim: int) -> int:

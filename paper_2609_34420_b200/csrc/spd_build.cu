@@ -283,3 +283,65 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
     GT_CUDA_TRY(cudaGetLastError());
     return GT_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// gt_spd_build_static: the same build, for callers that may not allocate device memory.
+//
+// Its scratch (work counters, per-graph batch offsets) lives in the file-scope device array
+// below, so the caller passes inputs and outputs only.  The array costs kStaticScratchBytes
+// of device memory on every GPU that loads this library, until the process exits.
+// ------------------------------------------------------------------------------------------
+namespace gt {
+namespace {
+
+constexpr size_t kStaticScratchBytes = (size_t)1 << 20;      // 1 MiB
+static __device__ __align__(256) unsigned char g_spd_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+
+// Device address of the scratch array on the CURRENT device.  In host code the array's name is
+// only a stand-in for the symbol, not an address a kernel could use, so the address is looked
+// up once per device (with that device current) and remembered.
+gt_status static_scratch_ptr(void** out)
+{
+    static void* ptrs[kMaxDevices] = {nullptr};
+    int dev = -1;
+    GT_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return GT_ERR_UNSUPPORTED;
+    if (ptrs[dev] == nullptr) {
+        void* p = nullptr;
+        GT_CUDA_TRY(cudaGetSymbolAddress(&p, g_spd_static_scratch));
+        if (p == nullptr) return GT_ERR_CUDA;
+        ptrs[dev] = p;
+    }
+    *out = ptrs[dev];
+    return GT_OK;
+}
+
+}  // namespace
+}  // namespace gt
+
+extern "C" size_t gt_spd_build_static_limit(void) { return gt::kStaticScratchBytes; }
+
+extern "C" gt_status gt_spd_build_static(const int32_t* row_ptr, const int32_t* col_idx, int64_t nnz,
+                                         const gt_batch* batch, int32_t max_dist,
+                                         const int64_t* spd_offsets, uint8_t* spd_out, void* stream)
+{
+    using namespace gt;
+    gt_status st = validate_batch(batch);
+    if (st != GT_OK) return st;
+    if (sm_count() <= 0) return GT_ERR_NO_DEVICE;
+    const size_t need = gt_spd_build_workspace(batch, nnz, max_dist);
+    if (need == 0) return GT_ERR_INVALID_ARG;
+    if (need > kStaticScratchBytes) {
+        if (getenv("GT_DEBUG"))
+            fprintf(stderr, "[gt_attn] gt_spd_build_static: this batch needs %zu bytes of scratch, the built-in "
+                            "array holds %zu; use gt_spd_build with a caller workspace\n", need, kStaticScratchBytes);
+        return GT_ERR_WORKSPACE;
+    }
+    void* scratch = nullptr;
+    if ((st = static_scratch_ptr(&scratch)) != GT_OK) return st;
+    // the array keeps whatever the previous call left: status words and work counters start at zero
+    GT_CUDA_TRY(cudaMemsetAsync(scratch, 0, kHeaderBytes, (cudaStream_t)stream));
+    return gt_spd_build(row_ptr, col_idx, nnz, batch, max_dist, spd_offsets, spd_out, scratch, kStaticScratchBytes, stream);
+}
