@@ -297,10 +297,10 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         for (int i = 0; i < n_q; ++i) {
             const int s = i & 1;
             float pr[kColsPerThread];
+            uint32_t acc[32];
             // ---------------- P^T = exp2(S^T c1 + b2 - lse2) ----------------
             mbar_wait(bar(kBarSFull), i & 1, abort_flag, p.status, 140);
             tc_fence_after();
-            uint32_t acc[32];
             tmem_ld32(tS, acc);
             mbar_wait(bar(kBarAuxFull + s), (i >> 1) & 1, abort_flag, p.status, 141);
             const uint8_t* spd_tile = smem + L::kSpd + s * L::kSpdBytes;
@@ -341,6 +341,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 tmem_st16(tS, pk);                      // P^T of this group: 16 packed columns at the start of its range
                 tmem_wait_st();
             }
+            mbar_wait(bar(kBarDpFull), i & 1, abort_flag, p.status, 142);
+            tc_fence_after();
+            tmem_ld32(tDp, acc);                        // dP^T of this tile: its latency hides behind the barrier
             tc_fence_before();
             named_barrier_sync(kNbPStored, kSoftmaxThreads);
             if (issuer_a) {
@@ -358,9 +361,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             }
 
             // ---------------- dS^T = P^T o (dP^T - Delta) ----------------
-            mbar_wait(bar(kBarDpFull), i & 1, abort_flag, p.status, 142);
-            tc_fence_after();
-            tmem_ld32(tDp, acc);
             const float4* dl4 = (const float4*)(smem + L::kDelta + s * 512 + grp * 128);
             tmem_wait_ld();
 #pragma unroll

@@ -70,7 +70,7 @@ __global__ void spd_setup_kernel(SpdParams p)
 }
 
 template <bool kSmemState>
-__global__ void __launch_bounds__(1024, 1) spd_bfs_kernel(SpdParams p)
+__global__ void __launch_bounds__(1024, kSmemState ? 1 : 2) spd_bfs_kernel(SpdParams p)
 {
     extern __shared__ uint32_t smem_words[];
     __shared__ int32_t s_batch;
@@ -138,10 +138,19 @@ __global__ void __launch_bounds__(1024, 1) spd_bfs_kernel(SpdParams p)
                 }
                 const int deg = e1 - e0;
                 if (f && deg <= kWarpDegree) {
-                    for (int e = e0; e < e1; ++e) {
-                        int w = p.col_idx[e] - node0;
-                        uint32_t add = f & ~vis[w];
-                        if (add) atomicOr(&nxt[w], add);
+                    // four edges per round: the index loads, then the state loads, are issued together so
+                    // that their latencies overlap; bits that are already visited (or, with the state in shared
+                    // memory where the extra read is cheap, already pending) at the target need no atomic
+                    for (int e = e0; e < e1; e += 4) {
+                        int w[4];
+                        uint32_t add[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) w[k] = e + k < e1 ? p.col_idx[e + k] - node0 : -1;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) add[k] = w[k] >= 0 ? f & ~(kSmemState ? (vis[w[k]] | nxt[w[k]]) : vis[w[k]]) : 0u;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            if (add[k]) atomicOr(&nxt[w[k]], add[k]);
                     }
                 }
                 uint32_t big = __ballot_sync(0xffffffffu, f != 0u && deg > kWarpDegree);
@@ -151,10 +160,16 @@ __global__ void __launch_bounds__(1024, 1) spd_bfs_kernel(SpdParams p)
                     uint32_t ff = __shfl_sync(0xffffffffu, f, src_lane);
                     int b0 = __shfl_sync(0xffffffffu, e0, src_lane);
                     int b1 = __shfl_sync(0xffffffffu, e1, src_lane);
-                    for (int e = b0 + lane; e < b1; e += 32) {
-                        int w = p.col_idx[e] - node0;
-                        uint32_t add = ff & ~vis[w];
-                        if (add) atomicOr(&nxt[w], add);
+                    for (int e = b0 + lane; e < b1; e += 128) {
+                        int w[4];
+                        uint32_t add[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) w[k] = e + 32 * k < b1 ? p.col_idx[e + 32 * k] - node0 : -1;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) add[k] = w[k] >= 0 ? ff & ~(kSmemState ? (vis[w[k]] | nxt[w[k]]) : vis[w[k]]) : 0u;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            if (add[k]) atomicOr(&nxt[w[k]], add[k]);
                     }
                 }
             }
@@ -220,6 +235,7 @@ SpdPlan make_plan(const gt_batch* b)
         int by_threads = 2048 / pl.threads;
         per_sm = per_sm < 1 ? 1 : (per_sm > by_threads ? by_threads : per_sm);
     }
+    if (!pl.smem_state) per_sm = 2;      // state in L2: two CTAs per SM keep more loads in flight
     long want = (long)sms * per_sm;
     pl.grid = (int)(max_batches < want ? max_batches : want);
     pl.smem_bytes = pl.smem_state ? state : 0;
