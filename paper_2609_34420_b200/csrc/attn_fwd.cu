@@ -9,11 +9,15 @@
 // tensor pipe works on one tile while the other is in its softmax) x all key tiles of the
 // graph (or of one key chunk for the chunked entry point).
 //
-//   warp 0      TMA producer: Q once, then K/V tiles through a 2-stage ring
-//   warp 1      MMA issuer: S_t = Q_t K^T (SS), O_t += P_t V (A from TMEM, B = V as MN-major)
-//   warps 2-3   SPD loaders: 256x128-byte index tile per key tile via cp.async (3-stage ring),
-//               16-byte chunks XOR-swizzled by row so that the row-per-thread reads are conflict free
-//   warps 4-7   softmax of tile 0 (thread = query row = TMEM lane), warps 8-11 of tile 1
+//   warp 0      TMA producer: Q once; K and V through separate 2-stage rings; on a single graph
+//               also the 256x128-byte SPD tile (3-stage ring, 128-byte swizzle)
+//   warp 1      issues S_t = Q_t K^T (SS MMAs) for both query tiles, one key tile ahead
+//   warp 3      issues O_t += P_t V (A from TMEM, B = V as MN-major)
+//               (two issuing warps: a helper warp shares its scheduler with busy softmax warps
+//               and gets few issue slots, so the MMA issue is split to keep it off the critical path)
+//   warp 2      SPD loader for packed batches (per-graph pitch: cp.async with the same XOR swizzle)
+//   warps 4-7   softmax of tile 0 (thread = query row = TMEM lane), warps 8-11 of tile 1;
+//               the two groups take turns in the exponential phase
 //
 // TMEM columns: S0 [0,128) S1 [128,256) P0 [256,320) P1 [320,384) O0 [384,448) O1 [448,512).
 #include <cuda_bf16.h>
@@ -32,7 +36,8 @@ constexpr int kRowsPerTile = 128;
 constexpr int kQTiles = 2;
 constexpr int kRowsPerCta = kRowsPerTile * kQTiles;
 constexpr int kKvTile = 128;
-constexpr int kKvStages = 2;
+constexpr int kKStages = 2;
+constexpr int kVStages = 2;
 constexpr int kSpdStages = 3;
 constexpr int kFwdThreads = 384;
 constexpr float kRescaleThreshold = 8.0f;     // log2 units: keep a stale max while P stays below 2^8
@@ -51,14 +56,17 @@ struct FwdParams {
     int32_t n_heads;
     int32_t n_buckets;
     int32_t kv_chunk_rows;     // chunked: keys per chunk (multiple of 128)
+    int32_t spd_tma;           // 1: single graph, SPD tiles come by TMA; 0: cp.async loader warp
     float c1;                  // log2(e) / sqrt(d)
 };
 
 enum FwdBarrier {
     kBarQFull = 0,
-    kBarKvFull = 1,                          // [kKvStages]
-    kBarKvEmpty = kBarKvFull + kKvStages,    // [kKvStages]
-    kBarSpdFull = kBarKvEmpty + kKvStages,   // [kSpdStages]
+    kBarKFull = 1,                           // [kKStages]
+    kBarKEmpty = kBarKFull + kKStages,       // [kKStages]  commit after S_1 of the key tile
+    kBarVFull = kBarKEmpty + kKStages,       // [kVStages]
+    kBarVEmpty = kBarVFull + kVStages,       // [kVStages]  commit after PV_1 of the key tile
+    kBarSpdFull = kBarVEmpty + kVStages,     // [kSpdStages]
     kBarSpdEmpty = kBarSpdFull + kSpdStages, // [kSpdStages]
     kBarSFull = kBarSpdEmpty + kSpdStages,   // [2]
     kBarSFree = kBarSFull + 2,               // [2]
@@ -74,8 +82,8 @@ struct FwdSmem {
     static constexpr int kSpdTileBytes = kRowsPerCta * kKvTile;
     static constexpr int kQ = 0;
     static constexpr int kK = kQ + kQTiles * kTileBytes;
-    static constexpr int kV = kK + kKvStages * kTileBytes;
-    static constexpr int kSpd = kV + kKvStages * kTileBytes;
+    static constexpr int kV = kK + kKStages * kTileBytes;
+    static constexpr int kSpd = kV + kVStages * kTileBytes;
     static constexpr int kBias = kSpd + kSpdStages * kSpdTileBytes;
     static constexpr int kBars = kBias + 256 * 4;
     static constexpr int kMisc = kBars + kNumFwdBarriers * 8;
@@ -93,7 +101,8 @@ __device__ __forceinline__ float max3(float a, float b, float c)
 template <int D, bool kPartial, bool kShflBias>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                const __grid_constant__ CUtensorMap tmap_v, const FwdParams p)
+                const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_spd,
+                const FwdParams p)
 {
     using L = FwdSmem<D>;
     extern __shared__ uint8_t smem_raw[];
@@ -139,8 +148,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     if (tid == 0) {
         misc[1] = 0u;
         mbar_init(bar(kBarQFull), 1);
-        for (int s = 0; s < kKvStages; ++s) { mbar_init(bar(kBarKvFull + s), 1); mbar_init(bar(kBarKvEmpty + s), 1); }
-        for (int s = 0; s < kSpdStages; ++s) { mbar_init(bar(kBarSpdFull + s), 64); mbar_init(bar(kBarSpdEmpty + s), 8); }
+        for (int s = 0; s < kKStages; ++s) { mbar_init(bar(kBarKFull + s), 1); mbar_init(bar(kBarKEmpty + s), 1); }
+        for (int s = 0; s < kVStages; ++s) { mbar_init(bar(kBarVFull + s), 1); mbar_init(bar(kBarVEmpty + s), 1); }
+        for (int s = 0; s < kSpdStages; ++s) { mbar_init(bar(kBarSpdFull + s), p.spd_tma ? 1 : 32); mbar_init(bar(kBarSpdEmpty + s), 8); }
         for (int t = 0; t < 2; ++t) {
             mbar_init(bar(kBarSFull + t), 1);
             mbar_init(bar(kBarSFree + t), 128);
@@ -151,6 +161,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         prefetch_tensormap(&tmap_q);
         prefetch_tensormap(&tmap_k);
         prefetch_tensormap(&tmap_v);
+        if (p.spd_tma) prefetch_tensormap(&tmap_spd);
     }
     if (warp == 1) { tmem_alloc(smem_u32(&misc[0]), 512); tmem_relinquish(); }
     for (int i = tid; i < 256; i += kFwdThreads)
@@ -171,53 +182,70 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                                 node0 + q0 + t * kRowsPerTile);
             }
             for (int j = 0; j < n_kv; ++j) {
-                const int s = j % kKvStages;
-                mbar_wait(bar(kBarKvEmpty + s), ((j / kKvStages) & 1) ^ 1, abort_flag, p.status, 10);
+                const int32_t kv0 = kv_begin + j * kKvTile;
+                const int32_t row = node0 + kv0;
+                const int ks = j % kKStages, vs = j % kVStages, ss = j % kSpdStages;
+                mbar_wait(bar(kBarKEmpty + ks), ((j / kKStages) & 1) ^ 1, abort_flag, p.status, 10);
                 if (lane == 0) {
-                    const int32_t row = node0 + kv_begin + j * kKvTile;
-                    mbar_arrive_expect_tx(bar(kBarKvFull + s), 2 * L::kTileBytes);
-                    tma_load_3d(smem_u32(smem + L::kK + s * L::kTileBytes), &tmap_k, bar(kBarKvFull + s), 0, h, row);
-                    tma_load_3d(smem_u32(smem + L::kV + s * L::kTileBytes), &tmap_v, bar(kBarKvFull + s), 0, h, row);
+                    mbar_arrive_expect_tx(bar(kBarKFull + ks), L::kTileBytes);
+                    tma_load_3d(smem_u32(smem + L::kK + ks * L::kTileBytes), &tmap_k, bar(kBarKFull + ks), 0, h, row);
+                }
+                if (p.spd_tma) {
+                    mbar_wait(bar(kBarSpdEmpty + ss), ((j / kSpdStages) & 1) ^ 1, abort_flag, p.status, 11);
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(bar(kBarSpdFull + ss), L::kSpdTileBytes);
+                        tma_load_2d(smem_u32(smem + L::kSpd + ss * L::kSpdTileBytes), &tmap_spd, bar(kBarSpdFull + ss), kv0, q0);
+                    }
+                }
+                mbar_wait(bar(kBarVEmpty + vs), ((j / kVStages) & 1) ^ 1, abort_flag, p.status, 12);
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(bar(kBarVFull + vs), L::kTileBytes);
+                    tma_load_3d(smem_u32(smem + L::kV + vs * L::kTileBytes), &tmap_v, bar(kBarVFull + vs), 0, h, row);
                 }
                 __syncwarp();
             }
         } else if (warp == 1) {
-            // The warp stays converged around the waits; one elected lane issues each group of MMAs.
+            // ---- S issuer: S_t(j+1) as soon as group t holds S_t(j) in registers ----
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
-            constexpr uint32_t idesc_o = make_idesc_bf16(128, D, false, true);
             const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
             const uint64_t desc_q0 = make_smem_desc(smem_u32(smem + L::kQ), L::kRowBytes, 0);
             const uint64_t desc_k0 = make_smem_desc(smem_u32(smem + L::kK), L::kRowBytes, 0);
-            const uint64_t desc_v0 = make_smem_desc(smem_u32(smem + L::kV), L::kRowBytes, 0);
-            auto issue_s = [&](int t, int stage) {
+            auto issue_s = [&](int t, int stage, bool release_k) {
                 if (elect_one()) {
                     const uint64_t da = advance_desc(desc_q0, t * L::kTileBytes);
                     const uint64_t db = advance_desc(desc_k0, stage * L::kTileBytes);
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)
-                        mma_ss(tm + t * 128, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
+                    for (int k = 0; k < D / 16; ++k)
+                        mma_ss(tm + t * 128, advance_desc(da, k * 32), advance_desc(db, k * 32), idesc_s, k > 0);
                     mma_commit(bar(kBarSFull + t));
+                    if (release_k) mma_commit(bar(kBarKEmpty + stage));
                 }
                 __syncwarp();
             };
             mbar_wait(bar(kBarQFull), 0, abort_flag, p.status, 20);
-            mbar_wait(bar(kBarKvFull + 0), 0, abort_flag, p.status, 21);
+            mbar_wait(bar(kBarKFull + 0), 0, abort_flag, p.status, 21);
             tc_fence_after();
-            issue_s(0, 0);
-            issue_s(1, 0);
-            for (int j = 0; j < n_kv; ++j) {
-                const int s = j % kKvStages;
-                if (j + 1 < n_kv) {
-                    const int s1 = (j + 1) % kKvStages;
-                    mbar_wait(bar(kBarKvFull + s1), ((j + 1) / kKvStages) & 1, abort_flag, p.status, 22);
+            issue_s(0, 0, false);
+            issue_s(1, 0, true);
+            for (int j = 0; j + 1 < n_kv; ++j) {
+                const int s1 = (j + 1) % kKStages;
+                mbar_wait(bar(kBarKFull + s1), ((j + 1) / kKStages) & 1, abort_flag, p.status, 22);
 #pragma unroll
-                    for (int t = 0; t < 2; ++t) {
-                        mbar_wait(bar(kBarSFree + t), j & 1, abort_flag, p.status, 23);
-                        tc_fence_after();
-                        issue_s(t, s1);
-                    }
+                for (int t = 0; t < 2; ++t) {
+                    mbar_wait(bar(kBarSFree + t), j & 1, abort_flag, p.status, 23);
+                    tc_fence_after();
+                    issue_s(t, s1, t == 1);
                 }
-                const uint64_t dv = advance_desc(desc_v0, s * L::kTileBytes);
+            }
+        } else if (warp == 3) {
+            // ---- PV issuer ----
+            constexpr uint32_t idesc_o = make_idesc_bf16(128, D, false, true);
+            const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+            const uint64_t desc_v0 = make_smem_desc(smem_u32(smem + L::kV), L::kRowBytes, 0);
+            for (int j = 0; j < n_kv; ++j) {
+                const int vs = j % kVStages;
+                mbar_wait(bar(kBarVFull + vs), (j / kVStages) & 1, abort_flag, p.status, 25);
+                const uint64_t dv = advance_desc(desc_v0, vs * L::kTileBytes);
                 const uint32_t acc0 = j > 0 ? 1u : 0u;
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
@@ -225,18 +253,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     tc_fence_after();
                     if (elect_one()) {
 #pragma unroll
-                        for (int ks = 0; ks < kKvTile / 16; ++ks)
-                            mma_ts(tm + 384 + t * 64, tm + 256 + t * 64 + ks * 8,
-                                   advance_desc(dv, ks * 16 * L::kRowBytes), idesc_o, ks > 0 ? 1u : acc0);
+                        for (int k = 0; k < kKvTile / 16; ++k)
+                            mma_ts(tm + 384 + t * 64, tm + 256 + t * 64 + k * 8,
+                                   advance_desc(dv, k * 16 * L::kRowBytes), idesc_o, k > 0 ? 1u : acc0);
                         mma_commit(bar(kBarODone + t));
-                        if (t == 1) mma_commit(bar(kBarKvEmpty + s));
+                        if (t == 1) mma_commit(bar(kBarVEmpty + vs));
                     }
                     __syncwarp();
                 }
             }
-        } else {
-            // warps 2 and 3: SPD tile loader, 128 of the 256 rows each
-            const int half = warp - 2;
+        } else if (!p.spd_tma) {
+            // ---- warp 2: SPD tile loader for packed batches ----
             for (int j = 0; j < n_kv; ++j) {
                 const int s2 = j % kSpdStages;
                 mbar_wait(bar(kBarSpdEmpty + s2), ((j / kSpdStages) & 1) ^ 1, abort_flag, p.status, 30);
@@ -246,8 +273,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 const int64_t col = (int64_t)kv0 + cc * 16;
                 const bool col_ok = col < ld;
 #pragma unroll 4
-                for (int i = 0; i < 32; ++i) {
-                    const int r = half * 128 + i * 4 + (lane >> 3);
+                for (int i = 0; i < 64; ++i) {
+                    const int r = i * 4 + (lane >> 3);
                     const bool valid = col_ok && (q0 + r < n_g);
                     const uint8_t* src = valid ? spd_g + (int64_t)(q0 + r) * ld + col : spd_g;
                     cp_async_16(dst0 + r * 128 + ((cc ^ (r & 7)) << 4), src, valid ? 16u : 0u);
@@ -530,13 +557,13 @@ int32_t chunk_rows(int32_t n, int32_t n_chunks)
 }
 
 template <int D, bool kPartial>
-gt_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& p,
-                     const gt_batch* batch, int grid_z, cudaStream_t s)
+gt_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tspd,
+                     const FwdParams& p, const gt_batch* batch, int grid_z, cudaStream_t s)
 {
     auto kern = p.n_buckets <= 32 ? attn_fwd_kernel<D, kPartial, true> : attn_fwd_kernel<D, kPartial, false>;
     GT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kDynamic));
     dim3 grid((unsigned)p.n_heads, (unsigned)((batch->max_seqlen + kRowsPerCta - 1) / kRowsPerCta), (unsigned)grid_z);
-    kern<<<grid, kFwdThreads, FwdSmem<D>::kDynamic, s>>>(tq, tk, tv, p);
+    kern<<<grid, kFwdThreads, FwdSmem<D>::kDynamic, s>>>(tq, tk, tv, tspd, p);
     GT_CUDA_TRY(cudaGetLastError());
     return GT_OK;
 }
@@ -577,7 +604,10 @@ extern "C" gt_status gt_biased_attn_fwd(const void* q, const void* k, const void
     if ((st = encode_thd_map(&tq, q, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
     if ((st = encode_thd_map(&tk, k, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
     if ((st = encode_thd_map(&tv, v, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
+    CUtensorMap tspd = tq;                       // placeholder when the cp.async loader is used
     FwdParams p{};
+    p.spd_tma = batch->n_graphs == 1 ? 1 : 0;
+    if (p.spd_tma && (st = encode_spd_map(&tspd, spd, batch->n_total, 256)) != GT_OK) return st;
     p.spd = spd;
     p.spd_offsets = batch->n_graphs > 1 ? spd_offsets : nullptr;
     p.cu_seqlens = batch->n_graphs > 1 ? batch->cu_seqlens : nullptr;
@@ -590,8 +620,8 @@ extern "C" gt_status gt_biased_attn_fwd(const void* q, const void* k, const void
     p.n_buckets = max_dist + 2;
     p.c1 = kLog2e / sqrtf((float)head_dim);
     cudaStream_t s = (cudaStream_t)stream;
-    return head_dim == 64 ? launch_fwd<64, false>(tq, tk, tv, p, batch, batch->n_graphs, s)
-                          : launch_fwd<32, false>(tq, tk, tv, p, batch, batch->n_graphs, s);
+    return head_dim == 64 ? launch_fwd<64, false>(tq, tk, tv, tspd, p, batch, batch->n_graphs, s)
+                          : launch_fwd<32, false>(tq, tk, tv, tspd, p, batch, batch->n_graphs, s);
 }
 
 extern "C" size_t gt_biased_attn_fwd_chunked_workspace(const gt_batch* batch, int32_t n_heads, int32_t head_dim,
@@ -623,7 +653,10 @@ extern "C" gt_status gt_biased_attn_fwd_chunked(const void* q, const void* k, co
     if ((st = encode_thd_map(&tv, v, batch->n_total, n_heads, head_dim)) != GT_OK) return st;
     const size_t rows = (size_t)batch->n_total * n_heads;
     uint8_t* ws = (uint8_t*)workspace;
+    CUtensorMap tspd;
+    if ((st = encode_spd_map(&tspd, spd, batch->n_total, 256)) != GT_OK) return st;
     FwdParams p{};
+    p.spd_tma = 1;
     p.spd = spd;
     p.bias = bias;
     p.part_lse = (float*)(ws + kHeaderBytes);
@@ -635,8 +668,8 @@ extern "C" gt_status gt_biased_attn_fwd_chunked(const void* q, const void* k, co
     p.kv_chunk_rows = chunk_rows(batch->n_total, n_kv_chunks);
     p.c1 = kLog2e / sqrtf((float)head_dim);
     cudaStream_t s = (cudaStream_t)stream;
-    st = head_dim == 64 ? launch_fwd<64, true>(tq, tk, tv, p, batch, n_kv_chunks, s)
-                        : launch_fwd<32, true>(tq, tk, tv, p, batch, n_kv_chunks, s);
+    st = head_dim == 64 ? launch_fwd<64, true>(tq, tk, tv, tspd, p, batch, n_kv_chunks, s)
+                        : launch_fwd<32, true>(tq, tk, tv, tspd, p, batch, n_kv_chunks, s);
     if (st != GT_OK) return st;
     const size_t n_thr = rows * (head_dim / 4);
     const unsigned blocks = (unsigned)((n_thr + 255) / 256);
