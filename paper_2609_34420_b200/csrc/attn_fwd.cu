@@ -5,21 +5,32 @@
 // are updated (the rule the paper states for its context-parallel online softmax), P goes
 // back to tensor memory as the A operand of the P V MMA.
 //
-// One CTA = one head x 256 query rows (two 128-row tiles, one softmax warpgroup each, so the
-// tensor pipe works on one tile while the other is in its softmax) x all key tiles of the
-// graph (or of one key chunk for the chunked entry point).
+// One CTA = one head x 256 query rows (two 128-row tiles, so the tensor pipe works on one tile
+// while the other is in its softmax) x all key tiles of the graph (or of one key chunk for the
+// chunked entry point).
 //
 //   warp 0      TMA producer: Q once; K and V through separate 2-stage rings; on a single graph
 //               also the 256x128-byte SPD tile (3-stage ring, 128-byte swizzle)
-//   warp 1      issues S_t = Q_t K^T (SS MMAs) for both query tiles, one key tile ahead
+//   warp 1      issues S_t = Q_t K^T (SS MMAs) for both query tiles
 //   warp 3      issues O_t += P_t V (A from TMEM, B = V as MN-major)
 //               (two issuing warps: a helper warp shares its scheduler with busy softmax warps
 //               and gets few issue slots, so the MMA issue is split to keep it off the critical path)
 //   warp 2      SPD loader for packed batches (per-graph pitch: cp.async with the same XOR swizzle)
-//   warps 4-7   softmax of tile 0 (thread = query row = TMEM lane), warps 8-11 of tile 1;
-//               the two groups take turns in the exponential phase
+//   warps 4-19  softmax: 8 warps per query tile, 4 per half of the 128 key columns (thread = query
+//               row = TMEM lane, 64 score elements per thread).
 //
-// TMEM columns: S0 [0,128) S1 [128,256) P0 [256,320) P1 [320,384) O0 [384,448) O1 [448,512).
+// Softmax is single pass and speculative: a key tile is exponentiated against the row's current
+// reference maximum without looking at the tile's own maximum first; the row sum of the tile tells
+// afterwards whether the reference was too low (sum above a threshold, or not finite), and only then
+// the tile is redone the classical way (maximum, rescale of l and O, exponentials).  The first key
+// tile always takes the classical way.  References only ever grow, and they are integers in log2
+// units, so rescale factors are exact powers of two and the bf16 mantissa of a P entry does not
+// depend on how the keys are tiled or chunked.
+//
+// TMEM columns: three score buffers [0,128) [128,256) [256,384) used in rotation by the steps
+// (key tile j, query tile t) -> buffer (2j+t) mod 3, so that the S MMA of a step never waits for a
+// softmax; P overwrites the part of the score buffer its own thread has read (bf16, half the
+// columns); O_0 [384,448), O_1 [448,512).
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -39,8 +50,14 @@ constexpr int kKvTile = 128;
 constexpr int kKStages = 2;
 constexpr int kVStages = 2;
 constexpr int kSpdStages = 3;
-constexpr int kFwdThreads = 384;
-constexpr float kRescaleThreshold = 8.0f;     // log2 units: keep a stale max while P stays below 2^8
+constexpr int kHalves = 2;                    // softmax threads per query row (column halves)
+constexpr int kSoftmaxWarps = 8 * kHalves;
+constexpr int kFwdThreads = 128 + 32 * kSoftmaxWarps;
+constexpr int kCols = kKvTile / kHalves;      // score columns per softmax thread
+constexpr int kCW = kHalves == 1 ? 32 : 16;   // columns per TMEM load
+constexpr int kChunks = kCols / kCW;
+static_assert(kChunks == 4, "the softmax pass is written for four chunks");
+constexpr float kSumThreshold = 1024.0f;      // tile row sum above which the reference maximum is raised
 
 struct FwdParams {
     const uint8_t* spd;
@@ -68,11 +85,11 @@ enum FwdBarrier {
     kBarVEmpty = kBarVFull + kVStages,       // [kVStages]  commit after PV_1 of the key tile
     kBarSpdFull = kBarVEmpty + kVStages,     // [kSpdStages]
     kBarSpdEmpty = kBarSpdFull + kSpdStages, // [kSpdStages]
-    kBarSFull = kBarSpdEmpty + kSpdStages,   // [2]
-    kBarSFree = kBarSFull + 2,               // [2]
-    kBarPFull = kBarSFree + 2,               // [2]
-    kBarODone = kBarPFull + 2,               // [2]
-    kNumFwdBarriers = kBarODone + 2
+    kBarSFull = kBarSpdEmpty + kSpdStages,   // [3]  per score buffer
+    kBarBufFree = kBarSFull + 3,             // [3]  P of the buffer consumed by its PV MMA
+    kBarPFull = kBarBufFree + 3,             // [2 tiles][2 key-tile parities]
+    kBarODone = kBarPFull + 4,               // [2 tiles][2 key-tile parities]
+    kNumFwdBarriers = kBarODone + 4
 };
 
 template <int D>
@@ -85,17 +102,26 @@ struct FwdSmem {
     static constexpr int kV = kK + kKStages * kTileBytes;
     static constexpr int kSpd = kV + kVStages * kTileBytes;
     static constexpr int kBias = kSpd + kSpdStages * kSpdTileBytes;
-    static constexpr int kBars = kBias + 256 * 4;
+    static constexpr int kXchg = kBias + 256 * 4;             // [2 tiles][max | sum][2 halves][128 rows] float
+    static constexpr int kBars = kXchg + 2 * 512 * 4;
     static constexpr int kMisc = kBars + kNumFwdBarriers * 8;
     static constexpr int kTotal = kMisc + 16;
     static constexpr int kDynamic = kTotal + 1024;   // slack for the 1024-byte alignment
 };
 
-__device__ __forceinline__ float max3(float a, float b, float c)
+enum FwdNamedBarrier { kNbPair = 2 /* + 4 t + lane quarter: the two warps that share 32 query rows */ };
+
+template <bool B> struct BoolTag { static constexpr bool value = B; };
+
+template <int N>
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, uint32_t (&r)[N])
 {
-    float r;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
-    return r;
+    if constexpr (N == 32) tmem_ld32(taddr, r); else tmem_ld16(taddr, r);
+}
+template <int N>
+__device__ __forceinline__ void tmem_st(uint32_t taddr, const uint32_t (&r)[N])
+{
+    if constexpr (N == 32) tmem_st32(taddr, r); else tmem_st16(taddr, r);
 }
 
 template <int D, bool kPartial, bool kShflBias>
@@ -150,13 +176,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         mbar_init(bar(kBarQFull), 1);
         for (int s = 0; s < kKStages; ++s) { mbar_init(bar(kBarKFull + s), 1); mbar_init(bar(kBarKEmpty + s), 1); }
         for (int s = 0; s < kVStages; ++s) { mbar_init(bar(kBarVFull + s), 1); mbar_init(bar(kBarVEmpty + s), 1); }
-        for (int s = 0; s < kSpdStages; ++s) { mbar_init(bar(kBarSpdFull + s), p.spd_tma ? 1 : 32); mbar_init(bar(kBarSpdEmpty + s), 8); }
-        for (int t = 0; t < 2; ++t) {
-            mbar_init(bar(kBarSFull + t), 1);
-            mbar_init(bar(kBarSFree + t), 128);
-            mbar_init(bar(kBarPFull + t), 128);
-            mbar_init(bar(kBarODone + t), 1);
-        }
+        for (int s = 0; s < kSpdStages; ++s) { mbar_init(bar(kBarSpdFull + s), p.spd_tma ? 1 : 32); mbar_init(bar(kBarSpdEmpty + s), kSoftmaxWarps); }
+        for (int b = 0; b < 3; ++b) { mbar_init(bar(kBarSFull + b), 1); mbar_init(bar(kBarBufFree + b), 1); }
+        for (int t = 0; t < 4; ++t) mbar_init(bar(kBarPFull + t), 128 * kHalves);
+        for (int t = 0; t < 4; ++t) mbar_init(bar(kBarODone + t), 1);
         fence_mbar_init();
         prefetch_tensormap(&tmap_q);
         prefetch_tensormap(&tmap_k);
@@ -173,7 +196,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 
     if (warp < 4) {
         // =========================== producer / MMA / SPD warps ===========================
-        setmaxnreg_dec_56();
+        if constexpr (kHalves == 2) setmaxnreg_dec_32(); else setmaxnreg_dec_56();
         if (warp == 0) {
             if (lane == 0) {
                 mbar_arrive_expect_tx(bar(kBarQFull), kQTiles * L::kTileBytes);
@@ -205,36 +228,31 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 __syncwarp();
             }
         } else if (warp == 1) {
-            // ---- S issuer: S_t(j+1) as soon as group t holds S_t(j) in registers ----
+            // ---- S issuer: step (j, t) goes to score buffer (2j+t) mod 3 once the PV MMA of the
+            // step that used the buffer before has drained it ----
             constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
             const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
             const uint64_t desc_q0 = make_smem_desc(smem_u32(smem + L::kQ), L::kRowBytes, 0);
             const uint64_t desc_k0 = make_smem_desc(smem_u32(smem + L::kK), L::kRowBytes, 0);
-            auto issue_s = [&](int t, int stage, bool release_k) {
-                if (elect_one()) {
-                    const uint64_t da = advance_desc(desc_q0, t * L::kTileBytes);
-                    const uint64_t db = advance_desc(desc_k0, stage * L::kTileBytes);
-#pragma unroll
-                    for (int k = 0; k < D / 16; ++k)
-                        mma_ss(tm + t * 128, advance_desc(da, k * 32), advance_desc(db, k * 32), idesc_s, k > 0);
-                    mma_commit(bar(kBarSFull + t));
-                    if (release_k) mma_commit(bar(kBarKEmpty + stage));
-                }
-                __syncwarp();
-            };
             mbar_wait(bar(kBarQFull), 0, abort_flag, p.status, 20);
-            mbar_wait(bar(kBarKFull + 0), 0, abort_flag, p.status, 21);
-            tc_fence_after();
-            issue_s(0, 0, false);
-            issue_s(1, 0, true);
-            for (int j = 0; j + 1 < n_kv; ++j) {
-                const int s1 = (j + 1) % kKStages;
-                mbar_wait(bar(kBarKFull + s1), ((j + 1) / kKStages) & 1, abort_flag, p.status, 22);
+            for (int j = 0; j < n_kv; ++j) {
+                const int ks = j % kKStages;
+                mbar_wait(bar(kBarKFull + ks), (j / kKStages) & 1, abort_flag, p.status, 22);
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
-                    mbar_wait(bar(kBarSFree + t), j & 1, abort_flag, p.status, 23);
+                    const int step = 2 * j + t, b = step % 3;
+                    if (step >= 3) mbar_wait(bar(kBarBufFree + b), (step / 3 - 1) & 1, abort_flag, p.status, 23);
                     tc_fence_after();
-                    issue_s(t, s1, t == 1);
+                    if (elect_one()) {
+                        const uint64_t da = advance_desc(desc_q0, t * L::kTileBytes);
+                        const uint64_t db = advance_desc(desc_k0, ks * L::kTileBytes);
+#pragma unroll
+                        for (int k = 0; k < D / 16; ++k)
+                            mma_ss(tm + b * 128, advance_desc(da, k * 32), advance_desc(db, k * 32), idesc_s, k > 0);
+                        mma_commit(bar(kBarSFull + b));
+                        if (t == 1) mma_commit(bar(kBarKEmpty + ks));
+                    }
+                    __syncwarp();
                 }
             }
         } else if (warp == 3) {
@@ -249,14 +267,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 const uint32_t acc0 = j > 0 ? 1u : 0u;
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
-                    mbar_wait(bar(kBarPFull + t), j & 1, abort_flag, p.status, 24);
+                    const int b = (2 * j + t) % 3;
+                    mbar_wait(bar(kBarPFull + 2 * t + (j & 1)), (j >> 1) & 1, abort_flag, p.status, 24);
                     tc_fence_after();
                     if (elect_one()) {
 #pragma unroll
-                        for (int k = 0; k < kKvTile / 16; ++k)
-                            mma_ts(tm + 384 + t * 64, tm + 256 + t * 64 + k * 8,
+                        for (int k = 0; k < kKvTile / 16; ++k)      // P of key half hf sits at the start of that half's score columns
+                            mma_ts(tm + 384 + t * 64, tm + b * 128 + (k / (kCols / 16)) * kCols + (k % (kCols / 16)) * 8,
                                    advance_desc(dv, k * 16 * L::kRowBytes), idesc_o, k > 0 ? 1u : acc0);
-                        mma_commit(bar(kBarODone + t));
+                        mma_commit(bar(kBarODone + 2 * t + (j & 1)));
+                        mma_commit(bar(kBarBufFree + b));
                         if (t == 1) mma_commit(bar(kBarVEmpty + vs));
                     }
                     __syncwarp();
@@ -283,215 +303,222 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             }
         }
     } else {
-        // ================================= softmax warpgroups =================================
-        setmaxnreg_inc_224();
-        const int t = (warp >> 2) - 1;
-        const int r = tid & 127;
+        // =================================== softmax warps ===================================
+        if constexpr (kHalves == 2) setmaxnreg_inc_112(); else setmaxnreg_inc_224();
+        const int sw = warp - 4;
+        const int t = sw / (4 * kHalves);
+        const int hf = (sw >> 2) & (kHalves - 1);
+        const int r = ((warp & 3) << 5) | lane;
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + t * 128 + lane_off;
-        const uint32_t tP = tmem + 256 + t * 64 + lane_off;
-        const uint32_t tO = tmem + 384 + t * 64 + lane_off;
-        const float c1 = p.c1;
+        constexpr int kOC = D / kHalves;                 // output columns per thread
+        constexpr int kOP = kOC < 32 ? kOC : 32;         // ... per TMEM access
+        const uint32_t tO = tmem + 384 + t * 64 + hf * kOC + lane_off;
+        const uint32_t pair_bar = kNbPair + t * 4 + (warp & 3);
+        float* xchg = (float*)(smem + L::kXchg) + t * 512;
         float m = -INFINITY, l = 0.f;
 
         // lane b of every softmax warp keeps table entry b (scaled by log2 e); entries past the
         // table repeat the last one.  With at most 32 buckets a score's bias is fetched by a
         // warp shuffle whose source lane is the raw SPD byte (only its low 5 bits select).
         const float tbl = s_bias[lane];
-        const uint64_t c1c1 = pack_f32x2(c1, c1);
+        const uint64_t c1c1 = pack_f32x2(p.c1, p.c1);
 
-        // The two softmax warpgroups take turns in the exponential phase (it saturates the
-        // special-function unit; the other group meanwhile runs its lookup / max phase on the
-        // other pipes).  Barrier 2+t lets group t in; the other group arrives on it when it leaves.
-        if (t == 1) named_barrier_arrive(2, 256);
-
-        // Software-pipelined over key tiles: the first 64 score columns and the SPD row of tile
-        // j+1 are fetched at the end of tile j, so their latency hides behind the P store.
-        uint32_t sa[32], sb[32];                // score chunks of 32 columns, alternating
-        uint4 wa[2], wb[2];                     // SPD bytes of those chunks (2 x 16 bytes each)
-        auto spd_row = [&](int j) {
-            return smem + L::kSpd + (j % kSpdStages) * L::kSpdTileBytes + (t * 128 + r) * 128;
+        uint32_t sa[kCW], sb[kCW];              // score chunks, alternating
+        uint4 wa[kCW / 16], wb[kCW / 16];       // their SPD bytes
+        uint32_t tS = 0;                        // this thread's score columns of the current step
+        const uint8_t* srow = nullptr;          // this thread's row of the current SPD tile
+        auto load_chunk = [&](int c, uint32_t (&sr)[kCW], uint4 (&ws)[kCW / 16]) {
+            tmem_ld<kCW>(tS + c * kCW, sr);
+#pragma unroll
+            for (int i = 0; i < kCW / 16; ++i)
+                ws[i] = *(const uint4*)(srow + (((hf * (kCols / 16) + c * (kCW / 16) + i) ^ (r & 7)) << 4));
         };
-        auto prefetch = [&](int j) {
-            mbar_wait(bar(kBarSFull + t), j & 1, abort_flag, p.status, 40);
+        // bias of 8 consecutive columns (two SPD words)
+        auto lookup8 = [&](uint32_t w0, uint32_t w1, float (&bb)[8]) {
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const uint32_t word = k == 0 ? w0 : w1;
+                if (kShflBias) {
+                    bb[4 * k + 0] = __shfl_sync(0xffffffffu, tbl, word);
+                    bb[4 * k + 1] = __shfl_sync(0xffffffffu, tbl, word >> 8);
+                    bb[4 * k + 2] = __shfl_sync(0xffffffffu, tbl, word >> 16);
+                    bb[4 * k + 3] = __shfl_sync(0xffffffffu, tbl, word >> 24);
+                } else {
+                    bb[4 * k + 0] = s_bias[word & 0xffu];
+                    bb[4 * k + 1] = s_bias[(word >> 8) & 0xffu];
+                    bb[4 * k + 2] = s_bias[(word >> 16) & 0xffu];
+                    bb[4 * k + 3] = s_bias[word >> 24];
+                }
+            }
+        };
+        // first chunk of key tile j: fetched at the end of tile j-1, behind the P store
+        auto begin_tile = [&](int j) {
+            const int step = 2 * j + t, b = step % 3;
+            tS = tmem + b * 128 + hf * kCols + lane_off;
+            mbar_wait(bar(kBarSFull + b), (step / 3) & 1, abort_flag, p.status, 40);
             tc_fence_after();
-            tmem_ld32(tS, sa);
             mbar_wait(bar(kBarSpdFull + (j % kSpdStages)), (j / kSpdStages) & 1, abort_flag, p.status, 41);
-            const uint8_t* srow = spd_row(j);
-            wa[0] = *(const uint4*)(srow + ((0 ^ (r & 7)) << 4));
-            wa[1] = *(const uint4*)(srow + ((1 ^ (r & 7)) << 4));
+            srow = smem + L::kSpd + (j % kSpdStages) * L::kSpdTileBytes + (t * 128 + r) * 128;
+            load_chunk(0, sa, wa);
         };
-        prefetch(0);
+        begin_tile(0);
 
         for (int j = 0; j < n_kv; ++j) {
-            uint64_t xp[64];                       // 128 scores of this row as f32x2 pairs
-            // one chunk = 32 columns: two rounds of (16 bias lookups, then 8 packed FMAs  x = s c1 + bias)
-            auto chunk = [&](int c, const uint32_t (&sr)[32], const uint4 (&ws)[2]) {
+            const int32_t kv0 = kv_begin + j * kKvTile;
+            const bool ragged = kv0 + kKvTile > kv_end;          // last key tile of the range
+            const int valid = kv_end - kv0 - hf * kCols;         // valid columns of this thread (may be <= 0)
+            uint32_t pk[kCols / 64][32];           // P of this thread's columns, bf16 pairs
+            float tile_sum = 0.f;
+            bool loaded = true;                    // chunk 0 is already on its way
+            bool exact = (j == 0);                 // take the tile maximum first
+
+            for (;;) {
+                if (exact) {
+                    // ---- classical way: tile maximum, new reference, rescale of l and O ----
+                    float mx0 = -INFINITY, mx1 = -INFINITY;
+                    auto max_chunk = [&](int c, const uint32_t (&sr)[kCW], const uint4 (&ws)[kCW / 16]) {
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    float bb[16];
-                    const uint32_t words[4] = {ws[hh].x, ws[hh].y, ws[hh].z, ws[hh].w};
+                        for (int q = 0; q < kCW / 8; ++q) {
+                            const uint4& ww = ws[q >> 1];
+                            float bb[8];
+                            lookup8((q & 1) ? ww.z : ww.x, (q & 1) ? ww.w : ww.y, bb);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        if (kShflBias) {
-                            bb[4 * k + 0] = __shfl_sync(0xffffffffu, tbl, words[k]);
-                            bb[4 * k + 1] = __shfl_sync(0xffffffffu, tbl, words[k] >> 8);
-                            bb[4 * k + 2] = __shfl_sync(0xffffffffu, tbl, words[k] >> 16);
-                            bb[4 * k + 3] = __shfl_sync(0xffffffffu, tbl, words[k] >> 24);
-                        } else {
-                            bb[4 * k + 0] = s_bias[words[k] & 0xffu];
-                            bb[4 * k + 1] = s_bias[(words[k] >> 8) & 0xffu];
-                            bb[4 * k + 2] = s_bias[(words[k] >> 16) & 0xffu];
-                            bb[4 * k + 3] = s_bias[words[k] >> 24];
+                            for (int i = 0; i < 4; ++i) {
+                                float lo, hi;
+                                unpack_f32x2(fma_f32x2(pack_u32x2(sr[q * 8 + 2 * i], sr[q * 8 + 2 * i + 1]), c1c1,
+                                                       pack_f32x2(bb[2 * i], bb[2 * i + 1])), lo, hi);
+                                const int col = c * kCW + q * 8 + 2 * i;
+                                if (ragged && col >= valid) lo = -INFINITY;
+                                if (ragged && col + 1 >= valid) hi = -INFINITY;
+                                mx0 = fmaxf(mx0, lo);
+                                mx1 = fmaxf(mx1, hi);
+                            }
+                        }
+                    };
+                    if (!loaded) load_chunk(0, sa, wa);
+                    tmem_wait_ld(); load_chunk(1, sb, wb); max_chunk(0, sa, wa);
+                    tmem_wait_ld(); load_chunk(2, sa, wa); max_chunk(1, sb, wb);
+                    tmem_wait_ld(); load_chunk(3, sb, wb); max_chunk(2, sa, wa);
+                    tmem_wait_ld(); max_chunk(3, sb, wb);
+                    loaded = false;
+                    float mt = fmaxf(mx0, mx1);
+                    if constexpr (kHalves == 2) {
+                        xchg[hf * 128 + r] = mt;
+                        named_barrier_sync(pair_bar, 64);
+                        mt = fmaxf(mt, xchg[(hf ^ 1) * 128 + r]);
+                    }
+                    const float m_new = fmaxf(m, ceilf(mt));
+                    const float alpha = ex2_approx(m - m_new);
+                    l *= alpha;
+                    if (j > 0) {
+                        mbar_wait(bar(kBarODone + 2 * t + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag, p.status, 42);
+                        tc_fence_after();
+#pragma unroll
+                        for (int c = 0; c < kOC / kOP; ++c) {
+                            uint32_t o[kOP];
+                            tmem_ld<kOP>(tO + c * kOP, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < kOP; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                            tmem_st<kOP>(tO + c * kOP, o);
                         }
                     }
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        xp[c * 16 + hh * 8 + i] = fma_f32x2(pack_u32x2(sr[hh * 16 + 2 * i], sr[hh * 16 + 2 * i + 1]), c1c1,
-                                                            pack_f32x2(bb[2 * i], bb[2 * i + 1]));
+                    m = m_new;
                 }
-            };
-            const uint8_t* srow = spd_row(j);
-            auto lds_words = [&](int c, uint4 (&ws)[2]) {
-                ws[0] = *(const uint4*)(srow + (((2 * c) ^ (r & 7)) << 4));
-                ws[1] = *(const uint4*)(srow + (((2 * c + 1) ^ (r & 7)) << 4));
-            };
-            tmem_wait_ld();                        // chunk 0 (prefetched at the end of the previous tile)
-            tmem_ld32(tS + 32, sb);
-            lds_words(1, wb);
-            chunk(0, sa, wa);
-            tmem_wait_ld();
-            tmem_ld32(tS + 64, sa);
-            lds_words(2, wa);
-            chunk(1, sb, wb);
-            tmem_wait_ld();
-            tmem_ld32(tS + 96, sb);
-            lds_words(3, wb);
+
+                // ---- P = 2^(s c1 + bias - m), row sum ----
+                const uint64_t neg_m = pack_f32x2(-m, -m);
+                uint64_t sum2 = pack_f32x2(0.f, 0.f);
+                auto exp_chunk = [&](int c, const uint32_t (&sr)[kCW], const uint4 (&ws)[kCW / 16], auto rag) {
+#pragma unroll
+                    for (int q = 0; q < kCW / 8; ++q) {
+                        const uint4& ww = ws[q >> 1];
+                        float bb[8];
+                        lookup8((q & 1) ? ww.z : ww.x, (q & 1) ? ww.w : ww.y, bb);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            float lo, hi;
+                            unpack_f32x2(add_f32x2(fma_f32x2(pack_u32x2(sr[q * 8 + 2 * i], sr[q * 8 + 2 * i + 1]), c1c1,
+                                                             pack_f32x2(bb[2 * i], bb[2 * i + 1])), neg_m), lo, hi);
+                            if constexpr (decltype(rag)::value) {
+                                const int col = c * kCW + q * 8 + 2 * i;
+                                if (col >= valid) lo = -INFINITY;
+                                if (col + 1 >= valid) hi = -INFINITY;
+                            }
+                            lo = ex2_approx(lo);
+                            hi = ex2_approx(hi);
+                            sum2 = add_f32x2(sum2, pack_f32x2(lo, hi));
+                            pk[(c * (kCW / 2) + q * 4 + i) >> 5][(c * (kCW / 2) + q * 4 + i) & 31] = pack_bf16x2(lo, hi);
+                        }
+                    }
+                };
+                auto exp_pass = [&](auto rag) {
+                    if (!loaded) load_chunk(0, sa, wa);
+                    tmem_wait_ld(); load_chunk(1, sb, wb); exp_chunk(0, sa, wa, rag);
+                    tmem_wait_ld(); load_chunk(2, sa, wa); exp_chunk(1, sb, wb, rag);
+                    tmem_wait_ld(); load_chunk(3, sb, wb); exp_chunk(2, sa, wa, rag);
+                    tmem_wait_ld(); exp_chunk(3, sb, wb, rag);
+                };
+                if (ragged) exp_pass(BoolTag<true>{}); else exp_pass(BoolTag<false>{});
+                loaded = false;
+                {
+                    float lo, hi;
+                    unpack_f32x2(sum2, lo, hi);
+                    tile_sum = lo + hi;
+                }
+                if (exact) break;
+                // reference too low for some row of this warp (pair of warps)?  Also catches inf / NaN.
+                const bool need = !(tile_sum <= kSumThreshold);
+                bool any_need;
+                if constexpr (kHalves == 2) any_need = named_barrier_or(pair_bar, 64, need);
+                else any_need = __any_sync(0xffffffffu, need);
+                if (!any_need) break;
+                exact = true;
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(kBarSpdEmpty + (j % kSpdStages)));
-            chunk(2, sa, wa);
-            tmem_wait_ld();
-            tc_fence_before();
-            mbar_arrive(bar(kBarSFree + t));
-            chunk(3, sb, wb);
+            l += tile_sum;
 
-            const int32_t kv0 = kv_begin + j * kKvTile;
-            if (kv0 + kKvTile > kv_end) {           // ragged last key tile
-                const int valid = kv_end - kv0;
+            // P over the first half of this thread's own score columns
 #pragma unroll
-                for (int i = 0; i < 64; ++i) {
-                    float lo, hi;
-                    unpack_f32x2(xp[i], lo, hi);
-                    if (2 * i >= valid) lo = -INFINITY;
-                    if (2 * i + 1 >= valid) hi = -INFINITY;
-                    xp[i] = pack_f32x2(lo, hi);
-                }
-            }
-            float mt0, mt1;
-            unpack_f32x2(xp[0], mt0, mt1);
-#pragma unroll
-            for (int i = 1; i < 64; i += 2) {
-                float a, b, c, d2;
-                unpack_f32x2(xp[i], a, b);
-                if (i + 1 < 64) {
-                    unpack_f32x2(xp[i + 1], c, d2);
-                    mt0 = max3(mt0, a, c);
-                    mt1 = max3(mt1, b, d2);
-                } else {
-                    mt0 = fmaxf(mt0, a);
-                    mt1 = fmaxf(mt1, b);
-                }
-            }
-            const float mt = fmaxf(mt0, mt1);
-            // The reference maximum is kept at an integer (log2 units): rescale factors are then
-            // exact powers of two and the bf16 mantissa of every P entry does not depend on how
-            // the keys are tiled or chunked, which keeps chunked and unchunked results within
-            // fp32 rounding of each other.
-            const float m_new = fmaxf(m, ceilf(mt));
-            const bool need = (m_new - m) > kRescaleThreshold;
-
-            if (j > 0) {
-                mbar_wait(bar(kBarODone + t), (j - 1) & 1, abort_flag, p.status, 42);
-                tc_fence_after();
-            }
-            if (__any_sync(0xffffffffu, need)) {
-                const float alpha = ex2_approx(m - m_new);
-                l *= alpha;
-                if (j > 0) {
-#pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t o[32];
-                        tmem_ld32(tO + c * 32, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                        tmem_st32(tO + c * 32, o);
-                    }
-                }
-                m = m_new;
-            }
-
-            // ---- exponential phase: the MUFU results are consumed kExpLag pairs after they are
-            // issued so that the in-order pipeline never waits on a result it has just asked for.
-            named_barrier_sync(2 + t, 256);
-            const uint64_t neg_m = pack_f32x2(-m, -m);
-#pragma unroll
-            for (int i = 0; i < 64; ++i) xp[i] = add_f32x2(xp[i], neg_m);
-            uint64_t sum2 = pack_f32x2(0.f, 0.f);
-            uint32_t pk0[32], pk1[32];
-            constexpr int kExpLag = 6;
-#pragma unroll
-            for (int i = 0; i < 64 + kExpLag; ++i) {
-                if (i < 64) {
-                    float lo, hi;
-                    unpack_f32x2(xp[i], lo, hi);
-                    xp[i] = pack_f32x2(ex2_approx(lo), ex2_approx(hi));
-                }
-                if (i >= kExpLag) {
-                    const int k = i - kExpLag;
-                    float lo, hi;
-                    unpack_f32x2(xp[k], lo, hi);
-                    sum2 = add_f32x2(sum2, xp[k]);
-                    if (k < 32) pk0[k] = pack_bf16x2(lo, hi);
-                    else pk1[k - 32] = pack_bf16x2(lo, hi);
-                }
-            }
-            named_barrier_arrive(2 + (t ^ 1), 256);
-            {
-                float lo, hi;
-                unpack_f32x2(sum2, lo, hi);
-                l += lo + hi;
-            }
-            tmem_st32(tP, pk0);
-            tmem_st32(tP + 32, pk1);
-            if (j + 1 < n_kv) prefetch(j + 1);
+            for (int c = 0; c < kCols / 64; ++c) tmem_st32(tS + c * 32, pk[c]);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bar(kBarPFull + t));
+            // Warps of a tile can be one step apart (nothing in the speculative pass waits for the
+            // previous PV MMA), so odd and even key tiles use different barriers, here and for the
+            // completion of the PV MMAs: a parity wait can only tell two states apart.  Two steps
+            // apart is impossible because S(j+2) needs a score buffer that is only freed after PV(j).
+            mbar_arrive(bar(kBarPFull + 2 * t + (j & 1)));
+            if (j + 1 < n_kv) begin_tile(j + 1);
         }
 
         // ---- epilogue: O / l, LSE ----
-        mbar_wait(bar(kBarODone + t), (n_kv - 1) & 1, abort_flag, p.status, 43);
+        mbar_wait(bar(kBarODone + 2 * t + ((n_kv - 1) & 1)), ((n_kv - 1) >> 1) & 1, abort_flag, p.status, 43);
         tc_fence_after();
+        if constexpr (kHalves == 2) {
+            xchg[256 + hf * 128 + r] = l;
+            named_barrier_sync(pair_bar, 64);
+            l += xchg[256 + (hf ^ 1) * 128 + r];
+        }
         const int32_t q = q0 + t * kRowsPerTile + r;
         const float inv_l = 1.0f / l;
         const float lse_nat = (m + log2f(l)) * kLn2;
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            tmem_ld32(tO + c * 32, o);
+        for (int c = 0; c < kOC / kOP; ++c) {
+            uint32_t o[kOP];
+            tmem_ld<kOP>(tO + c * kOP, o);
             tmem_wait_ld();
             if (q < n_g) {
                 if (kPartial) {
-                    float4* dst = (float4*)(p.part_o + (((size_t)chunk * p.n_total + q) * p.n_heads + h) * D + c * 32);
+                    float4* dst = (float4*)(p.part_o + (((size_t)chunk * p.n_total + q) * p.n_heads + h) * D + hf * kOC + c * kOP);
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
+                    for (int i = 0; i < kOP / 4; ++i)
                         dst[i] = make_float4(__uint_as_float(o[4 * i]) * inv_l, __uint_as_float(o[4 * i + 1]) * inv_l,
                                              __uint_as_float(o[4 * i + 2]) * inv_l, __uint_as_float(o[4 * i + 3]) * inv_l);
                 } else {
-                    uint4* dst = (uint4*)(p.out + ((size_t)(node0 + q) * p.n_heads + h) * D + c * 32);
+                    uint4* dst = (uint4*)(p.out + ((size_t)(node0 + q) * p.n_heads + h) * D + hf * kOC + c * kOP);
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
+                    for (int i = 0; i < kOP / 8; ++i) {
                         uint4 v;
                         v.x = pack_bf16x2(__uint_as_float(o[8 * i]) * inv_l, __uint_as_float(o[8 * i + 1]) * inv_l);
                         v.y = pack_bf16x2(__uint_as_float(o[8 * i + 2]) * inv_l, __uint_as_float(o[8 * i + 3]) * inv_l);
@@ -502,7 +529,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 }
             }
         }
-        if (q < n_g) {
+        if (q < n_g && hf == 0) {
             if (kPartial) p.part_lse[((size_t)chunk * p.n_heads + h) * p.n_total + q] = lse_nat;
             else p.lse[(size_t)h * p.n_total + node0 + q] = lse_nat;
         }

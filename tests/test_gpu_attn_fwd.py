@@ -61,6 +61,15 @@ def test_large_bias_spread_and_max_dist_254():
     check_forward(w)
 
 
+@pytest.mark.parametrize("n,d,max_dist", [(700, 64, 6), (1500, 64, 254), (1500, 32, 30), (900, 32, 254)])
+def test_reference_maximum_raised_in_late_key_tiles(n, d, max_dist):
+    # large bias spread over many key tiles: rows keep meeting keys far above
+    # their running reference, in different tiles for different rows of the same query tile
+    w = wl.small_workload([n], 2, d, max_dist, seed=n + d, avg_degree=1.3)
+    w.tensors().bias[:] *= 12.0
+    check_forward(w)
+
+
 @pytest.mark.parametrize("name", ["tiny_er256", "tiny_er256_sparse", "ba4096", "varlen_rgg64"])
 def test_named_workloads(name):
     check_forward(wl.make_workload(name), strict=True)     # the stated 1e-2 bound, no allowance
