@@ -9,23 +9,34 @@
 // gradient dB[h][b] = sum of dS over pairs in bucket b is binned in shared memory (one
 // private bin column per thread, no conflicts) and flushed once per CTA with fp64 atomics.
 //
+// The two per-query terms of the softmax gradient are folded into the MMAs: a pre-pass writes,
+// for every (query, head), a row of 16 bf16 holding -lse*sqrt(d) and -Delta, each split into three
+// bf16 terms (24 mantissa bits); one extra K=16 step against a constant tile of ones adds them,
+// so tensor memory already holds  S^T - lse*sqrt(d)  and  dP^T - Delta  and no thread loads or
+// subtracts a per-query value.
+//
+// Each query tile is processed as two halves of 64 queries with their own TMEM stage, MMAs and
+// barriers; eight softmax warps own each half.  While one half's MMAs (dV, dK, next S^T, next
+// dP^T) run, the other half's warps compute, and no softmax thread ever waits at a CTA-wide
+// barrier: it arrives on an mbarrier when its P^T / dS^T are stored and only waits for its own
+// next inputs.  All MMAs are issued by one thread, in an order that makes every TMEM reuse
+// (next S^T over P^T, next dP^T over dS^T) follow the MMA that reads the old contents.
+//
 // Because the scores are transposed, a thread walks along QUERY indices for a fixed key, i.e.
 // down a column of the SPD matrix.  A pre-pass therefore writes a transposed copy of the SPD
 // matrix into the workspace (values clamped to the last bucket on the way), so that the kernel
 // reads each thread's 32 bucket bytes as two 16-byte words instead of 32 byte loads.
 //
-//   warp 0        TMA producer: K, V once; Q_i, dO_i and (single graph) the SPD^T tile, 2-stage ring
-//   warp 1        aux loader: lse*log2(e) and Delta of the query tile; SPD^T tile for packed batches
-//   warp 2        issues S^T = K Q_i^T of the next query tile (not urgent, so it can live in a helper warp)
-//   warps 4-19    sixteen softmax warps = four groups of 128 threads; group g owns query columns
-//                 [32g, 32g+32) of the tile (32 score elements per thread).  Many warps rather than
-//                 long rows per thread: the per-element work is a chain of dependent shared-memory
-//                 lookups, which only thread-level parallelism hides.  Two of these warps also issue
-//                 the MMAs (after a barrier of all softmax threads): a separate MMA warp would be
-//                 starved of issue slots by the busy warps on its scheduler.
-//   warps 20-23   dQ reducer: TMEM -> red.global.add.v4.f32
+//   warp 0        TMA producer: K, V, the constant tiles once; Q_i, dO_i, the per-query rows and
+//                 (single graph) the SPD^T tile through a 2-stage ring
+//   warp 1        MMA issuer
+//   warp 2        SPD^T tile loader for packed batches (per-graph pitch: cp.async)
+//   warps 4-19    softmax: warps 4-11 own queries [0,64) of every tile, warps 12-19 queries [64,128);
+//                 within a half, four warps per 32 query columns (32 score elements per thread)
+//   warps 20-23   dQ reducer: TMEM -> shared memory -> TMA reduce-add into the fp32 accumulator
 //
-// TMEM columns: S^T/P^T [0,128)  dP^T/dS^T [128,256)  dV [256,320)  dK [320,384)  dQ0 [384,448)  dQ1 [448,512).
+// TMEM columns, half g: S^T/P^T [128g, 128g+64)  dP^T/dS^T [128g+64, 128g+128);
+//               dV [256,320)  dK [320,384)  dQ of even / odd tiles [384,448) / [448,512).
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -38,19 +49,19 @@ namespace {
 using namespace sm100;
 
 constexpr int kTile = 128;
+constexpr int kHalf = 64;                   // queries per TMEM stage
 constexpr int kStages = 2;
 constexpr int kBwdThreads = 768;
 constexpr int kSoftmaxThreads = 512;
-constexpr int kColsPerThread = 32;
-constexpr int kMaxPrivateBinBuckets = 28;   // 2 KB of shared memory per bucket
+constexpr int kMaxPrivateBinBuckets = 27;   // 2 KB of shared memory per bucket
+constexpr int kExtCols = 16;                // bf16 per (query, head) row of folded terms
+constexpr int kExtTileBytes = kTile * kExtCols * 2;
 
 struct BwdParams {
     const uint8_t* spd_t;    // transposed, clamped copy of the SPD blocks (workspace)
     const int64_t* spd_offsets;
     const int32_t* cu_seqlens;
     const float* bias;
-    const float* lse2;       // [H,T] lse * log2(e)      (workspace)
-    const float* delta;      // [H,T] rowsum(dO * O)     (workspace)
     float* dq_acc;           // [T,H,D] fp32             (workspace, zeroed)
     double* db_acc;          // [H,nb] fp64              (workspace, zeroed)
     __nv_bfloat16* dk;
@@ -65,19 +76,19 @@ struct BwdParams {
 };
 
 enum BwdBarrier {
-    kBarKvFull = 0,
-    kBarQdoFull = 1,                       // [2]
-    kBarAuxFull = kBarQdoFull + kStages,   // [2]  SPD tile + lse2 + Delta
-    kBarStageEmpty = kBarAuxFull + kStages,// [2]  one arrive: the dQ reducer, after its TMA reduce has read the stage
-    kBarDvDone = kBarStageEmpty + kStages, // [2]  commit after dV += P^T dO_i (dO_i no longer read)
-    kBarSFull = kBarDvDone + kStages,
-    kBarDpFull,
-    kBarDqFull,                            // [2]
-    kBarDqFree = kBarDqFull + 2,           // [2]
-    kBarFinal = kBarDqFree + 2,            //      two commits
+    kBarKvFull = 0,                          //      K, V and the constant tiles
+    kBarQdoFull = 1,                         // [2]  Q_i, dO_i and the per-query rows of tile i
+    kBarSpdFull = kBarQdoFull + kStages,     //      SPD^T tile (single buffer)
+    kBarSpdEmpty,                            //      16 arrivals: every softmax warp holds its bucket bytes in registers
+    kBarStageEmpty,                          // [2]  commit behind the last MMA that reads Q_i / dO_i
+    kBarInFull = kBarStageEmpty + kStages,   // [2]  per half: S^T and dP^T of the next tile are in tensor memory
+    kBarReady = kBarInFull + 2,              // [2]  per half: 256 arrivals, P^T and dS^T stored
+    kBarDqFull = kBarReady + 2,              // [2]
+    kBarDqFree = kBarDqFull + 2,             // [2]
+    kBarFinal = kBarDqFree + 2,
     kNumBwdBarriers
 };
-enum BwdNamedBarrier { kNbFlush = 1, kNbPStored = 2, kNbDsStored = 3, kNbDqStaged = 4 };
+enum BwdNamedBarrier { kNbFlush = 1, kNbDqStaged = 4, kNbDqStagingFree = 5 };
 
 template <int D>
 struct BwdSmem {
@@ -86,13 +97,14 @@ struct BwdSmem {
     static constexpr int kSpdBytes = kTile * kTile;
     static constexpr int kK = 0;
     static constexpr int kV = kK + kTileBytes;
-    static constexpr int kStageBytes = 2 * kTileBytes;              // Q_i then dO_i; later the dQ_i staging area
-    static constexpr int kQ = kV + kTileBytes;                      // [kStages] at stride kStageBytes
+    static constexpr int kOnes = kV + kTileBytes;                   // two constant groups of 8 x 16 bf16 (256 B each)
+    static constexpr int kStageBytes = 2 * kTileBytes;              // Q_i then dO_i
+    static constexpr int kQ = kOnes + 1024;                         // [kStages] at stride kStageBytes
     static constexpr int kDo = kQ + kTileBytes;                     // [kStages] at stride kStageBytes
-    static constexpr int kSpd = kQ + kStages * kStageBytes;         // [kStages]
-    static constexpr int kLse = kSpd + kStages * kSpdBytes;         // [kStages][128] float
-    static constexpr int kDelta = kLse + kStages * 512;             // [kStages][128] float
-    static constexpr int kDs = kDelta + kStages * 512;              // 2 atoms x 128 rows x 128 B
+    static constexpr int kExt = kQ + kStages * kStageBytes;         // [kStages] per-query rows
+    static constexpr int kSpd = kExt + kStages * kExtTileBytes;     // one tile: refilled while the threads work from registers
+    static constexpr int kStg = kSpd + kSpdBytes;                   // dQ staging: 128 rows x 32 floats
+    static constexpr int kDs = kStg + 16384;                        // 2 atoms x 128 rows x 128 B
     static constexpr int kBias = kDs + 32768;
     static constexpr int kBars = kBias + 256 * 4;
     static constexpr int kMisc = kBars + kNumBwdBarriers * 8;
@@ -100,10 +112,6 @@ struct BwdSmem {
     static size_t dynamic_bytes(int bin_floats) { return (size_t)kBins + (size_t)bin_floats * 4 + 1024; }
 };
 
-__device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src, uint32_t src_bytes)
-{
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
-}
 // register budget: the CTA is launched with 768 x 80 registers; after the re-split it holds
 // 128 x 40 + 512 x 96 + 128 x 48 = 60416 <= 61440 (an increase can only draw on what the CTA owns)
 __device__ __forceinline__ void setmaxnreg_inc_96() { asm volatile("setmaxnreg.inc.sync.aligned.u32 96;"); }
@@ -113,6 +121,7 @@ template <int D, bool kPrivateBins, bool kShflBias>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_do,
+                const __grid_constant__ CUtensorMap tmap_ext,
                 const __grid_constant__ CUtensorMap tmap_spd, const __grid_constant__ CUtensorMap tmap_dq,
                 const BwdParams p)
 {
@@ -148,20 +157,21 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         mbar_init(bar(kBarKvFull), 1);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar(kBarQdoFull + s), 1);
-            mbar_init(bar(kBarAuxFull + s), p.spd_tma ? 33 : 32);
             mbar_init(bar(kBarStageEmpty + s), 1);
-            mbar_init(bar(kBarDvDone + s), 1);
+            mbar_init(bar(kBarInFull + s), 1);
+            mbar_init(bar(kBarReady + s), kSoftmaxThreads / 2);
             mbar_init(bar(kBarDqFull + s), 1);
             mbar_init(bar(kBarDqFree + s), 128);
         }
-        mbar_init(bar(kBarSFull), 1);
-        mbar_init(bar(kBarDpFull), 1);
-        mbar_init(bar(kBarFinal), 2);
+        mbar_init(bar(kBarSpdFull), p.spd_tma ? 1 : 32);
+        mbar_init(bar(kBarSpdEmpty), 16);
+        mbar_init(bar(kBarFinal), 1);
         fence_mbar_init();
         prefetch_tensormap(&tmap_q);
         prefetch_tensormap(&tmap_k);
         prefetch_tensormap(&tmap_v);
         prefetch_tensormap(&tmap_do);
+        prefetch_tensormap(&tmap_ext);
         prefetch_tensormap(&tmap_dq);
         if (p.spd_tma) prefetch_tensormap(&tmap_spd);
     }
@@ -169,11 +179,21 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     for (int i = tid; i < 256; i += kBwdThreads)
         s_bias[i] = p.bias[(size_t)h * p.n_buckets + min(i, p.n_buckets - 1)] * kLog2e;
     for (int i = tid; i < n_bin_floats; i += kBwdThreads) s_bins[i] = 0.f;
+    if (tid < 32) {
+        // 8 rows x 32 bytes per group in the 32-byte swizzle: the 16-byte half that holds columns 0..7 sits
+        // first in rows 0-3 and second in rows 4-7.  Group 0: ones in columns 0..2 (multiplies the -lse terms),
+        // group 1: ones in columns 8..10 (the -Delta terms).
+        const int grp_ = tid >> 4, row = (tid >> 1) & 7, phys_half = tid & 1;
+        const int logical_half = phys_half ^ (row >> 2);
+        const bool has_ones = logical_half == grp_;
+        *(uint4*)(smem + L::kOnes + tid * 16) = has_ones ? make_uint4(0x3f803f80u, 0x00003f80u, 0u, 0u) : make_uint4(0u, 0u, 0u, 0u);
+        fence_proxy_async_smem();
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = misc[0];
-    constexpr uint32_t kColS = 0, kColDp = 128, kColDv = 256, kColDk = 320, kColDq = 384;
+    constexpr uint32_t kColDv = 256, kColDk = 320, kColDq = 384;
 
     if (warp < 4) {
         setmaxnreg_dec_40();
@@ -189,128 +209,153 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 mbar_wait(bar(kBarStageEmpty + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 110);
                 if (lane == 0) {
                     const int32_t row = node0 + i * kTile;
-                    mbar_arrive_expect_tx(bar(kBarQdoFull + s), 2 * L::kTileBytes);
+                    mbar_arrive_expect_tx(bar(kBarQdoFull + s), 2 * L::kTileBytes + kExtTileBytes);
                     tma_load_3d(smem_u32(smem + L::kQ + s * L::kStageBytes), &tmap_q, bar(kBarQdoFull + s), 0, h, row);
                     tma_load_3d(smem_u32(smem + L::kDo + s * L::kStageBytes), &tmap_do, bar(kBarQdoFull + s), 0, h, row);
-                    if (p.spd_tma) {
-                        mbar_arrive_expect_tx(bar(kBarAuxFull + s), L::kSpdBytes);
-                        tma_load_2d(smem_u32(smem + L::kSpd + s * L::kSpdBytes), &tmap_spd, bar(kBarAuxFull + s), i * kTile, kv0);
+                    tma_load_3d(smem_u32(smem + L::kExt + s * kExtTileBytes), &tmap_ext, bar(kBarQdoFull + s), 0, h, row);
+                }
+                __syncwarp();
+                if (p.spd_tma) {
+                    if (i > 0) mbar_wait(bar(kBarSpdEmpty), (i - 1) & 1, abort_flag, p.status, 111);
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(bar(kBarSpdFull), L::kSpdBytes);
+                        tma_load_2d(smem_u32(smem + L::kSpd), &tmap_spd, bar(kBarSpdFull), i * kTile, kv0);
                     }
+                    __syncwarp();
                 }
-                __syncwarp();
-            }
-        } else if (warp == 2) {
-            // ------------------------------ S^T issuer ------------------------------
-            // S^T of the NEXT query tile is not urgent (it is consumed a whole tile later), so it is
-            // issued from this otherwise idle warp as soon as Q_{i} has landed and dV of the previous
-            // tile (which reads P^T from the same TMEM columns) has completed; no softmax warp waits.
-            constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
-            const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
-            mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 160);
-            for (int i = 0; i < n_q; ++i) {
-                const int s = i & 1;
-                mbar_wait(bar(kBarQdoFull + s), (i >> 1) & 1, abort_flag, p.status, 161);
-                if (i > 0) mbar_wait(bar(kBarDvDone + (s ^ 1)), ((i - 1) >> 1) & 1, abort_flag, p.status, 162);
-                tc_fence_after();
-                if (elect_one()) {
-                    const uint64_t da = make_smem_desc(smem_u32(smem + L::kK), L::kRowBytes, 0);
-                    const uint64_t db = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes), L::kRowBytes, 0);
-#pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)
-                        mma_ss(tm + kColS, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
-                    mma_commit(bar(kBarSFull));
-                }
-                __syncwarp();
             }
         } else if (warp == 1) {
-            // ------------------------------ aux loader ------------------------------
+            // ------------------------------- MMA issuer -------------------------------
+            constexpr uint32_t idesc_in = make_idesc_bf16(128, kHalf, false, false);   // S^T, dP^T of 64 queries
+            constexpr uint32_t idesc_ts = make_idesc_bf16(128, D, false, true);        // A in TMEM, B MN-major
+            constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);         // A and B MN-major
+            const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+            const uint32_t sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV);
+            const uint64_t desc_k = make_smem_desc(sK, L::kRowBytes, 0), desc_v = make_smem_desc(sV, L::kRowBytes, 0);
+            // constant A operands of the extra K step: every 8-row group reads the same 256 bytes (group stride 0)
+            const uint64_t desc_ones_s = make_smem_desc_stride(smem_u32(smem + L::kOnes), kExtCols * 2, 0, 0);
+            const uint64_t desc_ones_dp = make_smem_desc_stride(smem_u32(smem + L::kOnes + 256), kExtCols * 2, 0, 0);
+            // S^T - lse sqrt(d) and dP^T - Delta of half `sub` of query tile i -> TMEM stage `sub`
+            auto issue_inputs = [&](int i, int sub) {
+                const int s = i & 1;
+                const uint64_t dq_ = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
+                const uint64_t ddo = make_smem_desc(smem_u32(smem + L::kDo + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
+                const uint64_t dext = make_smem_desc(smem_u32(smem + L::kExt + s * kExtTileBytes) + sub * kHalf * kExtCols * 2, kExtCols * 2, 0);
+                const uint32_t d_s = tm + sub * 128, d_dp = d_s + kHalf;
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    mma_ss(d_s, advance_desc(desc_k, ks * 32), advance_desc(dq_, ks * 32), idesc_in, ks > 0);
+                mma_ss(d_s, desc_ones_s, dext, idesc_in, 1u);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)
+                    mma_ss(d_dp, advance_desc(desc_v, ks * 32), advance_desc(ddo, ks * 32), idesc_in, ks > 0);
+                mma_ss(d_dp, desc_ones_dp, dext, idesc_in, 1u);
+                mma_commit(bar(kBarInFull + sub));
+            };
+            mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 120);
+            mbar_wait(bar(kBarQdoFull + 0), 0, abort_flag, p.status, 121);
+            tc_fence_after();
+            if (elect_one()) { issue_inputs(0, 0); issue_inputs(0, 1); }
+            __syncwarp();
             for (int i = 0; i < n_q; ++i) {
                 const int s = i & 1;
-                mbar_wait(bar(kBarStageEmpty + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 130);
-                const int32_t q0 = i * kTile;
-                if (!p.spd_tma) {
-                    // same layout as the TMA 128-byte swizzle: 16-byte chunk c of row r at chunk c ^ (r & 7)
-                    const uint32_t dst0 = smem_u32(smem + L::kSpd + s * L::kSpdBytes);
-#pragma unroll 4
-                    for (int it = 0; it < (kTile * 8) / 32; ++it) {
-                        const int c = it * 32 + lane;
-                        const int r = c >> 3, cc = c & 7;
-                        const int64_t col = (int64_t)q0 + cc * 16;
-                        const bool valid = (kv0 + r < n_g) && (col < ld);
-                        const uint8_t* src = valid ? spd_g + (int64_t)(kv0 + r) * ld + col : spd_g;
-                        cp_async_16(dst0 + r * 128 + ((cc ^ (r & 7)) << 4), src, valid ? 16u : 0u);
-                    }
-                }
-                const uint32_t dl = smem_u32(smem + L::kLse + s * 512), dd = smem_u32(smem + L::kDelta + s * 512);
 #pragma unroll
-                for (int it = 0; it < 4; ++it) {
-                    const int r = it * 32 + lane;
-                    const bool valid = q0 + r < n_g;
-                    const size_t off = (size_t)h * p.n_total + node0 + (valid ? q0 + r : 0);
-                    cp_async_4(dl + r * 4, p.lse2 + off, valid ? 4u : 0u);
-                    cp_async_4(dd + r * 4, p.delta + off, valid ? 4u : 0u);
+                for (int sub = 0; sub < 2; ++sub) {
+                    if (sub == 0 && i + 1 < n_q)
+                        mbar_wait(bar(kBarQdoFull + (s ^ 1)), ((i + 1) >> 1) & 1, abort_flag, p.status, 122);
+                    if (sub == 1) mbar_wait(bar(kBarDqFree + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 125);
+                    mbar_wait(bar(kBarReady + sub), i & 1, abort_flag, p.status, 123);
+                    tc_fence_after();
+                    if (elect_one()) {
+                        const uint32_t t_p = tm + sub * 128, t_ds = t_p + kHalf;
+                        const uint64_t ddo = make_smem_desc(smem_u32(smem + L::kDo + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
+                        const uint64_t dq_ = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
+#pragma unroll
+                        for (int ks = 0; ks < kHalf / 16; ++ks)     // dV += P^T dO   (P^T of query group ks/2 at the start of its 32 columns)
+                            mma_ts(tm + kColDv, t_p + (ks >> 1) * 32 + (ks & 1) * 8,
+                                   advance_desc(ddo, ks * 16 * L::kRowBytes), idesc_ts, (i > 0 || sub > 0 || ks > 0) ? 1u : 0u);
+#pragma unroll
+                        for (int ks = 0; ks < kHalf / 16; ++ks)     // dK += dS^T Q
+                            mma_ts(tm + kColDk, t_ds + (ks >> 1) * 32 + (ks & 1) * 8,
+                                   advance_desc(dq_, ks * 16 * L::kRowBytes), idesc_ts, (i > 0 || sub > 0 || ks > 0) ? 1u : 0u);
+                        if (sub == 1) mma_commit(bar(kBarStageEmpty + s));   // Q_i, dO_i and their per-query rows are dead
+                        if (i + 1 < n_q) issue_inputs(i + 1, sub);   // over P^T / dS^T just consumed (MMAs run in issue order)
+                        if (sub == 1) {                              // dQ_i = dS K
+                            const uint64_t da = make_smem_desc(smem_u32(smem + L::kDs), 128, 16384);
+#pragma unroll
+                            for (int ks = 0; ks < 8; ++ks)
+                                mma_ss(tm + kColDq + s * 64, advance_desc(da, ks * 2048),
+                                       advance_desc(desc_k, ks * 16 * L::kRowBytes), idesc_dq, ks > 0);
+                            mma_commit(bar(kBarDqFull + s));
+                            if (i + 1 == n_q) mma_commit(bar(kBarFinal));
+                        }
+                    }
+                    __syncwarp();
                 }
-                cp_async_mbar_arrive_noinc(bar(kBarAuxFull + s));
+            }
+        } else if (warp == 2 && !p.spd_tma) {
+            // --------------------- SPD^T tile loader for packed batches ---------------------
+            for (int i = 0; i < n_q; ++i) {
+                if (i > 0) mbar_wait(bar(kBarSpdEmpty), (i - 1) & 1, abort_flag, p.status, 130);
+                const int32_t q0 = i * kTile;
+                // same layout as the TMA 128-byte swizzle: 16-byte chunk c of row r at chunk c ^ (r & 7)
+                const uint32_t dst0 = smem_u32(smem + L::kSpd);
+#pragma unroll 4
+                for (int it = 0; it < (kTile * 8) / 32; ++it) {
+                    const int c = it * 32 + lane;
+                    const int r = c >> 3, cc = c & 7;
+                    const int64_t col = (int64_t)q0 + cc * 16;
+                    const bool valid = (kv0 + r < n_g) && (col < ld);
+                    const uint8_t* src = valid ? spd_g + (int64_t)(kv0 + r) * ld + col : spd_g;
+                    cp_async_16(dst0 + r * 128 + ((cc ^ (r & 7)) << 4), src, valid ? 16u : 0u);
+                }
+                cp_async_mbar_arrive_noinc(bar(kBarSpdFull));
             }
         }
     } else if (warp < 20) {
         // ================================ softmax warps ================================
         setmaxnreg_inc_96();
-        const int grp = (warp - 4) >> 2;                // query-column group: columns [32 grp, 32 grp + 32)
+        const int half = (warp - 4) >> 3;               // query half of every tile = TMEM stage
+        const int grp = (warp - 4) >> 2;                // query-column group: columns [32 grp, 32 grp + 32) of the tile
         const int r = ((warp & 3) << 5) | lane;         // key row within the tile = TMEM lane
         const int st = tid - 128;                       // 0..511 index among softmax threads
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + kColS + grp * 32 + lane_off;
-        const uint32_t tDp = tmem + kColDp + grp * 32 + lane_off;
+        const uint32_t tS = tmem + half * 128 + (grp & 1) * 32 + lane_off;
+        const uint32_t tDp = tS + kHalf;
         const bool kv_valid = kv0 + r < n_g;
-        const float c1 = p.c1;
+        const uint64_t c1c1 = pack_f32x2(p.c1, p.c1);
         const float tbl = s_bias[lane];
         float* my_bins = s_bins + (kPrivateBins ? st : lane);
         // the thread's 32 bucket bytes: row r of the SPD^T tile, 16-byte chunks 2 grp and 2 grp + 1 (swizzled by r & 7)
         const uint32_t spd_off0 = r * 128 + (((2 * grp) ^ (r & 7)) << 4), spd_off1 = r * 128 + (((2 * grp + 1) ^ (r & 7)) << 4);
         const uint32_t bins_base = smem_u32(my_bins);
-
-        // ---- MMA issue duty (after the barriers of all softmax threads) ----
-        const bool issuer_a = warp == 4;                // dV
-        const bool issuer_b = warp == 9;                // dK, dQ, dP^T
-        constexpr uint32_t idesc_s = make_idesc_bf16(128, 128, false, false);
-        constexpr uint32_t idesc_ts = make_idesc_bf16(128, D, false, true);    // A in TMEM, B MN-major
-        constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);     // A and B MN-major
-        const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
-        const uint32_t sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV);
-        auto issue_dpt = [&](int i) {                   // dP^T = V dO_i^T
-            const int s = i & 1;
-            mbar_wait(bar(kBarQdoFull + s), (i >> 1) & 1, abort_flag, p.status, 121);
-            tc_fence_after();
-            if (elect_one()) {
-                const uint64_t da = make_smem_desc(sV, L::kRowBytes, 0);
-                const uint64_t db = make_smem_desc(smem_u32(smem + L::kDo + s * L::kStageBytes), L::kRowBytes, 0);
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ss(tm + kColDp, advance_desc(da, ks * 32), advance_desc(db, ks * 32), idesc_s, ks > 0);
-                mma_commit(bar(kBarDpFull));
-            }
-            __syncwarp();
-        };
-        if (issuer_b) { mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 123); issue_dpt(0); }
+        uint8_t* ds_row = smem + L::kDs + half * 16384 + r * 128;
 
         for (int i = 0; i < n_q; ++i) {
             const int s = i & 1;
-            float pr[kColsPerThread];
-            uint32_t acc[32];
-            // ---------------- P^T = exp2(S^T c1 + b2 - lse2) ----------------
-            mbar_wait(bar(kBarSFull), i & 1, abort_flag, p.status, 140);
+            float pr[32];
+            uint32_t dpa[16], dpb[16];
+            mbar_wait(bar(kBarInFull + half), i & 1, abort_flag, p.status, 140);
             tc_fence_after();
-            tmem_ld32(tS, acc);
-            mbar_wait(bar(kBarAuxFull + s), (i >> 1) & 1, abort_flag, p.status, 141);
-            const uint8_t* spd_tile = smem + L::kSpd + s * L::kSpdBytes;
+            {
+                uint32_t sv[32];
+                tmem_ld32(tS, sv);
+                tmem_ld16(tDp, dpa);
+                mbar_wait(bar(kBarSpdFull), i & 1, abort_flag, p.status, 141);
+                tmem_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 32; ++c) pr[c] = __uint_as_float(sv[c]);
+            }
+            const uint8_t* spd_tile = smem + L::kSpd;
             const uint4 w0 = *(const uint4*)(spd_tile + spd_off0), w1 = *(const uint4*)(spd_tile + spd_off1);
             const uint32_t bw[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};   // bucket bytes, already clamped
-            const float4* lse4 = (const float4*)(smem + L::kLse + s * 512 + grp * 128);
-            tmem_wait_ld();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarSpdEmpty));     // the single SPD buffer may be refilled
+
+            // ---------------- P^T = exp2((S^T - lse sqrt(d)) c1 + b2) ----------------
 #pragma unroll
             for (int rnd = 0; rnd < 2; ++rnd) {             // 16 elements per round: lookups first, math after
-                float bb[16], ls[16];
+                float bb[16];
 #pragma unroll
                 for (int k = 0; k < 16; ++k) {
                     const int c = rnd * 16 + k;
@@ -318,14 +363,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     bb[k] = kShflBias ? __shfl_sync(0xffffffffu, tbl, sh) : s_bias[sh & 0xffu];
                 }
 #pragma unroll
-                for (int k4 = 0; k4 < 4; ++k4) {
-                    const float4 l4 = lse4[rnd * 4 + k4];
-                    ls[4 * k4] = l4.x; ls[4 * k4 + 1] = l4.y; ls[4 * k4 + 2] = l4.z; ls[4 * k4 + 3] = l4.w;
-                }
-#pragma unroll
-                for (int k = 0; k < 16; ++k) {
+                for (int k = 0; k < 16; k += 2) {
                     const int c = rnd * 16 + k;
-                    pr[c] = ex2_approx(fmaf(__uint_as_float(acc[c]), c1, bb[k]) - ls[k]);
+                    float lo, hi;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(pr[c], pr[c + 1]), c1c1, pack_f32x2(bb[k], bb[k + 1])), lo, hi);
+                    pr[c] = ex2_approx(lo);
+                    pr[c + 1] = ex2_approx(hi);
                 }
             }
             const int nq_valid = n_g - i * kTile - grp * 32;      // valid query columns of this group
@@ -339,42 +382,15 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 #pragma unroll
                 for (int c = 0; c < 16; ++c) pk[c] = pack_bf16x2(pr[2 * c], pr[2 * c + 1]);
                 tmem_st16(tS, pk);                      // P^T of this group: 16 packed columns at the start of its range
-                tmem_wait_st();
             }
-            mbar_wait(bar(kBarDpFull), i & 1, abort_flag, p.status, 142);
-            tc_fence_after();
-            tmem_ld32(tDp, acc);                        // dP^T of this tile: its latency hides behind the barrier
-            tc_fence_before();
-            named_barrier_sync(kNbPStored, kSoftmaxThreads);
-            if (issuer_a) {
-                tc_fence_after();
-                if (elect_one()) {                      // dV += P^T dO_i
-                    const uint64_t db = make_smem_desc(smem_u32(smem + L::kDo + s * L::kStageBytes), L::kRowBytes, 0);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        mma_ts(tm + kColDv, tm + kColS + (ks >> 1) * 32 + (ks & 1) * 8,
-                               advance_desc(db, ks * 16 * L::kRowBytes), idesc_ts, (i > 0 || ks > 0) ? 1u : 0u);
-                    mma_commit(bar(kBarDvDone + s));
-                    if (i + 1 == n_q) mma_commit(bar(kBarFinal));
-                }
-                __syncwarp();
-            }
+            tmem_ld16(tDp + 16, dpb);
 
-            // ---------------- dS^T = P^T o (dP^T - Delta) ----------------
-            const float4* dl4 = (const float4*)(smem + L::kDelta + s * 512 + grp * 128);
-            tmem_wait_ld();
+            // ---------------- dS^T = P^T o (dP^T - Delta), bias-gradient bins ----------------
+            auto ds_round = [&](int rnd, const uint32_t (&dp)[16]) {
 #pragma unroll
-            for (int rnd = 0; rnd < 2; ++rnd) {
-                float dl[16];
-#pragma unroll
-                for (int k4 = 0; k4 < 4; ++k4) {
-                    const float4 d4 = dl4[rnd * 4 + k4];
-                    dl[4 * k4] = d4.x; dl[4 * k4 + 1] = d4.y; dl[4 * k4 + 2] = d4.z; dl[4 * k4 + 3] = d4.w;
-                }
-#pragma unroll
-                for (int k = 0; k < 16; ++k) {
+                for (int k = 0; k < 16; k += 2) {
                     const int c = rnd * 16 + k;
-                    pr[c] = pr[c] * (__uint_as_float(acc[c]) - dl[k]);
+                    unpack_f32x2(mul_f32x2(pack_f32x2(pr[c], pr[c + 1]), pack_u32x2(dp[k], dp[k + 1])), pr[c], pr[c + 1]);
                 }
 #pragma unroll
                 for (int k = 0; k < 16; ++k) {
@@ -392,13 +408,17 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         atomicAdd((float*)((uint8_t*)my_bins + off), pr[c]);
                     }
                 }
-            }
+            };
+            ds_round(0, dpa);
+            tmem_wait_ld();
+            ds_round(1, dpb);
             {
                 uint32_t pk[16];
 #pragma unroll
                 for (int c = 0; c < 16; ++c) pk[c] = pack_bf16x2(pr[2 * c], pr[2 * c + 1]);
                 tmem_st16(tDp, pk);
-                uint8_t* ds_row = smem + L::kDs + (grp >> 1) * 16384 + r * 128;
+                // dQ of the previous tile has read the dS^T tile in shared memory
+                if (i > 0) mbar_wait(bar(kBarDqFull + (s ^ 1)), ((i - 1) >> 1) & 1, abort_flag, p.status, 142);
 #pragma unroll
                 for (int c8 = 0; c8 < 4; ++c8)
                     *(uint4*)(ds_row + ((((grp & 1) * 4 + c8) ^ (r & 7)) << 4)) =
@@ -407,53 +427,31 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             }
             fence_proxy_async_smem();
             tc_fence_before();
-            named_barrier_sync(kNbDsStored, kSoftmaxThreads);
-            if (issuer_b) {
-                mbar_wait(bar(kBarDqFree + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 125);
-                tc_fence_after();
-                if (elect_one()) {                      // dK += dS^T Q_i ;  dQ_i = dS K
-                    const uint64_t dbq = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes), L::kRowBytes, 0);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        mma_ts(tm + kColDk, tm + kColDp + (ks >> 1) * 32 + (ks & 1) * 8,
-                               advance_desc(dbq, ks * 16 * L::kRowBytes), idesc_ts, (i > 0 || ks > 0) ? 1u : 0u);
-                    const uint64_t da = make_smem_desc(smem_u32(smem + L::kDs), 128, 16384);
-                    const uint64_t dbk = make_smem_desc(sK, L::kRowBytes, 0);
-#pragma unroll
-                    for (int ks = 0; ks < 8; ++ks)
-                        mma_ss(tm + kColDq + s * 64, advance_desc(da, ks * 2048),
-                               advance_desc(dbk, ks * 16 * L::kRowBytes), idesc_dq, ks > 0);
-                    mma_commit(bar(kBarDqFull + s));
-                    if (i + 1 == n_q) mma_commit(bar(kBarFinal));
-                }
-                __syncwarp();
-                if (i + 1 < n_q) issue_dpt(i + 1);
-            }
+            mbar_arrive(bar(kBarReady + half));
         }
 
-        // ---------------- epilogue: dV (group 0) and dK (group 1) ----------------
-        if (grp < 2) {
+        // ---------------- epilogue: dV (first half's warps) and dK (second half's) ----------------
+        {
             mbar_wait(bar(kBarFinal), 0, abort_flag, p.status, 143);
             tc_fence_after();
-            const uint32_t tacc = tmem + (grp == 0 ? kColDv : kColDk) + lane_off;
-            const float mul = grp == 0 ? 1.0f : p.scale;
-            __nv_bfloat16* dst_base = (grp == 0 ? p.dv : p.dk) + ((size_t)(node0 + kv0 + r) * p.n_heads + h) * D;
+            constexpr int kOC = D / 2;                  // output columns per thread
+            const int ch = grp & 1;
+            const uint32_t tacc = tmem + (half == 0 ? kColDv : kColDk) + ch * kOC + lane_off;
+            const float mul = half == 0 ? 1.0f : p.scale;
+            __nv_bfloat16* dst_base = (half == 0 ? p.dv : p.dk) + ((size_t)(node0 + kv0 + r) * p.n_heads + h) * D + ch * kOC;
+            uint32_t o[kOC];
+            if constexpr (kOC == 32) tmem_ld32(tacc, o); else tmem_ld16(tacc, o);
+            tmem_wait_ld();
+            if (kv_valid) {
+                uint4* dst = (uint4*)dst_base;
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t o[32];
-                tmem_ld32(tacc + c * 32, o);
-                tmem_wait_ld();
-                if (kv_valid) {
-                    uint4* dst = (uint4*)(dst_base + c * 32);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        uint4 v;
-                        v.x = pack_bf16x2(__uint_as_float(o[8 * k]) * mul, __uint_as_float(o[8 * k + 1]) * mul);
-                        v.y = pack_bf16x2(__uint_as_float(o[8 * k + 2]) * mul, __uint_as_float(o[8 * k + 3]) * mul);
-                        v.z = pack_bf16x2(__uint_as_float(o[8 * k + 4]) * mul, __uint_as_float(o[8 * k + 5]) * mul);
-                        v.w = pack_bf16x2(__uint_as_float(o[8 * k + 6]) * mul, __uint_as_float(o[8 * k + 7]) * mul);
-                        dst[k] = v;
-                    }
+                for (int k = 0; k < kOC / 8; ++k) {
+                    uint4 v;
+                    v.x = pack_bf16x2(__uint_as_float(o[8 * k]) * mul, __uint_as_float(o[8 * k + 1]) * mul);
+                    v.y = pack_bf16x2(__uint_as_float(o[8 * k + 2]) * mul, __uint_as_float(o[8 * k + 3]) * mul);
+                    v.z = pack_bf16x2(__uint_as_float(o[8 * k + 4]) * mul, __uint_as_float(o[8 * k + 5]) * mul);
+                    v.w = pack_bf16x2(__uint_as_float(o[8 * k + 6]) * mul, __uint_as_float(o[8 * k + 7]) * mul);
+                    dst[k] = v;
                 }
             }
         }
@@ -474,46 +472,40 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
     } else {
         // ================================ dQ reducer ================================
-        // dQ_i (fp32, 128 x D) goes TMEM -> registers -> the shared-memory area of this stage's Q_i and
-        // dO_i (both dead once dK and dV of this tile are done) in 128-byte-swizzled rows of 32
-        // floats, and from there to the global fp32 accumulator with TMA reduce-add: full lines
-        // to L2 instead of 16-byte scattered atomics.  Only then is the stage handed back.
+        // dQ_i (fp32, 128 x D) goes TMEM -> registers -> a staging buffer in 128-byte-swizzled rows of
+        // 32 floats, and from there to the global fp32 accumulator with TMA reduce-add: full lines
+        // to L2 instead of 16-byte scattered atomics.
         setmaxnreg_dec_48();
         const int r = ((warp & 3) << 5) | lane;
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+        uint8_t* row = smem + L::kStg + r * 128;
         for (int i = 0; i < n_q; ++i) {
             const int s = i & 1;
             mbar_wait(bar(kBarDqFull + s), (i >> 1) & 1, abort_flag, p.status, 150);
-            mbar_wait(bar(kBarDvDone + s), (i >> 1) & 1, abort_flag, p.status, 151);
             tc_fence_after();
-            uint8_t* stage = smem + L::kQ + s * L::kStageBytes;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t o[32];
                 tmem_ld32(tmem + kColDq + s * 64 + c * 32 + lane_off, o);
                 tmem_wait_ld();
-                uint8_t* row = stage + c * 16384 + r * 128;
+                if (c == D / 32 - 1) { tc_fence_before(); mbar_arrive(bar(kBarDqFree + s)); }
+                if (warp == 20 && elect_one()) bulk_wait_group_read0();      // the previous reduce has read the staging buffer
+                named_barrier_sync(kNbDqStagingFree, 128);
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
                     *(uint4*)(row + ((k ^ (r & 7)) << 4)) = make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
-            }
-            tc_fence_before();
-            mbar_arrive(bar(kBarDqFree + s));
-            fence_proxy_async_smem();
-            named_barrier_sync(kNbDqStaged, 128);
-            if (warp == 20) {
-                if (elect_one()) {
-#pragma unroll
-                    for (int c = 0; c < D / 32; ++c)
-                        tma_reduce_add_2d(&tmap_dq, smem_u32(stage + c * 16384), h * D + c * 32, node0 + i * kTile);
-                    bulk_commit_group();
-                    bulk_wait_group_read0();
-                    mbar_arrive(bar(kBarStageEmpty + s));
-                    if (i + 1 == n_q) bulk_wait_group0();      // all adds have landed before the CTA retires
+                fence_proxy_async_smem();
+                named_barrier_sync(kNbDqStaged, 128);
+                if (warp == 20) {
+                    if (elect_one()) {
+                        tma_reduce_add_2d(&tmap_dq, smem_u32(smem + L::kStg), h * D + c * 32, node0 + i * kTile);
+                        bulk_commit_group();
+                    }
+                    __syncwarp();
                 }
-                __syncwarp();
             }
         }
+        if (warp == 20 && elect_one()) bulk_wait_group0();      // all adds have landed before the CTA retires
     }
 
     tc_fence_before();
@@ -558,11 +550,22 @@ __global__ void __launch_bounds__(256) spd_transpose_clamp_kernel(const uint8_t*
     }
 }
 
-// Delta[h][t] = sum_c dO[t,h,c] * O[t,h,c];  lse2[h][t] = lse[h][t] * log2(e).
+// For every (t, h): ext[t][h][0..2] = three-term bf16 split of -lse * sqrt(d), ext[t][h][8..10] = split of
+// -Delta with Delta = sum_c dO[t,h,c] * O[t,h,c], zeros elsewhere.
+__device__ __forceinline__ void split3_bf16(float v, uint32_t& w01, uint32_t& w2)
+{
+    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+    const float r1 = v - __bfloat162float(hi);
+    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+    const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+    w01 = (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(mid) << 16);
+    w2 = (uint32_t)__bfloat16_as_ushort(lo);
+}
+
 template <int D>
 __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
-                                      const float* __restrict__ lse, float* __restrict__ delta, float* __restrict__ lse2,
-                                      int32_t n_total, int32_t n_heads)
+                                      const float* __restrict__ lse, uint4* __restrict__ ext,
+                                      int32_t n_total, int32_t n_heads, float sqrt_d)
 {
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // = t * H + h
     if (idx >= (size_t)n_total * n_heads) return;
@@ -580,9 +583,11 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ out, con
             acc += __uint_as_float(aw[k] & 0xffff0000u) * __uint_as_float(bw[k] & 0xffff0000u);
         }
     }
-    const size_t o = (size_t)h * n_total + t;
-    delta[o] = acc;
-    lse2[o] = lse[o] * kLog2e;
+    uint4 e0 = make_uint4(0u, 0u, 0u, 0u), e1 = make_uint4(0u, 0u, 0u, 0u);
+    split3_bf16(-lse[(size_t)h * n_total + t] * sqrt_d, e0.x, e0.y);
+    split3_bf16(-acc, e1.x, e1.y);
+    ext[2 * idx] = e0;
+    ext[2 * idx + 1] = e1;
 }
 
 // dq = bf16(scale * dq_acc);  dbias = float(db_acc)
@@ -600,7 +605,7 @@ __global__ void bwd_finalize_kernel(const float* __restrict__ dq_acc, __nv_bfloa
 }
 
 struct BwdWorkspace {
-    size_t db_off, delta_off, lse2_off, dq_off, spdt_off, total;
+    size_t db_off, ext_off, dq_off, spdt_off, total;
 };
 
 BwdWorkspace bwd_workspace(const gt_batch* b, int32_t n_heads, int32_t head_dim, int32_t max_dist)
@@ -608,9 +613,8 @@ BwdWorkspace bwd_workspace(const gt_batch* b, int32_t n_heads, int32_t head_dim,
     BwdWorkspace w{};
     const size_t rows = (size_t)b->n_total * n_heads;
     w.db_off = kHeaderBytes;
-    w.delta_off = w.db_off + align_up((size_t)n_heads * (max_dist + 2) * sizeof(double), 256);
-    w.lse2_off = w.delta_off + align_up(rows * sizeof(float), 256);
-    w.dq_off = w.lse2_off + align_up(rows * sizeof(float), 256);
+    w.ext_off = w.db_off + align_up((size_t)n_heads * (max_dist + 2) * sizeof(double), 256);
+    w.dq_off = w.ext_off + align_up(rows * kExtCols * 2, 256);
     w.spdt_off = w.dq_off + align_up(rows * head_dim * sizeof(float), 256);
     // transposed SPD copy: at most sum n_g * round_up(n_g,16) <= n_total * round_up(max_seqlen,16) bytes
     w.total = w.spdt_off + align_up((size_t)b->n_total * (size_t)((b->max_seqlen + 15) & ~15), 256);
@@ -619,7 +623,8 @@ BwdWorkspace bwd_workspace(const gt_batch* b, int32_t n_heads, int32_t head_dim,
 
 template <int D>
 gt_status launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
-                     const CUtensorMap& tspd, const BwdParams& p, const gt_batch* batch, cudaStream_t s)
+                     const CUtensorMap& text, const CUtensorMap& tspd, const BwdParams& p,
+                     const gt_batch* batch, cudaStream_t s)
 {
     dim3 grid((unsigned)p.n_heads, (unsigned)((batch->max_seqlen + kTile - 1) / kTile), (unsigned)batch->n_graphs);
     CUtensorMap tdq;
@@ -630,7 +635,7 @@ gt_status launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtenso
     auto kern = priv ? (p.n_buckets <= 32 ? attn_bwd_kernel<D, true, true> : attn_bwd_kernel<D, true, false>)
                      : (p.n_buckets <= 32 ? attn_bwd_kernel<D, false, true> : attn_bwd_kernel<D, false, false>);
     GT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kern<<<grid, kBwdThreads, smem, s>>>(tq, tk, tv, tdo, tspd, tdq, p);
+    kern<<<grid, kBwdThreads, smem, s>>>(tq, tk, tv, tdo, text, tspd, tdq, p);
     GT_CUDA_TRY(cudaGetLastError());
     return GT_OK;
 }
@@ -682,8 +687,6 @@ extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void
     p.spd_offsets = batch->n_graphs > 1 ? spd_offsets : nullptr;
     p.cu_seqlens = batch->n_graphs > 1 ? batch->cu_seqlens : nullptr;
     p.bias = bias;
-    p.lse2 = (float*)(ws + wsp.lse2_off);
-    p.delta = (float*)(ws + wsp.delta_off);
     p.dq_acc = (float*)(ws + wsp.dq_off);
     p.db_acc = (double*)(ws + wsp.db_off);
     p.dk = (__nv_bfloat16*)dk;
@@ -705,16 +708,18 @@ extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void
         GT_CUDA_TRY(cudaGetLastError());
     }
     const unsigned pre_blocks = (unsigned)((rows + 255) / 256);
+    uint4* ext = (uint4*)(ws + wsp.ext_off);
     if (head_dim == 64)
         bwd_preprocess_kernel<64><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse,
-                                                             (float*)(ws + wsp.delta_off), (float*)(ws + wsp.lse2_off),
-                                                             batch->n_total, n_heads);
+                                                             ext, batch->n_total, n_heads, sqrtf(64.f));
     else
         bwd_preprocess_kernel<32><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse,
-                                                             (float*)(ws + wsp.delta_off), (float*)(ws + wsp.lse2_off),
-                                                             batch->n_total, n_heads);
+                                                             ext, batch->n_total, n_heads, sqrtf(32.f));
     GT_CUDA_TRY(cudaGetLastError());
-    st = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, tspd, p, batch, s) : launch_bwd<32>(tq, tk, tv, tdo, tspd, p, batch, s);
+    CUtensorMap text;
+    if ((st = encode_thd_map(&text, ext, batch->n_total, n_heads, kExtCols)) != GT_OK) return st;
+    st = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, text, tspd, p, batch, s)
+                        : launch_bwd<32>(tq, tk, tv, tdo, text, tspd, p, batch, s);
     if (st != GT_OK) return st;
     const size_t n_vec4 = rows * head_dim / 4;
     const size_t n_fin = n_vec4 > (size_t)n_db ? n_vec4 : (size_t)n_db;

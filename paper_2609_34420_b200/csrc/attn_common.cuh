@@ -13,7 +13,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 
 // 3-D tensor map over a bf16 [T, H, d] tensor; one box = 128 consecutive rows of one head
 // (d x 1 x 128 elements), written to shared memory as 128 rows of 2d bytes with the
-// swizzle mode that matches the row length (128B for d=64, 64B for d=32).
+// swizzle mode that matches the row length (128B for d=64, 64B for d=32, 32B for d=16).
 gt_status encode_thd_map(CUtensorMap* map, const void* base, int32_t n_total, int32_t n_heads, int32_t head_dim);
 
 // 2-D tensor map over the uint8 SPD matrix of a single graph (n rows of pitch round_up(n,16));

@@ -204,6 +204,18 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr, uint32_t 
     d |= layout << 61;
     return d;
 }
+// same, with an explicit stride between 8-row groups (0 makes every group read the same bytes)
+__device__ __forceinline__ uint64_t make_smem_desc_stride(uint32_t smem_addr, uint32_t row_bytes, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    const uint64_t layout = row_bytes == 128 ? 2ull : (row_bytes == 64 ? 4ull : 6ull);
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;
+    d |= layout << 61;
+    return d;
+}
 __device__ __forceinline__ uint64_t advance_desc(uint64_t desc, uint32_t bytes) { return desc + (uint64_t)(bytes >> 4); }
 
 // Issue wrappers.  They are meant to be called by ONE lane, inside `if (elect_one()) { ... }`

@@ -33,7 +33,7 @@ gt_status encode_thd_map(CUtensorMap* map, const void* base, int32_t n_total, in
     cuuint32_t elem_strides[3] = {1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, elem_strides,
                     CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    head_dim == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                    head_dim == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : (head_dim == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B),
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? GT_OK : GT_ERR_CUDA;
 }
