@@ -36,7 +36,7 @@
 //   warps 20-23   dQ reducer: TMEM -> shared memory -> TMA reduce-add into the fp32 accumulator
 //
 // TMEM columns, half g: S^T/P^T [128g, 128g+64)  dP^T/dS^T [128g+64, 128g+128);
-//               dV [256,320)  dK [320,384)  dQ of even / odd tiles [384,448) / [448,512).
+//               dV [256,320)  dK [320,384)  dQ [384,448)  K [448,480)  V [480,512) (bf16 pairs).
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -81,11 +81,14 @@ enum BwdBarrier {
     kBarSpdFull = kBarQdoFull + kStages,     //      SPD^T tile (single buffer)
     kBarSpdEmpty,                            //      16 arrivals: every softmax warp holds its bucket bytes in registers
     kBarStageEmpty,                          // [2]  commit behind the last MMA that reads Q_i / dO_i
-    kBarInFull = kBarStageEmpty + kStages,   // [2]  per half: S^T and dP^T of the next tile are in tensor memory
-    kBarReady = kBarInFull + 2,              // [2]  per half: 256 arrivals, P^T and dS^T stored
-    kBarDqFull = kBarReady + 2,              // [2]
-    kBarDqFree = kBarDqFull + 2,             // [2]
-    kBarFinal = kBarDqFree + 2,
+    kBarSFull = kBarStageEmpty + kStages,    // [2]  per half: S^T of the next tile is in tensor memory
+    kBarDpFull = kBarSFull + 2,              // [2]  per half: dP^T of the next tile
+    kBarPReady = kBarDpFull + 2,             // [2]  per half: 256 arrivals, P^T stored
+    kBarDsReady = kBarPReady + 2,            // [2]  per half: 256 arrivals, dS^T stored (tensor and shared memory)
+    kBarDqFull = kBarDsReady + 2,
+    kBarDqFree,
+    kBarKvTmem,                              //      256 arrivals: K and V rows copied to tensor memory
+    kBarFinal,
     kNumBwdBarriers
 };
 enum BwdNamedBarrier { kNbFlush = 1, kNbDqStaged = 4, kNbDqStagingFree = 5 };
@@ -158,11 +161,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar(kBarQdoFull + s), 1);
             mbar_init(bar(kBarStageEmpty + s), 1);
-            mbar_init(bar(kBarInFull + s), 1);
-            mbar_init(bar(kBarReady + s), kSoftmaxThreads / 2);
-            mbar_init(bar(kBarDqFull + s), 1);
-            mbar_init(bar(kBarDqFree + s), 128);
+            mbar_init(bar(kBarSFull + s), 1);
+            mbar_init(bar(kBarDpFull + s), 1);
+            mbar_init(bar(kBarPReady + s), kSoftmaxThreads / 2);
+            mbar_init(bar(kBarDsReady + s), kSoftmaxThreads / 2);
         }
+        mbar_init(bar(kBarDqFull), 1);
+        mbar_init(bar(kBarDqFree), 128);
+        mbar_init(bar(kBarKvTmem), 256);
         mbar_init(bar(kBarSpdFull), p.spd_tma ? 1 : 32);
         mbar_init(bar(kBarSpdEmpty), 16);
         mbar_init(bar(kBarFinal), 1);
@@ -193,7 +199,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = misc[0];
-    constexpr uint32_t kColDv = 256, kColDk = 320, kColDq = 384;
+    constexpr uint32_t kColDv = 256, kColDk = 320, kColDq = 384, kColK = 448, kColV = 480;
 
     if (warp < 4) {
         setmaxnreg_dec_40();
@@ -230,67 +236,112 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             constexpr uint32_t idesc_ts = make_idesc_bf16(128, D, false, true);        // A in TMEM, B MN-major
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);         // A and B MN-major
             const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
-            const uint32_t sK = smem_u32(smem + L::kK), sV = smem_u32(smem + L::kV);
-            const uint64_t desc_k = make_smem_desc(sK, L::kRowBytes, 0), desc_v = make_smem_desc(sV, L::kRowBytes, 0);
+            const uint32_t sK = smem_u32(smem + L::kK);
+            const uint64_t desc_k = make_smem_desc(sK, L::kRowBytes, 0);
             // constant A operands of the extra K step: every 8-row group reads the same 256 bytes (group stride 0)
             const uint64_t desc_ones_s = make_smem_desc_stride(smem_u32(smem + L::kOnes), kExtCols * 2, 0, 0);
             const uint64_t desc_ones_dp = make_smem_desc_stride(smem_u32(smem + L::kOnes + 256), kExtCols * 2, 0, 0);
-            // S^T - lse sqrt(d) and dP^T - Delta of half `sub` of query tile i -> TMEM stage `sub`
-            auto issue_inputs = [&](int i, int sub) {
+            // S^T - lse sqrt(d)  /  dP^T - Delta  of half `sub` of query tile i -> TMEM stage `sub`
+            auto issue_s = [&](int i, int sub) {
                 const int s = i & 1;
                 const uint64_t dq_ = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
+                const uint64_t dext = make_smem_desc(smem_u32(smem + L::kExt + s * kExtTileBytes) + sub * kHalf * kExtCols * 2, kExtCols * 2, 0);
+                const uint32_t d_s = tm + sub * 128;
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks)     // A = K from tensor memory: 8 packed columns per K step
+                    mma_ts(d_s, tm + kColK + ks * 8, advance_desc(dq_, ks * 32), idesc_in, ks > 0);
+                mma_ss(d_s, desc_ones_s, dext, idesc_in, 1u);
+                mma_commit(bar(kBarSFull + sub));
+            };
+            auto issue_dp = [&](int i, int sub) {
+                const int s = i & 1;
                 const uint64_t ddo = make_smem_desc(smem_u32(smem + L::kDo + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
                 const uint64_t dext = make_smem_desc(smem_u32(smem + L::kExt + s * kExtTileBytes) + sub * kHalf * kExtCols * 2, kExtCols * 2, 0);
-                const uint32_t d_s = tm + sub * 128, d_dp = d_s + kHalf;
+                const uint32_t d_dp = tm + sub * 128 + kHalf;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ss(d_s, advance_desc(desc_k, ks * 32), advance_desc(dq_, ks * 32), idesc_in, ks > 0);
-                mma_ss(d_s, desc_ones_s, dext, idesc_in, 1u);
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ss(d_dp, advance_desc(desc_v, ks * 32), advance_desc(ddo, ks * 32), idesc_in, ks > 0);
+                    mma_ts(d_dp, tm + kColV + ks * 8, advance_desc(ddo, ks * 32), idesc_in, ks > 0);
                 mma_ss(d_dp, desc_ones_dp, dext, idesc_in, 1u);
-                mma_commit(bar(kBarInFull + sub));
+                mma_commit(bar(kBarDpFull + sub));
             };
             mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 120);
+            mbar_wait(bar(kBarKvTmem), 0, abort_flag, p.status, 124);
             mbar_wait(bar(kBarQdoFull + 0), 0, abort_flag, p.status, 121);
             tc_fence_after();
-            if (elect_one()) { issue_inputs(0, 0); issue_inputs(0, 1); }
+            if (elect_one()) { issue_s(0, 0); issue_s(0, 1); issue_dp(0, 0); issue_dp(0, 1); }
             __syncwarp();
-            for (int i = 0; i < n_q; ++i) {
-                const int s = i & 1;
+            // Event loop.  Per half the events come in a fixed order (P^T(i) stored, dS^T(i) stored, P^T(i+1), ...)
+            // but the two halves drift against each other, so the barriers are polled.  Every reuse of tensor
+            // memory is ordered by issue order: S^T(i+1) after dV(i) has read P^T(i), dP^T(i+1) after dK(i).
+            int ev[2] = {0, 0};                 // next event of each half: 2 i = P^T(i) stored, 2 i + 1 = dS^T(i) stored
+            int dq_next = 0;                    // next tile whose dQ is to be issued
+            bool dv_started = false, dk_started = false;   // the first MMA into an accumulator overwrites it
+            uint32_t idle = 0;
+            auto ready = [&](int b, uint32_t parity) { return __any_sync(0xffffffffu, mbar_test_wait(bar(b), parity)) != 0; };
+            while (dq_next < n_q) {
+                bool progressed = false;
 #pragma unroll
                 for (int sub = 0; sub < 2; ++sub) {
-                    if (sub == 0 && i + 1 < n_q)
-                        mbar_wait(bar(kBarQdoFull + (s ^ 1)), ((i + 1) >> 1) & 1, abort_flag, p.status, 122);
-                    if (sub == 1) mbar_wait(bar(kBarDqFree + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 125);
-                    mbar_wait(bar(kBarReady + sub), i & 1, abort_flag, p.status, 123);
-                    tc_fence_after();
-                    if (elect_one()) {
-                        const uint32_t t_p = tm + sub * 128, t_ds = t_p + kHalf;
-                        const uint64_t ddo = make_smem_desc(smem_u32(smem + L::kDo + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
-                        const uint64_t dq_ = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
+                    const int e = ev[sub], i = e >> 1, s = i & 1;
+                    if (e >= 2 * n_q) continue;
+                    if ((e & 1) == 0) {
+                        if (!ready(kBarPReady + sub, i & 1)) continue;
+                        if (i + 1 < n_q && !ready(kBarQdoFull + (s ^ 1), ((i + 1) >> 1) & 1)) continue;
+                        tc_fence_after();
+                        if (elect_one()) {
+                            const uint32_t t_p = tm + sub * 128;
+                            const uint64_t ddo = make_smem_desc(smem_u32(smem + L::kDo + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
 #pragma unroll
-                        for (int ks = 0; ks < kHalf / 16; ++ks)     // dV += P^T dO   (P^T of query group ks/2 at the start of its 32 columns)
-                            mma_ts(tm + kColDv, t_p + (ks >> 1) * 32 + (ks & 1) * 8,
-                                   advance_desc(ddo, ks * 16 * L::kRowBytes), idesc_ts, (i > 0 || sub > 0 || ks > 0) ? 1u : 0u);
-#pragma unroll
-                        for (int ks = 0; ks < kHalf / 16; ++ks)     // dK += dS^T Q
-                            mma_ts(tm + kColDk, t_ds + (ks >> 1) * 32 + (ks & 1) * 8,
-                                   advance_desc(dq_, ks * 16 * L::kRowBytes), idesc_ts, (i > 0 || sub > 0 || ks > 0) ? 1u : 0u);
-                        if (sub == 1) mma_commit(bar(kBarStageEmpty + s));   // Q_i, dO_i and their per-query rows are dead
-                        if (i + 1 < n_q) issue_inputs(i + 1, sub);   // over P^T / dS^T just consumed (MMAs run in issue order)
-                        if (sub == 1) {                              // dQ_i = dS K
-                            const uint64_t da = make_smem_desc(smem_u32(smem + L::kDs), 128, 16384);
-#pragma unroll
-                            for (int ks = 0; ks < 8; ++ks)
-                                mma_ss(tm + kColDq + s * 64, advance_desc(da, ks * 2048),
-                                       advance_desc(desc_k, ks * 16 * L::kRowBytes), idesc_dq, ks > 0);
-                            mma_commit(bar(kBarDqFull + s));
-                            if (i + 1 == n_q) mma_commit(bar(kBarFinal));
+                            for (int ks = 0; ks < kHalf / 16; ++ks)     // dV += P^T dO   (P^T of query group ks/2 at the start of its 32 columns)
+                                mma_ts(tm + kColDv, t_p + (ks >> 1) * 32 + (ks & 1) * 8,
+                                       advance_desc(ddo, ks * 16 * L::kRowBytes), idesc_ts, (dv_started || ks > 0) ? 1u : 0u);
+                            if (i + 1 < n_q) issue_s(i + 1, sub);
                         }
+                        __syncwarp();
+                        dv_started = true;
+                    } else {
+                        if (!ready(kBarDsReady + sub, i & 1)) continue;
+                        tc_fence_after();
+                        if (elect_one()) {
+                            const uint32_t t_ds = tm + sub * 128 + kHalf;
+                            const uint64_t dq_ = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
+#pragma unroll
+                            for (int ks = 0; ks < kHalf / 16; ++ks)     // dK += dS^T Q
+                                mma_ts(tm + kColDk, t_ds + (ks >> 1) * 32 + (ks & 1) * 8,
+                                       advance_desc(dq_, ks * 16 * L::kRowBytes), idesc_ts, (dk_started || ks > 0) ? 1u : 0u);
+                            if (i + 1 < n_q) issue_dp(i + 1, sub);
+                        }
+                        __syncwarp();
+                        dk_started = true;
+                    }
+                    ev[sub] = e + 1;
+                    progressed = true;
+                }
+                // dQ_i = dS K once both halves have stored dS^T(i) and the reducer has drained dQ_{i-1}
+                if (ev[0] >= 2 * dq_next + 2 && ev[1] >= 2 * dq_next + 2 && ready(kBarDqFree, (dq_next & 1) ^ 1)) {
+                    const int i = dq_next;
+                    if (elect_one()) {
+                        mma_commit(bar(kBarStageEmpty + (i & 1)));      // Q_i, dO_i and their per-query rows are dead
+                        const uint64_t da = make_smem_desc(smem_u32(smem + L::kDs), 128, 16384);
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks)
+                            mma_ss(tm + kColDq, advance_desc(da, ks * 2048),
+                                   advance_desc(desc_k, ks * 16 * L::kRowBytes), idesc_dq, ks > 0);
+                        mma_commit(bar(kBarDqFull));
+                        if (i + 1 == n_q) mma_commit(bar(kBarFinal));
                     }
                     __syncwarp();
+                    ++dq_next;
+                    progressed = true;
+                }
+                if (progressed) {
+                    idle = 0;
+                } else if (++idle > kWaitIterations || ((idle & 255u) == 255u && *abort_flag)) {
+                    if (!*abort_flag) {
+                        *abort_flag = 1u;
+                        if (lane == 0 && atomicCAS(p.status, 0u, 5u /* GT_ERR_DEVICE_TIMEOUT */) == 0u) p.status[1] = 126;
+                    }
+                    break;
                 }
             }
         } else if (warp == 2 && !p.spd_tma) {
@@ -331,16 +382,34 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const uint32_t bins_base = smem_u32(my_bins);
         uint8_t* ds_row = smem + L::kDs + half * 16384 + r * 128;
 
+        // K (warps 4-7) and V (warps 8-11) rows -> tensor memory, where they stay as the A operands of
+        // S^T = K Q^T and dP^T = V dO^T: one shared-memory read instead of one per query half tile
+        if (warp < 12) {
+            mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 144);
+            const uint8_t* src = smem + (warp < 8 ? L::kK : L::kV) + r * L::kRowBytes;
+            uint32_t w[D / 2];
+#pragma unroll
+            for (int c = 0; c < D / 8; ++c) {
+                const int phys = D == 64 ? (c ^ (r & 7)) : (c ^ ((r >> 1) & 3));     // 128-byte / 64-byte swizzle
+                const uint4 v4 = *(const uint4*)(src + (phys << 4));
+                w[4 * c] = v4.x; w[4 * c + 1] = v4.y; w[4 * c + 2] = v4.z; w[4 * c + 3] = v4.w;
+            }
+            const uint32_t dst = tmem + (warp < 8 ? kColK : kColV) + lane_off;
+            if constexpr (D == 64) tmem_st32(dst, w); else tmem_st16(dst, w);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar(kBarKvTmem));
+        }
+
         for (int i = 0; i < n_q; ++i) {
             const int s = i & 1;
             float pr[32];
             uint32_t dpa[16], dpb[16];
-            mbar_wait(bar(kBarInFull + half), i & 1, abort_flag, p.status, 140);
+            mbar_wait(bar(kBarSFull + half), i & 1, abort_flag, p.status, 140);
             tc_fence_after();
             {
                 uint32_t sv[32];
                 tmem_ld32(tS, sv);
-                tmem_ld16(tDp, dpa);
                 mbar_wait(bar(kBarSpdFull), i & 1, abort_flag, p.status, 141);
                 tmem_wait_ld();
 #pragma unroll
@@ -383,7 +452,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 for (int c = 0; c < 16; ++c) pk[c] = pack_bf16x2(pr[2 * c], pr[2 * c + 1]);
                 tmem_st16(tS, pk);                      // P^T of this group: 16 packed columns at the start of its range
             }
+            mbar_wait(bar(kBarDpFull + half), i & 1, abort_flag, p.status, 145);
+            tc_fence_after();
+            tmem_ld16(tDp, dpa);
             tmem_ld16(tDp + 16, dpb);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar(kBarPReady + half));    // dV of this half and the next S^T can go
+            tmem_wait_ld();
 
             // ---------------- dS^T = P^T o (dP^T - Delta), bias-gradient bins ----------------
             auto ds_round = [&](int rnd, const uint32_t (&dp)[16]) {
@@ -392,25 +468,33 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     const int c = rnd * 16 + k;
                     unpack_f32x2(mul_f32x2(pack_f32x2(pr[c], pr[c + 1]), pack_u32x2(dp[k], dp[k + 1])), pr[c], pr[c + 1]);
                 }
-#pragma unroll
-                for (int k = 0; k < 16; ++k) {
-                    const int c = rnd * 16 + k;
-                    // byte offset of bin b: b * stride * 4, formed by one funnel shift and one mask
-                    constexpr int kLog = kPrivateBins ? 11 : 7;               // log2(kBinStride * 4)
+                // byte offset of bin b: b * stride * 4, formed by one funnel shift and one mask
+                constexpr int kLog = kPrivateBins ? 11 : 7;               // log2(kBinStride * 4)
+                auto bin_off = [&](int c) {
                     const int sh = 8 * (c & 3) - kLog;
-                    const uint32_t off = (sh >= 0 ? (bw[c >> 2] >> (sh >= 0 ? sh : 0)) : (bw[c >> 2] << (sh < 0 ? -sh : 0))) & (0xffu << kLog);
-                    if (kPrivateBins) {
-                        float v;
-                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(bins_base + off));
-                        v += pr[c];
-                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(bins_base + off), "f"(v));
-                    } else {
-                        atomicAdd((float*)((uint8_t*)my_bins + off), pr[c]);
+                    return (sh >= 0 ? (bw[c >> 2] >> (sh >= 0 ? sh : 0)) : (bw[c >> 2] << (sh < 0 ? -sh : 0))) & (0xffu << kLog);
+                };
+                if (kPrivateBins) {
+                    // read-modify-write of the thread's own bins, two elements at a time so that two loads are
+                    // in flight; when both hit the same bin the second add takes the first one's result
+#pragma unroll
+                    for (int k = 0; k < 16; k += 2) {
+                        const int c = rnd * 16 + k;
+                        const uint32_t o0 = bin_off(c), o1 = bin_off(c + 1);
+                        float v0, v1;
+                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v0) : "r"(bins_base + o0));
+                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v1) : "r"(bins_base + o1));
+                        v0 += pr[c];
+                        v1 = (o1 == o0 ? v0 : v1) + pr[c + 1];
+                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(bins_base + o0), "f"(v0));
+                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(bins_base + o1), "f"(v1));
                     }
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) atomicAdd((float*)((uint8_t*)my_bins + bin_off(rnd * 16 + k)), pr[rnd * 16 + k]);
                 }
             };
             ds_round(0, dpa);
-            tmem_wait_ld();
             ds_round(1, dpb);
             {
                 uint32_t pk[16];
@@ -418,7 +502,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 for (int c = 0; c < 16; ++c) pk[c] = pack_bf16x2(pr[2 * c], pr[2 * c + 1]);
                 tmem_st16(tDp, pk);
                 // dQ of the previous tile has read the dS^T tile in shared memory
-                if (i > 0) mbar_wait(bar(kBarDqFull + (s ^ 1)), ((i - 1) >> 1) & 1, abort_flag, p.status, 142);
+                if (i > 0) mbar_wait(bar(kBarDqFull), (i - 1) & 1, abort_flag, p.status, 142);
 #pragma unroll
                 for (int c8 = 0; c8 < 4; ++c8)
                     *(uint4*)(ds_row + ((((grp & 1) * 4 + c8) ^ (r & 7)) << 4)) =
@@ -427,7 +511,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             }
             fence_proxy_async_smem();
             tc_fence_before();
-            mbar_arrive(bar(kBarReady + half));
+            mbar_arrive(bar(kBarDsReady + half));
         }
 
         // ---------------- epilogue: dV (first half's warps) and dK (second half's) ----------------
@@ -481,14 +565,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         uint8_t* row = smem + L::kStg + r * 128;
         for (int i = 0; i < n_q; ++i) {
             const int s = i & 1;
-            mbar_wait(bar(kBarDqFull + s), (i >> 1) & 1, abort_flag, p.status, 150);
+            mbar_wait(bar(kBarDqFull), i & 1, abort_flag, p.status, 150);
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t o[32];
-                tmem_ld32(tmem + kColDq + s * 64 + c * 32 + lane_off, o);
+                tmem_ld32(tmem + kColDq + c * 32 + lane_off, o);
                 tmem_wait_ld();
-                if (c == D / 32 - 1) { tc_fence_before(); mbar_arrive(bar(kBarDqFree + s)); }
+                if (c == D / 32 - 1) { tc_fence_before(); mbar_arrive(bar(kBarDqFree)); }
                 if (warp == 20 && elect_one()) bulk_wait_group_read0();      // the previous reduce has read the staging buffer
                 named_barrier_sync(kNbDqStagingFree, 128);
 #pragma unroll

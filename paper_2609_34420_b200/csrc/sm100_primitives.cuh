@@ -47,6 +47,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
+// non-blocking test (try_wait may suspend the thread for a while; a poller of several barriers must not)
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+
 // Bounded wait.  `abort_flag` (shared memory) is set by the first wait of the CTA that runs
 // out; once it is set every later wait returns at once, so a CTA that lost a signal drains
 // in bounded time instead of hanging.  Returns false if the wait was abandoned.
