@@ -19,8 +19,9 @@
 // barriers; eight softmax warps own each half.  While one half's MMAs (dV, dK, next S^T, next
 // dP^T) run, the other half's warps compute, and no softmax thread ever waits at a CTA-wide
 // barrier: it arrives on an mbarrier when its P^T / dS^T are stored and only waits for its own
-// next inputs.  All MMAs are issued by one thread, in an order that makes every TMEM reuse
-// (next S^T over P^T, next dP^T over dS^T) follow the MMA that reads the old contents.
+// next inputs.  Three helper warps issue the MMAs; each accumulator and each part of a TMEM stage
+// belongs to one of them, so that every TMEM reuse (next S^T over P^T, next dP^T over dS^T) follows,
+// in that thread's issue order, the MMA that reads the old contents.
 //
 // Because the scores are transposed, a thread walks along QUERY indices for a fixed key, i.e.
 // down a column of the SPD matrix.  A pre-pass therefore writes a transposed copy of the SPD
@@ -29,8 +30,8 @@
 //
 //   warp 0        TMA producer: K, V, the constant tiles once; Q_i, dO_i, the per-query rows and
 //                 (single graph) the SPD^T tile through a 2-stage ring
-//   warp 1        MMA issuer
-//   warp 2        SPD^T tile loader for packed batches (per-graph pitch: cp.async)
+//                 (packed batches: the SPD^T tile by cp.async, per-graph pitch)
+//   warps 1, 3, 2 MMA issuers: dV and the next S^T; dK and the next dP^T; dQ
 //   warps 4-19    softmax: warps 4-11 own queries [0,64) of every tile, warps 12-19 queries [64,128);
 //                 within a half, four warps per 32 query columns (32 score elements per thread)
 //   warps 20-23   dQ reducer: TMEM -> shared memory -> TMA reduce-add into the fp32 accumulator
@@ -160,7 +161,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         mbar_init(bar(kBarKvFull), 1);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar(kBarQdoFull + s), 1);
-            mbar_init(bar(kBarStageEmpty + s), 1);
+            mbar_init(bar(kBarStageEmpty + s), 2);
             mbar_init(bar(kBarSFull + s), 1);
             mbar_init(bar(kBarDpFull + s), 1);
             mbar_init(bar(kBarPReady + s), kSoftmaxThreads / 2);
@@ -171,7 +172,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         mbar_init(bar(kBarKvTmem), 256);
         mbar_init(bar(kBarSpdFull), p.spd_tma ? 1 : 32);
         mbar_init(bar(kBarSpdEmpty), 16);
-        mbar_init(bar(kBarFinal), 1);
+        mbar_init(bar(kBarFinal), 3);
         fence_mbar_init();
         prefetch_tensormap(&tmap_q);
         prefetch_tensormap(&tmap_k);
@@ -221,117 +222,98 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     tma_load_3d(smem_u32(smem + L::kExt + s * kExtTileBytes), &tmap_ext, bar(kBarQdoFull + s), 0, h, row);
                 }
                 __syncwarp();
+                if (i > 0) mbar_wait(bar(kBarSpdEmpty), (i - 1) & 1, abort_flag, p.status, 111);
                 if (p.spd_tma) {
-                    if (i > 0) mbar_wait(bar(kBarSpdEmpty), (i - 1) & 1, abort_flag, p.status, 111);
                     if (lane == 0) {
                         mbar_arrive_expect_tx(bar(kBarSpdFull), L::kSpdBytes);
                         tma_load_2d(smem_u32(smem + L::kSpd), &tmap_spd, bar(kBarSpdFull), i * kTile, kv0);
                     }
                     __syncwarp();
+                } else {
+                    // packed batch (per-graph pitch): cp.async in the layout of the TMA 128-byte swizzle,
+                    // 16-byte chunk c of row r at chunk c ^ (r & 7)
+                    const int32_t q0 = i * kTile;
+                    const uint32_t dst0 = smem_u32(smem + L::kSpd);
+#pragma unroll 4
+                    for (int it = 0; it < (kTile * 8) / 32; ++it) {
+                        const int c = it * 32 + lane;
+                        const int r = c >> 3, cc = c & 7;
+                        const int64_t col = (int64_t)q0 + cc * 16;
+                        const bool valid = (kv0 + r < n_g) && (col < ld);
+                        const uint8_t* src = valid ? spd_g + (int64_t)(kv0 + r) * ld + col : spd_g;
+                        cp_async_16(dst0 + r * 128 + ((cc ^ (r & 7)) << 4), src, valid ? 16u : 0u);
+                    }
+                    cp_async_mbar_arrive_noinc(bar(kBarSpdFull));
                 }
             }
-        } else if (warp == 1) {
-            // ------------------------------- MMA issuer -------------------------------
+        } else if (warp == 1 || warp == 3) {
+            // ------------------------------- MMA issuers -------------------------------
+            // warp 1: on "P^T(i) of a half stored": dV += P^T dO_i, then S^T of the next tile over the P^T just read
+            // warp 3: on "dS^T(i) of a half stored": dK += dS^T Q_i, then dP^T of the next tile over that dS^T
+            // Each accumulator and each TMEM stage region is touched by one issuing thread only, so every reuse
+            // is ordered by that thread's issue order.  (One issuer for everything spends most of the tile
+            // issuing: a helper warp gets few issue slots next to four busy softmax warps.)
+            const bool on_p = warp == 1;
             constexpr uint32_t idesc_in = make_idesc_bf16(128, kHalf, false, false);   // S^T, dP^T of 64 queries
             constexpr uint32_t idesc_ts = make_idesc_bf16(128, D, false, true);        // A in TMEM, B MN-major
-            constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);         // A and B MN-major
             const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
-            const uint32_t sK = smem_u32(smem + L::kK);
-            const uint64_t desc_k = make_smem_desc(sK, L::kRowBytes, 0);
-            // constant A operands of the extra K step: every 8-row group reads the same 256 bytes (group stride 0)
-            const uint64_t desc_ones_s = make_smem_desc_stride(smem_u32(smem + L::kOnes), kExtCols * 2, 0, 0);
-            const uint64_t desc_ones_dp = make_smem_desc_stride(smem_u32(smem + L::kOnes + 256), kExtCols * 2, 0, 0);
-            // S^T - lse sqrt(d)  /  dP^T - Delta  of half `sub` of query tile i -> TMEM stage `sub`
-            auto issue_s = [&](int i, int sub) {
+            // constant A operand of the extra K step: every 8-row group reads the same 256 bytes (group stride 0)
+            const uint64_t desc_ones = make_smem_desc_stride(smem_u32(smem + L::kOnes + (on_p ? 0 : 256)), kExtCols * 2, 0, 0);
+            const int acc_b_off = on_p ? L::kDo : L::kQ;       // B of the accumulating MMA: dO_i (dV) / Q_i (dK)
+            const int in_b_off = on_p ? L::kQ : L::kDo;        // B of the next input MMA:   Q (S^T)  / dO (dP^T)
+            const uint32_t acc_col = on_p ? kColDv : kColDk;
+            const uint32_t reg_off = on_p ? 0 : kHalf;          // S^T/P^T or dP^T/dS^T part of a TMEM stage
+            const uint32_t in_a_col = on_p ? kColK : kColV;
+            const int bar_ready = on_p ? kBarPReady : kBarDsReady, bar_full = on_p ? kBarSFull : kBarDpFull;
+            auto issue_input = [&](int i, int sub) {            // (S^T - lse sqrt(d)) or (dP^T - Delta) of a half tile
                 const int s = i & 1;
-                const uint64_t dq_ = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
+                const uint64_t db = make_smem_desc(smem_u32(smem + in_b_off + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
                 const uint64_t dext = make_smem_desc(smem_u32(smem + L::kExt + s * kExtTileBytes) + sub * kHalf * kExtCols * 2, kExtCols * 2, 0);
-                const uint32_t d_s = tm + sub * 128;
+                const uint32_t d = tm + sub * 128 + reg_off;
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)     // A = K from tensor memory: 8 packed columns per K step
-                    mma_ts(d_s, tm + kColK + ks * 8, advance_desc(dq_, ks * 32), idesc_in, ks > 0);
-                mma_ss(d_s, desc_ones_s, dext, idesc_in, 1u);
-                mma_commit(bar(kBarSFull + sub));
+                for (int ks = 0; ks < D / 16; ++ks)             // A = K or V from tensor memory: 8 packed columns per K step
+                    mma_ts(d, tm + in_a_col + ks * 8, advance_desc(db, ks * 32), idesc_in, ks > 0);
+                mma_ss(d, desc_ones, dext, idesc_in, 1u);
+                mma_commit(bar(bar_full + sub));
             };
-            auto issue_dp = [&](int i, int sub) {
-                const int s = i & 1;
-                const uint64_t ddo = make_smem_desc(smem_u32(smem + L::kDo + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
-                const uint64_t dext = make_smem_desc(smem_u32(smem + L::kExt + s * kExtTileBytes) + sub * kHalf * kExtCols * 2, kExtCols * 2, 0);
-                const uint32_t d_dp = tm + sub * 128 + kHalf;
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ts(d_dp, tm + kColV + ks * 8, advance_desc(ddo, ks * 32), idesc_in, ks > 0);
-                mma_ss(d_dp, desc_ones_dp, dext, idesc_in, 1u);
-                mma_commit(bar(kBarDpFull + sub));
-            };
-            mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 120);
             mbar_wait(bar(kBarKvTmem), 0, abort_flag, p.status, 124);
             mbar_wait(bar(kBarQdoFull + 0), 0, abort_flag, p.status, 121);
             tc_fence_after();
-            if (elect_one()) { issue_s(0, 0); issue_s(0, 1); issue_dp(0, 0); issue_dp(0, 1); }
+            if (elect_one()) { issue_input(0, 0); issue_input(0, 1); }
             __syncwarp();
-            // Event loop.  Per half the events come in a fixed order (P^T(i) stored, dS^T(i) stored, P^T(i+1), ...)
-            // but the two halves drift against each other, so the barriers are polled.  Every reuse of tensor
-            // memory is ordered by issue order: S^T(i+1) after dV(i) has read P^T(i), dP^T(i+1) after dK(i).
-            int ev[2] = {0, 0};                 // next event of each half: 2 i = P^T(i) stored, 2 i + 1 = dS^T(i) stored
-            int dq_next = 0;                    // next tile whose dQ is to be issued
-            bool dv_started = false, dk_started = false;   // the first MMA into an accumulator overwrites it
+            // The two halves drift against each other, so their barriers are polled.
+            int next_tile[2] = {0, 0};
+            int done_tiles = 0;                 // tiles with both halves handled
+            bool acc_started = false;           // the first MMA into the accumulator overwrites it
             uint32_t idle = 0;
             auto ready = [&](int b, uint32_t parity) { return __any_sync(0xffffffffu, mbar_test_wait(bar(b), parity)) != 0; };
-            while (dq_next < n_q) {
+            while (done_tiles < n_q) {
                 bool progressed = false;
 #pragma unroll
                 for (int sub = 0; sub < 2; ++sub) {
-                    const int e = ev[sub], i = e >> 1, s = i & 1;
-                    if (e >= 2 * n_q) continue;
-                    if ((e & 1) == 0) {
-                        if (!ready(kBarPReady + sub, i & 1)) continue;
-                        if (i + 1 < n_q && !ready(kBarQdoFull + (s ^ 1), ((i + 1) >> 1) & 1)) continue;
-                        tc_fence_after();
-                        if (elect_one()) {
-                            const uint32_t t_p = tm + sub * 128;
-                            const uint64_t ddo = make_smem_desc(smem_u32(smem + L::kDo + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
-#pragma unroll
-                            for (int ks = 0; ks < kHalf / 16; ++ks)     // dV += P^T dO   (P^T of query group ks/2 at the start of its 32 columns)
-                                mma_ts(tm + kColDv, t_p + (ks >> 1) * 32 + (ks & 1) * 8,
-                                       advance_desc(ddo, ks * 16 * L::kRowBytes), idesc_ts, (dv_started || ks > 0) ? 1u : 0u);
-                            if (i + 1 < n_q) issue_s(i + 1, sub);
-                        }
-                        __syncwarp();
-                        dv_started = true;
-                    } else {
-                        if (!ready(kBarDsReady + sub, i & 1)) continue;
-                        tc_fence_after();
-                        if (elect_one()) {
-                            const uint32_t t_ds = tm + sub * 128 + kHalf;
-                            const uint64_t dq_ = make_smem_desc(smem_u32(smem + L::kQ + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
-#pragma unroll
-                            for (int ks = 0; ks < kHalf / 16; ++ks)     // dK += dS^T Q
-                                mma_ts(tm + kColDk, t_ds + (ks >> 1) * 32 + (ks & 1) * 8,
-                                       advance_desc(dq_, ks * 16 * L::kRowBytes), idesc_ts, (dk_started || ks > 0) ? 1u : 0u);
-                            if (i + 1 < n_q) issue_dp(i + 1, sub);
-                        }
-                        __syncwarp();
-                        dk_started = true;
-                    }
-                    ev[sub] = e + 1;
-                    progressed = true;
-                }
-                // dQ_i = dS K once both halves have stored dS^T(i) and the reducer has drained dQ_{i-1}
-                if (ev[0] >= 2 * dq_next + 2 && ev[1] >= 2 * dq_next + 2 && ready(kBarDqFree, (dq_next & 1) ^ 1)) {
-                    const int i = dq_next;
+                    const int i = next_tile[sub], s = i & 1;
+                    if (i >= n_q) continue;
+                    if (!ready(bar_ready + sub, i & 1)) continue;
+                    if (i + 1 < n_q && !ready(kBarQdoFull + (s ^ 1), ((i + 1) >> 1) & 1)) continue;
+                    tc_fence_after();
+                    const bool tile_done = next_tile[sub ^ 1] > i;
                     if (elect_one()) {
-                        mma_commit(bar(kBarStageEmpty + (i & 1)));      // Q_i, dO_i and their per-query rows are dead
-                        const uint64_t da = make_smem_desc(smem_u32(smem + L::kDs), 128, 16384);
+                        const uint32_t t_a = tm + sub * 128 + reg_off;
+                        const uint64_t db = make_smem_desc(smem_u32(smem + acc_b_off + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
 #pragma unroll
-                        for (int ks = 0; ks < 8; ++ks)
-                            mma_ss(tm + kColDq, advance_desc(da, ks * 2048),
-                                   advance_desc(desc_k, ks * 16 * L::kRowBytes), idesc_dq, ks > 0);
-                        mma_commit(bar(kBarDqFull));
-                        if (i + 1 == n_q) mma_commit(bar(kBarFinal));
+                        for (int ks = 0; ks < kHalf / 16; ++ks)     // A: bf16 pairs of query group ks/2 at the start of its 32 columns
+                            mma_ts(tm + acc_col, t_a + (ks >> 1) * 32 + (ks & 1) * 8,
+                                   advance_desc(db, ks * 16 * L::kRowBytes), idesc_ts, (acc_started || ks > 0) ? 1u : 0u);
+                        if (tile_done) {
+                            mma_commit(bar(kBarStageEmpty + s));    // this issuer's reads of Q_i / dO_i are done (the other one commits too)
+                            if (i + 1 == n_q) mma_commit(bar(kBarFinal));
+                        }
+                        if (i + 1 < n_q) issue_input(i + 1, sub);
                     }
                     __syncwarp();
-                    ++dq_next;
+                    acc_started = true;
+                    next_tile[sub] = i + 1;
+                    if (tile_done) ++done_tiles;
                     progressed = true;
                 }
                 if (progressed) {
@@ -344,23 +326,27 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     break;
                 }
             }
-        } else if (warp == 2 && !p.spd_tma) {
-            // --------------------- SPD^T tile loader for packed batches ---------------------
+        } else if (warp == 2) {
+            // ------------------------------- dQ issuer -------------------------------
+            constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);         // A and B MN-major
+            const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+            const uint64_t desc_k = make_smem_desc(smem_u32(smem + L::kK), L::kRowBytes, 0);
+            const uint64_t da = make_smem_desc(smem_u32(smem + L::kDs), 128, 16384);
+            mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 120);
             for (int i = 0; i < n_q; ++i) {
-                if (i > 0) mbar_wait(bar(kBarSpdEmpty), (i - 1) & 1, abort_flag, p.status, 130);
-                const int32_t q0 = i * kTile;
-                // same layout as the TMA 128-byte swizzle: 16-byte chunk c of row r at chunk c ^ (r & 7)
-                const uint32_t dst0 = smem_u32(smem + L::kSpd);
-#pragma unroll 4
-                for (int it = 0; it < (kTile * 8) / 32; ++it) {
-                    const int c = it * 32 + lane;
-                    const int r = c >> 3, cc = c & 7;
-                    const int64_t col = (int64_t)q0 + cc * 16;
-                    const bool valid = (kv0 + r < n_g) && (col < ld);
-                    const uint8_t* src = valid ? spd_g + (int64_t)(kv0 + r) * ld + col : spd_g;
-                    cp_async_16(dst0 + r * 128 + ((cc ^ (r & 7)) << 4), src, valid ? 16u : 0u);
+                // dQ_i = dS K once both halves have stored dS^T(i) and the reducer has drained dQ_{i-1}
+                mbar_wait(bar(kBarDsReady + 0), i & 1, abort_flag, p.status, 127);
+                mbar_wait(bar(kBarDsReady + 1), i & 1, abort_flag, p.status, 128);
+                mbar_wait(bar(kBarDqFree), (i & 1) ^ 1, abort_flag, p.status, 125);
+                tc_fence_after();
+                if (elect_one()) {
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks)
+                        mma_ss(tm + kColDq, advance_desc(da, ks * 2048), advance_desc(desc_k, ks * 16 * L::kRowBytes), idesc_dq, ks > 0);
+                    mma_commit(bar(kBarDqFull));
+                    if (i + 1 == n_q) mma_commit(bar(kBarFinal));
                 }
-                cp_async_mbar_arrive_noinc(bar(kBarSpdFull));
+                __syncwarp();
             }
         }
     } else if (warp < 20) {
