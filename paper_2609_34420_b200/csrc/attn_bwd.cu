@@ -544,23 +544,29 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         // ================================ dQ reducer ================================
         // dQ_i (fp32, 128 x D) goes TMEM -> registers -> a staging buffer in 128-byte-swizzled rows of
         // 32 floats, and from there to the global fp32 accumulator with TMA reduce-add: full lines
-        // to L2 instead of 16-byte scattered atomics.
+        // to L2 instead of 16-byte scattered atomics.  The reduce engine of an SM moves about 19 bytes
+        // per clock, so it has to run all the time: with d = 64 two staging buffers alternate (the second
+        // one is the V tile, dead once V sits in tensor memory) and a buffer is only waited for when it
+        // comes round again.
         setmaxnreg_dec_48();
         const int r = ((warp & 3) << 5) | lane;
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-        uint8_t* row = smem + L::kStg + r * 128;
+        constexpr int kStgBufs = D == 64 ? 2 : 1;
         for (int i = 0; i < n_q; ++i) {
-            const int s = i & 1;
             mbar_wait(bar(kBarDqFull), i & 1, abort_flag, p.status, 150);
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
+                uint8_t* stg = smem + ((kStgBufs == 2 && c == 1) ? L::kV : L::kStg);
                 uint32_t o[32];
                 tmem_ld32(tmem + kColDq + c * 32 + lane_off, o);
                 tmem_wait_ld();
                 if (c == D / 32 - 1) { tc_fence_before(); mbar_arrive(bar(kBarDqFree)); }
-                if (warp == 20 && elect_one()) bulk_wait_group_read0();      // the previous reduce has read the staging buffer
+                if (warp == 20 && elect_one()) {        // the reduce that last used this buffer has read it
+                    if (kStgBufs == 2) bulk_wait_group_read1(); else bulk_wait_group_read0();
+                }
                 named_barrier_sync(kNbDqStagingFree, 128);
+                uint8_t* row = stg + r * 128;
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
                     *(uint4*)(row + ((k ^ (r & 7)) << 4)) = make_uint4(o[4 * k], o[4 * k + 1], o[4 * k + 2], o[4 * k + 3]);
@@ -568,7 +574,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 named_barrier_sync(kNbDqStaged, 128);
                 if (warp == 20) {
                     if (elect_one()) {
-                        tma_reduce_add_2d(&tmap_dq, smem_u32(smem + L::kStg), h * D + c * 32, node0 + i * kTile);
+                        tma_reduce_add_2d(&tmap_dq, smem_u32(stg), h * D + c * 32, node0 + i * kTile);
                         bulk_commit_group();
                     }
                     __syncwarp();
