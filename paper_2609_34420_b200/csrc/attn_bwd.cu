@@ -388,7 +388,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
 
         for (int i = 0; i < n_q; ++i) {
-            const int s = i & 1;
             float pr[32];
             uint32_t dpa[16], dpb[16];
             mbar_wait(bar(kBarSFull + half), i & 1, abort_flag, p.status, 140);
