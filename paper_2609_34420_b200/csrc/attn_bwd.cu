@@ -281,22 +281,16 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             tc_fence_after();
             if (elect_one()) { issue_input(0, 0); issue_input(0, 1); }
             __syncwarp();
-            // The two halves drift against each other, so their barriers are polled.
-            int next_tile[2] = {0, 0};
-            int done_tiles = 0;                 // tiles with both halves handled
+            // The halves are served in turn with blocking waits (the hardware suspends a waiting thread; polling
+            // the barriers of both halves instead costs shared-memory wavefronts the softmax warps need).
             bool acc_started = false;           // the first MMA into the accumulator overwrites it
-            uint32_t idle = 0;
-            auto ready = [&](int b, uint32_t parity) { return __any_sync(0xffffffffu, mbar_test_wait(bar(b), parity)) != 0; };
-            while (done_tiles < n_q) {
-                bool progressed = false;
+            for (int i = 0; i < n_q; ++i) {
+                const int s = i & 1;
+                if (i + 1 < n_q) mbar_wait(bar(kBarQdoFull + (s ^ 1)), ((i + 1) >> 1) & 1, abort_flag, p.status, 122);
 #pragma unroll
                 for (int sub = 0; sub < 2; ++sub) {
-                    const int i = next_tile[sub], s = i & 1;
-                    if (i >= n_q) continue;
-                    if (!ready(bar_ready + sub, i & 1)) continue;
-                    if (i + 1 < n_q && !ready(kBarQdoFull + (s ^ 1), ((i + 1) >> 1) & 1)) continue;
+                    mbar_wait(bar(bar_ready + sub), i & 1, abort_flag, p.status, 123);
                     tc_fence_after();
-                    const bool tile_done = next_tile[sub ^ 1] > i;
                     if (elect_one()) {
                         const uint32_t t_a = tm + sub * 128 + reg_off;
                         const uint64_t db = make_smem_desc(smem_u32(smem + acc_b_off + s * L::kStageBytes) + sub * kHalf * L::kRowBytes, L::kRowBytes, 0);
@@ -304,7 +298,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         for (int ks = 0; ks < kHalf / 16; ++ks)     // A: bf16 pairs of query group ks/2 at the start of its 32 columns
                             mma_ts(tm + acc_col, t_a + (ks >> 1) * 32 + (ks & 1) * 8,
                                    advance_desc(db, ks * 16 * L::kRowBytes), idesc_ts, (acc_started || ks > 0) ? 1u : 0u);
-                        if (tile_done) {
+                        if (sub == 1) {
                             mma_commit(bar(kBarStageEmpty + s));    // this issuer's reads of Q_i / dO_i are done (the other one commits too)
                             if (i + 1 == n_q) mma_commit(bar(kBarFinal));
                         }
@@ -312,18 +306,6 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     }
                     __syncwarp();
                     acc_started = true;
-                    next_tile[sub] = i + 1;
-                    if (tile_done) ++done_tiles;
-                    progressed = true;
-                }
-                if (progressed) {
-                    idle = 0;
-                } else if (++idle > kWaitIterations || ((idle & 255u) == 255u && *abort_flag)) {
-                    if (!*abort_flag) {
-                        *abort_flag = 1u;
-                        if (lane == 0 && atomicCAS(p.status, 0u, 5u /* GT_ERR_DEVICE_TIMEOUT */) == 0u) p.status[1] = 126;
-                    }
-                    break;
                 }
             }
         } else if (warp == 2) {
