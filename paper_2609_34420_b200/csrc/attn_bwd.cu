@@ -84,11 +84,11 @@ enum BwdBarrier {
     kBarStageEmpty,                          // [2]  commit behind the last MMA that reads Q_i / dO_i
     kBarSFull = kBarStageEmpty + kStages,    // [2]  per half: S^T of the next tile is in tensor memory
     kBarDpFull = kBarSFull + 2,              // [2]  per half: dP^T of the next tile
-    kBarPReady = kBarDpFull + 2,             // [2]  per half: 256 arrivals, P^T stored
-    kBarDsReady = kBarPReady + 2,            // [2]  per half: 256 arrivals, dS^T stored (tensor and shared memory)
+    kBarPReady = kBarDpFull + 2,             // [2]  per half: 8 warp arrivals, P^T stored
+    kBarDsReady = kBarPReady + 2,            // [2]  per half: 8 warp arrivals, dS^T stored (tensor and shared memory)
     kBarDqFull = kBarDsReady + 2,
     kBarDqFree,
-    kBarKvTmem,                              //      256 arrivals: K and V rows copied to tensor memory
+    kBarKvTmem,                              //      8 warp arrivals: K and V rows copied to tensor memory
     kBarFinal,
     kNumBwdBarriers
 };
@@ -164,12 +164,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             mbar_init(bar(kBarStageEmpty + s), 2);
             mbar_init(bar(kBarSFull + s), 1);
             mbar_init(bar(kBarDpFull + s), 1);
-            mbar_init(bar(kBarPReady + s), kSoftmaxThreads / 2);
-            mbar_init(bar(kBarDsReady + s), kSoftmaxThreads / 2);
+            mbar_init(bar(kBarPReady + s), kSoftmaxThreads / 64);     // one arrival per warp (32 arrivals of a warp on one
+            mbar_init(bar(kBarDsReady + s), kSoftmaxThreads / 64);    // barrier are 32 serialized shared-memory atomics)
         }
         mbar_init(bar(kBarDqFull), 1);
-        mbar_init(bar(kBarDqFree), 128);
-        mbar_init(bar(kBarKvTmem), 256);
+        mbar_init(bar(kBarDqFree), 4);
+        mbar_init(bar(kBarKvTmem), 8);
         mbar_init(bar(kBarSpdFull), p.spd_tma ? 1 : 32);
         mbar_init(bar(kBarSpdEmpty), 16);
         mbar_init(bar(kBarFinal), 3);
@@ -366,7 +366,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             if constexpr (D == 64) tmem_st32(dst, w); else tmem_st16(dst, w);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bar(kBarKvTmem));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarKvTmem));
         }
 
         for (int i = 0; i < n_q; ++i) {
@@ -425,7 +426,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             tmem_ld16(tDp + 16, dpb);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bar(kBarPReady + half));    // dV of this half and the next S^T can go
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarPReady + half));    // dV of this half and the next S^T can go
             tmem_wait_ld();
 
             // ---------------- dS^T = P^T o (dP^T - Delta), bias-gradient bins ----------------
@@ -478,7 +480,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             }
             fence_proxy_async_smem();
             tc_fence_before();
-            mbar_arrive(bar(kBarDsReady + half));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarDsReady + half));
         }
 
         // ---------------- epilogue: dV (first half's warps) and dK (second half's) ----------------
@@ -542,7 +545,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 uint32_t o[32];
                 tmem_ld32(tmem + kColDq + c * 32 + lane_off, o);
                 tmem_wait_ld();
-                if (c == D / 32 - 1) { tc_fence_before(); mbar_arrive(bar(kBarDqFree)); }
+                if (c == D / 32 - 1) { tc_fence_before(); __syncwarp(); if (lane == 0) mbar_arrive(bar(kBarDqFree)); }
                 if (warp == 20 && elect_one()) {        // the reduce that last used this buffer has read it
                     if (kStgBufs == 2) bulk_wait_group_read1(); else bulk_wait_group_read0();
                 }

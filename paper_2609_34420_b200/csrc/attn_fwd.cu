@@ -178,7 +178,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         for (int s = 0; s < kVStages; ++s) { mbar_init(bar(kBarVFull + s), 1); mbar_init(bar(kBarVEmpty + s), 1); }
         for (int s = 0; s < kSpdStages; ++s) { mbar_init(bar(kBarSpdFull + s), p.spd_tma ? 1 : 32); mbar_init(bar(kBarSpdEmpty + s), kSoftmaxWarps); }
         for (int b = 0; b < 3; ++b) { mbar_init(bar(kBarSFull + b), 1); mbar_init(bar(kBarBufFree + b), 1); }
-        for (int t = 0; t < 4; ++t) mbar_init(bar(kBarPFull + t), 128 * kHalves);
+        for (int t = 0; t < 4; ++t) mbar_init(bar(kBarPFull + t), 4 * kHalves);     // one arrival per warp
         for (int t = 0; t < 4; ++t) mbar_init(bar(kBarODone + t), 1);
         fence_mbar_init();
         prefetch_tensormap(&tmap_q);
@@ -488,7 +488,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             // previous PV MMA), so odd and even key tiles use different barriers, here and for the
             // completion of the PV MMAs: a parity wait can only tell two states apart.  Two steps
             // apart is impossible because S(j+2) needs a score buffer that is only freed after PV(j).
-            mbar_arrive(bar(kBarPFull + 2 * t + (j & 1)));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kBarPFull + 2 * t + (j & 1)));
             if (j + 1 < n_kv) begin_tile(j + 1);
         }
 
