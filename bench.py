@@ -38,7 +38,7 @@ ORACLE_SAMPLE_ROWS = 256
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the backward kernel, from the ncu
 # capture summarised in profiles/attn_bwd_kernel_powerlaw16k.md (16 384-node graph, scaled by N^2).
-BWD_KERNEL_DRAM_BYTES_PER_N2 = 1013.9e6 / (16384.0 ** 2)
+BWD_KERNEL_DRAM_BYTES_PER_N2 = 1036.5e6 / (16384.0 ** 2)
 
 
 def load_peaks():
