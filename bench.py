@@ -222,7 +222,10 @@ def run_cuda(args) -> int:
         if marks is not None:
             marks[4].record()
 
-    kernels_per_step = 2 + 1 + 4 + (2 if single else 0)     # spd(setup,bfs) fwd bwd(transpose,pre,main,finalize) chunked(partial,merge)
+    # spd: setup + BFS, or for a single graph beyond the shared-memory state setup + item scan + item table +
+    # bit-matrix BFS; fwd; bwd: transpose, pre-pass, main, finalize; chunked: partial + merge
+    dense_spd = single and 12 * b.max_seqlen > 200 * 1024
+    kernels_per_step = (4 if dense_spd else 2) + 1 + 4 + (2 if single else 0)
 
     for _ in range(max(args.warmup, 0)):
         step()
@@ -306,7 +309,7 @@ def run_cuda(args) -> int:
         "flops_per_launch": f_bwd, "ms_per_launch": bwd_ms,
     }
     roofline_spd = {
-        "kernel": "spd_bfs_kernel", "bound": "hbm", "achieved": spd_alg_bytes / (spd_ms * 1e-3) / 1e9,
+        "kernel": "spd_dense_kernel" if dense_spd else "spd_bfs_kernel", "bound": "hbm", "achieved": spd_alg_bytes / (spd_ms * 1e-3) / 1e9,
         "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
         "frac": spd_alg_bytes / (spd_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"]), "peak_kind": f"hbm_gbs of {peak_kind}",
         "bytes_per_launch": spd_alg_bytes, "ms_per_launch": spd_ms, "traffic": None,

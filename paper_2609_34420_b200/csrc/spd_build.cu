@@ -12,7 +12,8 @@
 // contiguous run of one SPD row.  Every output byte is written exactly once (distances when
 // they are discovered, "unreachable" and row padding at the end), so the HBM traffic is the
 // matrix itself plus the CSR.  The frontier / next / visited words live in shared memory
-// when 12 bytes per vertex fit, otherwise in an L2-resident slice of the workspace.
+// when 12 bytes per vertex fit, otherwise in an L2-resident slice of the workspace (batches with a
+// graph beyond that size); a single graph beyond that size takes the bit-matrix build further down.
 #include "gt_common.cuh"
 
 namespace gt {
@@ -210,18 +211,385 @@ __global__ void __launch_bounds__(1024, kSmemState ? 1 : 2) spd_bfs_kernel(SpdPa
     }
 }
 
+// ------------------------------------------------------------------------------------------
+// Single large graphs (state beyond one CTA's shared memory): level-synchronous BFS on bit matrices.
+//
+// Row s of a bit matrix is a set of targets.  With F_l[s] = { t : dist(s,t) = l } the recurrence
+//     F_{l+1}[s] = ( OR over out-neighbours u of s of F_l[u] ) & ~V[s],      V[s] |= F_{l+1}[s]
+// advances ALL sources one level with plain loads and ORs: no atomics on the frontier, which is
+// what limits the per-source push above once its state lives in L2 (4.8e9 L2 atomics at 65 536
+// vertices).  The targets are processed in column blocks of 8192 (1 KB rows: a warp reads a row with
+// two 16-byte loads per lane; narrower rows make the kernel latency bound, wider ones spill), and one
+// persistent cooperative kernel walks over column blocks and levels with a grid barrier per level.
+// A warp owns a (vertex, chunk of 64 out-edges) item; vertices with more edges are split over several
+// warps that OR into an accumulator row, and the last one to finish finalises the vertex.  Items are
+// handed out in batches from a counter.  Rows of empty frontiers are not read, complete vertices are
+// skipped, and a vertex stops reading neighbours once everything it still misses is covered.
+// Distances are written as the bits appear: the 32 output bytes of a word are read (only if some of
+// them were final already), blended and written back; unreachable pairs and padding follow at the
+// end of a column block.  Cost model: per level and column block nnz x 1 KB of row reads (L2 / HBM),
+// so a graph of large diameter is slow here (levels x blocks barriers) - the kernel is meant for the
+// small-world graphs of the paper's workloads.
+// ------------------------------------------------------------------------------------------
+constexpr int kDenseBlockBits = 8192;                    // targets per column block
+constexpr int kDenseRowWords = kDenseBlockBits / 32;     // 256 words = 1 KB per row
+constexpr int kDenseVecs = kDenseRowWords / 128;         // 16-byte vectors per lane and row
+constexpr int kDenseChunk = 64;                          // out-edges per work item
+constexpr int kDenseBatch = 4;                           // work items a warp takes at a time
+constexpr uint32_t kGridWaitIterations = 1u << 24;
+
+struct DenseParams {
+    uint32_t* vis;          // [n_max][kDenseRowWords]
+    uint32_t* fr[2];        // [n_max][kDenseRowWords] current / next frontier
+    uint32_t* acc;          // [n_max][kDenseRowWords] accumulator rows of split vertices (all zero between uses)
+    uint32_t* acc_cnt;      // [n_max] finished chunks of a split vertex
+    uint8_t* nonempty[2];   // [n_max] frontier row of that buffer has a bit set
+    uint8_t* row_done;      // [n_max] every valid target of the block is visited
+    int32_t* item_start;    // [n_max + 1] prefix sum of chunks per vertex (of the current graph)
+    int32_t* item_vertex;   // [n_items] vertex of a work item
+    uint32_t* sync;         // [0] barrier counter, [1] abort, [2..5] "some frontier bit" and [8..11] work counter, by level mod 4
+    int32_t n_max;
+};
+
+// item_start[v] = sum_{u<v} max(1, ceil(deg(u)/64)) for the vertices of one graph.  One block.
+__global__ void spd_dense_items_kernel(const int32_t* __restrict__ rp, int32_t n, int32_t* __restrict__ item_start)
+{
+    __shared__ int32_t carry;
+    __shared__ int32_t part[1024];
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int base = 0; base < n; base += blockDim.x) {
+        const int v = base + threadIdx.x;
+        int32_t cnt = 0;
+        if (v < n) {
+            const int32_t deg = rp[v + 1] - rp[v];
+            cnt = deg <= kDenseChunk ? 1 : (deg + kDenseChunk - 1) / kDenseChunk;
+        }
+        part[threadIdx.x] = cnt;
+        __syncthreads();
+        for (int off = 1; off < (int)blockDim.x; off <<= 1) {
+            int32_t add = threadIdx.x >= (unsigned)off ? part[threadIdx.x - off] : 0;
+            __syncthreads();
+            part[threadIdx.x] += add;
+            __syncthreads();
+        }
+        if (v < n) item_start[v] = carry + part[threadIdx.x] - cnt;
+        __syncthreads();
+        if (threadIdx.x == blockDim.x - 1) carry += part[threadIdx.x];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) item_start[n] = carry;
+}
+
+__global__ void spd_dense_item_vertex_kernel(const int32_t* __restrict__ item_start, int32_t n, int32_t* __restrict__ item_vertex)
+{
+    const int v = blockIdx.x * blockDim.x + threadIdx.x;
+    if (v >= n) return;
+    for (int32_t i = item_start[v]; i < item_start[v + 1]; ++i) item_vertex[i] = v;
+}
+
+// Grid barrier with a bounded wait (the kernel is launched cooperatively, so all CTAs are resident).
+// Returns false once any CTA has given up; every CTA then leaves the kernel.
+__device__ __forceinline__ bool dense_grid_sync(uint32_t* sync, uint32_t& epoch, uint32_t* status)
+{
+    __shared__ uint32_t s_ok;
+    ++epoch;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t target = epoch * gridDim.x;
+        __threadfence();
+        atomicAdd(&sync[0], 1u);
+        uint32_t ok = 0;
+        for (uint32_t it = 0; it < kGridWaitIterations; ++it) {
+            if (*(volatile uint32_t*)&sync[0] >= target) { ok = 1; break; }
+            if (*(volatile uint32_t*)&sync[1]) break;
+            __nanosleep(32);
+        }
+        if (!ok && atomicExch(&sync[1], 1u) == 0u) {
+            if (atomicCAS(status, 0u, 5u /* GT_ERR_DEVICE_TIMEOUT */) == 0u) status[1] = 200;
+        }
+        __threadfence();
+        s_ok = ok;
+    }
+    __syncthreads();
+    return s_ok != 0;
+}
+
+// the 16 output bytes of 16 targets: bytes whose bit is set in m16 take `code`, the others keep `old`
+__device__ __forceinline__ uint4 dense_blend16(uint4 old, uint32_t m16, uint32_t code4)
+{
+    uint32_t o[4] = {old.x, old.y, old.z, old.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint32_t nib = (m16 >> (4 * j)) & 0xFu;
+        const uint32_t bm = ((nib * 0x00204081u) & 0x01010101u) * 0xFFu;      // bit i of the nibble -> byte i
+        o[j] = (o[j] & ~bm) | (code4 & bm);
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// bytes of word `w` (32 targets from t0) of output row `row`: bits of `set` take `code`; bytes whose bit is in
+// `keep` are final already and are preserved (the row is only read when there are any)
+__device__ __forceinline__ void dense_write_word(uint8_t* row, int32_t t0, uint32_t set, uint32_t keep, uint32_t code)
+{
+    const uint32_t code4 = code * 0x01010101u;
+#pragma unroll
+    for (int hlf = 0; hlf < 2; ++hlf) {
+        const uint32_t m = (set >> (16 * hlf)) & 0xFFFFu;
+        if (m) {
+            uint4* ptr = (uint4*)(row + t0 + 16 * hlf);
+            uint4 old = make_uint4(0u, 0u, 0u, 0u);
+            if ((keep >> (16 * hlf)) & 0xFFFFu) old = __ldcg(ptr);      // written by another SM in an earlier level
+            *ptr = dense_blend16(old, m, code4);
+        }
+    }
+}
+
+// word index of component j of vector q of a lane: a lane holds kDenseVecs vectors of four consecutive words,
+// vector q of all lanes together is a contiguous 512-byte piece of the row
+__device__ __forceinline__ int dense_word(int lane, int q, int j) { return q * 128 + lane * 4 + j; }
+
+__global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DenseParams d)
+{
+    const int lane = threadIdx.x & 31;
+    const int gw = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+    const int n_gw = (int)((gridDim.x * blockDim.x) >> 5);
+    const int32_t n = p.n_total;
+    const int64_t ld = (int64_t)((n + 15) & ~15);
+    const int32_t* __restrict__ rp = p.row_ptr;
+    const int32_t* __restrict__ ci = p.col_idx;
+    const int32_t n_items = d.item_start[n];
+    const uint32_t unreach = (uint32_t)(p.max_dist + 1);
+    uint32_t epoch = 0;
+    uint32_t step = 0;                         // levels over all column blocks: index of the rotating "any" flags
+
+    // finalise vertex s for this level: new bits, visited, next frontier row, flags, output bytes
+    auto finalise = [&](int s, const uint32_t (&acc)[kDenseVecs][4], int32_t col0, uint32_t* vis_row, uint32_t* next_row,
+                        uint8_t* next_nonempty, uint32_t code, uint32_t flag_idx) {
+        bool any_new = false, full = true;
+        const bool rewrite = __ldcg(&next_nonempty[s]) != 0;      // the row this level overwrites has bits set
+#pragma unroll
+        for (int q = 0; q < kDenseVecs; ++q) {
+            const uint4 v4 = __ldcg((const uint4*)&vis_row[dense_word(lane, q, 0)]);   // written by other SMs earlier: from L2
+            const uint32_t v[4] = {v4.x, v4.y, v4.z, v4.w};
+            uint32_t nw[4];
+            bool vec_new = false;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int32_t t0 = col0 + dense_word(lane, q, j) * 32;
+                const int32_t nv = n - t0;
+                const uint32_t vm = nv >= 32 ? 0xffffffffu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
+                nw[j] = acc[q][j] & ~v[j] & vm;
+                if (nw[j]) {
+                    dense_write_word(p.spd + (int64_t)s * ld, t0, nw[j], v[j], code);
+                    vec_new = true;
+                }
+                full = full && (((v[j] | nw[j]) & vm) == vm);
+            }
+            if (vec_new || rewrite) *(uint4*)&next_row[dense_word(lane, q, 0)] = make_uint4(nw[0], nw[1], nw[2], nw[3]);
+            if (vec_new) *(uint4*)&vis_row[dense_word(lane, q, 0)] = make_uint4(v[0] | nw[0], v[1] | nw[1], v[2] | nw[2], v[3] | nw[3]);
+            any_new = any_new || vec_new;
+        }
+        const bool row_new = __any_sync(0xffffffffu, any_new);
+        const bool row_full = __all_sync(0xffffffffu, full);
+        if (lane == 0) {
+            next_nonempty[s] = row_new ? 1 : 0;
+            if (row_new) d.sync[2 + flag_idx] = 1u;
+            if (row_full) d.row_done[s] = 1;
+        }
+    };
+
+    for (int32_t col0 = 0; col0 < (int32_t)ld; col0 += kDenseBlockBits) {
+        // ---- level 0 of this column block: every vertex has reached itself ----
+        for (int s = gw; s < n; s += n_gw) {
+#pragma unroll
+            for (int q = 0; q < kDenseVecs; ++q) {
+                uint32_t bit[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int32_t rel = s - col0 - dense_word(lane, q, j) * 32;
+                    bit[j] = (rel >= 0 && rel < 32) ? (1u << rel) : 0u;
+                }
+                const uint4 b4 = make_uint4(bit[0], bit[1], bit[2], bit[3]);
+                *(uint4*)&d.vis[(size_t)s * kDenseRowWords + dense_word(lane, q, 0)] = b4;
+                *(uint4*)&d.fr[0][(size_t)s * kDenseRowWords + dense_word(lane, q, 0)] = b4;
+            }
+            if (lane == 0) {
+                const bool mine = s >= col0 && s < col0 + kDenseBlockBits;
+                d.nonempty[0][s] = mine ? 1 : 0;
+                d.nonempty[1][s] = 1;                  // the other buffer holds stale bits: level 1 rewrites every row
+                d.row_done[s] = 0;
+                if (mine) p.spd[(int64_t)s * ld + s] = 0;
+            }
+        }
+        if (!dense_grid_sync(d.sync, epoch, p.header)) return;
+
+        int cur = 0;
+        for (int level = 1;; ++level) {
+            const uint32_t code = (uint32_t)min(level, p.max_dist);
+            const uint32_t flag_idx = step & 3u;
+            const uint32_t* fcur = d.fr[cur];
+            uint32_t* fnext = d.fr[cur ^ 1];
+            const uint8_t* ne_cur = d.nonempty[cur];
+            uint8_t* ne_next = d.nonempty[cur ^ 1];
+            // Items cost between one flag read and 64 KB of row reads, so warps take them in batches of four
+            // from a counter (one per level, four in rotation) and ask for the next batch before working.
+            uint32_t* counter = &d.sync[8 + flag_idx];
+            int batch_next = 0;
+            if (lane == 0) batch_next = (int)atomicAdd(counter, kDenseBatch);
+            for (;;) {
+                const int batch = __shfl_sync(0xffffffffu, batch_next, 0);
+                if (batch >= n_items) break;
+                if (lane == 0) batch_next = (int)atomicAdd(counter, kDenseBatch);
+              for (int item = batch; item < min(batch + kDenseBatch, n_items); ++item) {
+                const int s = d.item_vertex[item];
+                const int32_t first = d.item_start[s];
+                const int32_t n_chunks = d.item_start[s + 1] - first;
+                const int32_t c = item - first;
+                uint32_t acc[kDenseVecs][4];
+#pragma unroll
+                for (int q = 0; q < kDenseVecs; ++q)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) acc[q][j] = 0u;
+                uint32_t* vis_row = d.vis + (size_t)s * kDenseRowWords;
+                const bool done = __ldcg(&d.row_done[s]) != 0;
+                // a complete vertex whose row in the next-frontier buffer is already empty needs nothing at all
+                // (every chunk of a split vertex sees the same two flags, so they all skip together)
+                if (done && !__ldcg(&ne_next[s])) continue;
+                if (!done) {
+                    // bits this vertex still misses: once the neighbours read so far cover them all, the rest
+                    // of the edge list cannot add anything (at the dense levels a few rows are enough)
+                    uint32_t need[kDenseVecs][4];
+#pragma unroll
+                    for (int q = 0; q < kDenseVecs; ++q) {
+                        const uint4 v4 = __ldcg((const uint4*)&vis_row[dense_word(lane, q, 0)]);
+                        const uint32_t v[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int32_t nv = n - (col0 + dense_word(lane, q, j) * 32);
+                            const uint32_t vm = nv >= 32 ? 0xffffffffu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
+                            need[q][j] = ~v[j] & vm;
+                        }
+                    }
+                    bool covered = false;
+                    const int32_t e0 = rp[s] + c * kDenseChunk;
+                    const int32_t e1 = min(rp[s + 1], e0 + kDenseChunk);
+#pragma unroll
+                    for (int part = 0; part < kDenseChunk / 32 && !covered; ++part) {
+                        const int32_t e = e0 + part * 32 + lane;
+                        int32_t u = e < e1 ? ci[e] : -1;
+                        if (u >= 0 && !__ldcg(&ne_cur[u])) u = -1;     // empty frontier row: nothing to OR
+                        uint32_t m = __ballot_sync(0xffffffffu, u >= 0);
+                        while (m) {                                   // two frontier rows (2 x 1 KB) in flight
+                            const int b0 = __ffs(m) - 1;
+                            m &= m - 1;
+                            const int u0 = __shfl_sync(0xffffffffu, u, b0);
+                            int u1 = -1;
+                            if (m) { const int b1 = __ffs(m) - 1; m &= m - 1; u1 = __shfl_sync(0xffffffffu, u, b1); }
+                            uint4 x[kDenseVecs], y[kDenseVecs];
+                            const uint32_t* r0 = fcur + (size_t)u0 * kDenseRowWords;
+#pragma unroll
+                            for (int q = 0; q < kDenseVecs; ++q) x[q] = __ldcg((const uint4*)&r0[dense_word(lane, q, 0)]);
+#pragma unroll
+                            for (int q = 0; q < kDenseVecs; ++q) y[q] = make_uint4(0u, 0u, 0u, 0u);
+                            if (u1 >= 0) {
+                                const uint32_t* r1 = fcur + (size_t)u1 * kDenseRowWords;
+#pragma unroll
+                                for (int q = 0; q < kDenseVecs; ++q) y[q] = __ldcg((const uint4*)&r1[dense_word(lane, q, 0)]);
+                            }
+#pragma unroll
+                            for (int q = 0; q < kDenseVecs; ++q) {
+                                acc[q][0] |= x[q].x | y[q].x; acc[q][1] |= x[q].y | y[q].y;
+                                acc[q][2] |= x[q].z | y[q].z; acc[q][3] |= x[q].w | y[q].w;
+                            }
+                            uint32_t left = 0u;
+#pragma unroll
+                            for (int q = 0; q < kDenseVecs; ++q)
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) left |= need[q][j] & ~acc[q][j];
+                            if (__all_sync(0xffffffffu, left == 0u)) { covered = true; break; }
+                        }
+                    }
+                }
+                uint32_t* next_row = fnext + (size_t)s * kDenseRowWords;
+                if (n_chunks == 1) {
+                    finalise(s, acc, col0, vis_row, next_row, ne_next, code, flag_idx);
+                } else {
+                    uint32_t* acc_row = d.acc + (size_t)s * kDenseRowWords;
+#pragma unroll
+                    for (int q = 0; q < kDenseVecs; ++q)
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (acc[q][j]) atomicOr(&acc_row[dense_word(lane, q, j)], acc[q][j]);
+                    __threadfence();
+                    __syncwarp();
+                    uint32_t last = 0;
+                    if (lane == 0) last = atomicAdd(&d.acc_cnt[s], 1u) == (uint32_t)(n_chunks - 1) ? 1u : 0u;
+                    last = __shfl_sync(0xffffffffu, last, 0);
+                    if (last) {                            // all chunks of the vertex are in: take the row and clear it
+                        __threadfence();
+#pragma unroll
+                        for (int q = 0; q < kDenseVecs; ++q) {
+                            const uint4 a4 = __ldcg((const uint4*)&acc_row[dense_word(lane, q, 0)]);
+                            acc[q][0] = a4.x; acc[q][1] = a4.y; acc[q][2] = a4.z; acc[q][3] = a4.w;
+                            if (a4.x | a4.y | a4.z | a4.w) *(uint4*)&acc_row[dense_word(lane, q, 0)] = make_uint4(0u, 0u, 0u, 0u);
+                        }
+                        if (lane == 0) d.acc_cnt[s] = 0u;
+                        finalise(s, acc, col0, vis_row, next_row, ne_next, code, flag_idx);
+                    }
+                }
+              }
+            }
+            if (!dense_grid_sync(d.sync, epoch, p.header)) return;
+            const uint32_t any = *(volatile uint32_t*)&d.sync[2 + flag_idx];
+            if (blockIdx.x == 0 && threadIdx.x == 0) {          // next written two levels from now
+                d.sync[2 + ((step + 2u) & 3u)] = 0u;
+                d.sync[8 + ((step + 2u) & 3u)] = 0u;
+            }
+            ++step;
+            cur ^= 1;
+            if (!any) break;
+        }
+
+        // ---- unreachable pairs and row padding of this column block ----
+        for (int s = gw; s < n; s += n_gw) {
+            uint8_t* row = p.spd + (int64_t)s * ld;
+#pragma unroll
+            for (int q = 0; q < kDenseVecs; ++q) {
+                const uint4 v4 = __ldcg((const uint4*)&d.vis[(size_t)s * kDenseRowWords + dense_word(lane, q, 0)]);
+                const uint32_t v[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int32_t t0 = col0 + dense_word(lane, q, j) * 32;
+                    if (t0 >= (int32_t)ld) continue;
+                    const int32_t nv = n - t0, np = (int32_t)ld - t0;
+                    const uint32_t vm = nv >= 32 ? 0xffffffffu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
+                    const uint32_t pm = (np >= 32 ? 0xffffffffu : ((1u << np) - 1u)) & ~vm;       // padding columns
+                    const uint32_t miss = ~v[j] & vm;
+                    if (miss) dense_write_word(row, t0, miss, v[j] | pm, unreach);
+                    if (pm) dense_write_word(row, t0, pm, vm, 255u);
+                }
+            }
+        }
+        // the same warps own the same vertices in the next block's level 0, and nothing else touches the
+        // bit matrices until the barrier behind it
+    }
+}
+
 size_t spd_state_bytes(int32_t max_seqlen) { return (size_t)3 * (size_t)max_seqlen * sizeof(uint32_t); }
 constexpr size_t kSmemStateLimit = 200 * 1024;
 
 struct SpdPlan {
     bool smem_state;
+    bool dense;                // single large graph: bit-matrix BFS (persistent cooperative kernel)
+    size_t dense_off[11];      // vis, fr0, fr1, acc, acc_cnt, nonempty0, nonempty1, row_done, item_start, sync, item_vertex
     int threads;
     int grid;
     size_t smem_bytes;
     size_t batch_start_off, scratch_off, scratch_words_per_cta, total_bytes;
 };
 
-SpdPlan make_plan(const gt_batch* b)
+SpdPlan make_plan(const gt_batch* b, int64_t nnz)
 {
     SpdPlan pl{};
     size_t state = spd_state_bytes(b->max_seqlen);
@@ -243,6 +611,30 @@ SpdPlan make_plan(const gt_batch* b)
     pl.scratch_off = align_up(pl.batch_start_off + sizeof(int32_t) * ((size_t)b->n_graphs + 1), 256);
     pl.scratch_words_per_cta = pl.smem_state ? 0 : align_up((size_t)3 * b->max_seqlen, 64);
     pl.total_bytes = pl.scratch_off + pl.scratch_words_per_cta * sizeof(uint32_t) * (size_t)pl.grid;
+    pl.dense = false;
+    if (!pl.smem_state && b->n_graphs == 1) {
+        int dev = 0, coop = 0, per_sm_dense = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && coop &&
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm_dense, spd_dense_kernel, 512, 0) == cudaSuccess && per_sm_dense >= 1) {
+            pl.dense = true;
+            pl.threads = 512;
+            pl.grid = sms * per_sm_dense;
+            const size_t n = (size_t)b->n_total;
+            const size_t mat = align_up(n * kDenseRowWords * sizeof(uint32_t), 256);
+            size_t off = pl.scratch_off;
+            for (int i = 0; i < 4; ++i) { pl.dense_off[i] = off; off += mat; }
+            pl.dense_off[4] = off; off += align_up(n * sizeof(uint32_t), 256);
+            for (int i = 5; i < 8; ++i) { pl.dense_off[i] = off; off += align_up(n, 256); }
+            pl.dense_off[8] = off; off += align_up((n + 1) * sizeof(int32_t), 256);
+            pl.dense_off[9] = off; off += 256;
+            // work items: one per vertex plus one per further 64 out-edges
+            pl.dense_off[10] = off; off += align_up((n + (size_t)(nnz > 0 ? nnz : 0) / kDenseChunk + 1) * sizeof(int32_t), 256);
+            pl.total_bytes = off;
+        } else {
+            cudaGetLastError();
+        }
+    }
     return pl;
 }
 
@@ -251,9 +643,9 @@ SpdPlan make_plan(const gt_batch* b)
 
 extern "C" size_t gt_spd_build_workspace(const gt_batch* batch, int64_t nnz, int32_t max_dist)
 {
-    (void)nnz; (void)max_dist;
+    (void)max_dist;
     if (gt::validate_batch(batch) != GT_OK) return 0;
-    return gt::make_plan(batch).total_bytes;
+    return gt::make_plan(batch, nnz).total_bytes;
 }
 
 extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx, int64_t nnz,
@@ -268,7 +660,7 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
     if (max_dist < 1 || max_dist > 254) return GT_ERR_INVALID_ARG;
     if (batch->n_graphs > 1 && spd_offsets == nullptr) return GT_ERR_INVALID_ARG;
     if (sm_count() <= 0) return GT_ERR_NO_DEVICE;
-    SpdPlan pl = make_plan(batch);
+    SpdPlan pl = make_plan(batch, nnz);
     if (workspace == nullptr || workspace_bytes < pl.total_bytes || misaligned16(workspace)) return GT_ERR_WORKSPACE;
 
     cudaStream_t s = (cudaStream_t)stream;
@@ -290,6 +682,31 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
     GT_CUDA_TRY(cudaMemsetAsync(ws + 8, 0, 8, s));     // work counter and item count
     spd_setup_kernel<<<1, 1024, 0, s>>>(p);
     GT_CUDA_TRY(cudaGetLastError());
+    if (pl.dense) {
+        DenseParams d{};
+        d.vis = (uint32_t*)(ws + pl.dense_off[0]);
+        d.fr[0] = (uint32_t*)(ws + pl.dense_off[1]);
+        d.fr[1] = (uint32_t*)(ws + pl.dense_off[2]);
+        d.acc = (uint32_t*)(ws + pl.dense_off[3]);
+        d.acc_cnt = (uint32_t*)(ws + pl.dense_off[4]);
+        d.nonempty[0] = ws + pl.dense_off[5];
+        d.nonempty[1] = ws + pl.dense_off[6];
+        d.row_done = ws + pl.dense_off[7];
+        d.item_start = (int32_t*)(ws + pl.dense_off[8]);
+        d.sync = (uint32_t*)(ws + pl.dense_off[9]);
+        d.item_vertex = (int32_t*)(ws + pl.dense_off[10]);
+        d.n_max = batch->n_total;
+        // accumulator rows, their counters and the barrier words start at zero
+        GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[3], 0, pl.dense_off[5] - pl.dense_off[3], s));
+        GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[9], 0, 256, s));
+        spd_dense_items_kernel<<<1, 1024, 0, s>>>(row_ptr, batch->n_total, d.item_start);
+        GT_CUDA_TRY(cudaGetLastError());
+        spd_dense_item_vertex_kernel<<<(unsigned)((batch->n_total + 255) / 256), 256, 0, s>>>(d.item_start, batch->n_total, d.item_vertex);
+        GT_CUDA_TRY(cudaGetLastError());
+        void* args[] = {(void*)&p, (void*)&d};
+        GT_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)spd_dense_kernel, dim3((unsigned)pl.grid), dim3((unsigned)pl.threads), args, 0, s));
+        return GT_OK;
+    }
     if (pl.smem_state) {
         GT_CUDA_TRY(cudaFuncSetAttribute(spd_bfs_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes));
         spd_bfs_kernel<true><<<pl.grid, pl.threads, pl.smem_bytes, s>>>(p);

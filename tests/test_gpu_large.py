@@ -83,3 +83,44 @@ def test_powerlaw16k_full_spd_and_row_slab_attention():
 
 def test_powerlaw64k_full_spd_and_row_slab_attention():
     run_large("powerlaw64k", n_slab=128, full_spd_oracle=True)
+
+
+# ---- single graphs beyond the shared-memory BFS state: the bit-matrix build ----
+def _spd_of(csr, max_dist):
+    w = wl.Workload("big", wl.pack_graphs([csr]), 1, 32, max_dist)
+    bt = device_batch(w.batch)
+    rp, ci = device_csr(w.batch)
+    spd = torch.empty(w.batch.spd_bytes, dtype=torch.uint8, device="cuda")
+    gt.gt_spd_build(rp, ci, bt, max_dist, spd)
+    torch.cuda.synchronize()
+    n = w.batch.n_total
+    return w, spd.cpu().numpy().reshape(n, -1)
+
+
+def test_bit_matrix_build_directed_ragged_with_hub_and_isolated_vertices():
+    n = 18001                                   # pitch 18016: padding columns; three column blocks, the last ragged
+    rng = np.random.Generator(np.random.PCG64(5))
+    m = 3 * n
+    src = rng.integers(0, n - 200, size=m)      # the last 200 vertices have no out-edges
+    dst = rng.integers(0, n - 100, size=m)      # the last 100 are isolated
+    hub_dst = rng.choice(n - 100, size=3000, replace=False)      # a vertex split over many work items
+    src = np.concatenate([src, np.full(3000, 7)])
+    dst = np.concatenate([dst, hub_dst])
+    csr = wl.csr_from_edges(n, src, dst, symmetric=False)
+    w, got = _spd_of(csr, 7)
+    exp = ospd.spd_matrix(w.batch.row_ptr, w.batch.col_idx, 7)
+    assert got.shape == exp.shape
+    np.testing.assert_array_equal(got, exp)
+
+
+def test_bit_matrix_build_ring_runs_thousands_of_levels_and_clips():
+    n = 17500
+    i = np.arange(n)
+    csr = wl.csr_from_edges(n, i, (i + 1) % n, symmetric=True)
+    w, got = _spd_of(csr, 50)
+    rows = np.array([0, 1, 8191, 8192, 12345, n - 1])
+    j = np.arange(n)
+    for r in rows:
+        ring = np.minimum((j - r) % n, (r - j) % n)
+        np.testing.assert_array_equal(got[r, :n], np.minimum(ring, 50))
+    assert (got[:, n:] == 255).all()
