@@ -221,7 +221,7 @@ __global__ void __launch_bounds__(1024, kSmemState ? 1 : 2) spd_bfs_kernel(SpdPa
 // vertices).  The targets are processed in column blocks of 8192 (1 KB rows: a warp reads a row with
 // two 16-byte loads per lane; narrower rows make the kernel latency bound, wider ones spill), and one
 // persistent cooperative kernel walks over column blocks and levels with a grid barrier per level.
-// A warp owns a (vertex, chunk of 64 out-edges) item; vertices with more edges are split over several
+// A warp owns a (vertex, chunk of 32 out-edges) item; vertices with more edges are split over several
 // warps that OR into an accumulator row, and the last one to finish finalises the vertex.  Items are
 // handed out in batches from a counter.  Rows of empty frontiers are not read, complete vertices are
 // skipped, and a vertex stops reading neighbours once everything it still misses is covered.
@@ -234,7 +234,7 @@ __global__ void __launch_bounds__(1024, kSmemState ? 1 : 2) spd_bfs_kernel(SpdPa
 constexpr int kDenseBlockBits = 8192;                    // targets per column block
 constexpr int kDenseRowWords = kDenseBlockBits / 32;     // 256 words = 1 KB per row
 constexpr int kDenseVecs = kDenseRowWords / 128;         // 16-byte vectors per lane and row
-constexpr int kDenseChunk = 64;                          // out-edges per work item
+constexpr int kDenseChunk = 32;                          // out-edges per work item
 constexpr int kDenseBatch = 4;                           // work items a warp takes at a time
 constexpr uint32_t kGridWaitIterations = 1u << 24;
 
@@ -432,16 +432,19 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
             uint32_t* fnext = d.fr[cur ^ 1];
             const uint8_t* ne_cur = d.nonempty[cur];
             uint8_t* ne_next = d.nonempty[cur ^ 1];
-            // Items cost between one flag read and 64 KB of row reads, so warps take them in batches of four
-            // from a counter (one per level, four in rotation) and ask for the next batch before working.
+            // Items cost between one flag read and tens of KB of row reads, so warps take them in batches of four
+            // from a counter (one per level, four in rotation) and ask for the next batch before working.  The
+            // four items of a batch lie a quarter of the list apart: the chunks of one high-degree vertex are
+            // neighbours in the list and would otherwise queue up in one warp.
             uint32_t* counter = &d.sync[8 + flag_idx];
+            const int n_batches = (n_items + kDenseBatch - 1) / kDenseBatch;
             int batch_next = 0;
-            if (lane == 0) batch_next = (int)atomicAdd(counter, kDenseBatch);
+            if (lane == 0) batch_next = (int)atomicAdd(counter, 1u);
             for (;;) {
                 const int batch = __shfl_sync(0xffffffffu, batch_next, 0);
-                if (batch >= n_items) break;
-                if (lane == 0) batch_next = (int)atomicAdd(counter, kDenseBatch);
-              for (int item = batch; item < min(batch + kDenseBatch, n_items); ++item) {
+                if (batch >= n_batches) break;
+                if (lane == 0) batch_next = (int)atomicAdd(counter, 1u);
+              for (int item = batch; item < n_items; item += n_batches) {
                 const int s = d.item_vertex[item];
                 const int32_t first = d.item_start[s];
                 const int32_t n_chunks = d.item_start[s + 1] - first;
