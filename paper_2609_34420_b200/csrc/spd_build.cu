@@ -236,6 +236,7 @@ constexpr int kDenseRowWords = kDenseBlockBits / 32;     // 256 words = 1 KB per
 constexpr int kDenseVecs = kDenseRowWords / 128;         // 16-byte vectors per lane and row
 constexpr int kDenseChunk = 32;                          // out-edges per work item
 constexpr int kDenseBatch = 4;                           // work items a warp takes at a time
+constexpr int kDenseMaxGroups = 4;                       // CTA groups working on different column blocks at once
 constexpr uint32_t kGridWaitIterations = 1u << 24;
 
 struct DenseParams {
@@ -249,6 +250,7 @@ struct DenseParams {
     int32_t* item_vertex;   // [n_items] vertex of a work item
     uint32_t* sync;         // [0] barrier counter, [1] abort, [2..5] "some frontier bit" and [8..11] work counter, by level mod 4
     int32_t n_max;
+    int32_t n_groups;       // CTA groups that work on different column blocks at the same time (own state each)
 };
 
 // item_start[v] = sum_{u<v} max(1, ceil(deg(u)/64)) for the vertices of one graph.  One block.
@@ -290,13 +292,13 @@ __global__ void spd_dense_item_vertex_kernel(const int32_t* __restrict__ item_st
 
 // Grid barrier with a bounded wait (the kernel is launched cooperatively, so all CTAs are resident).
 // Returns false once any CTA has given up; every CTA then leaves the kernel.
-__device__ __forceinline__ bool dense_grid_sync(uint32_t* sync, uint32_t& epoch, uint32_t* status)
+__device__ __forceinline__ bool dense_grid_sync(uint32_t* sync, uint32_t& epoch, uint32_t* status, uint32_t n_ctas)
 {
     __shared__ uint32_t s_ok;
     ++epoch;
     __syncthreads();
     if (threadIdx.x == 0) {
-        const uint32_t target = epoch * gridDim.x;
+        const uint32_t target = epoch * n_ctas;
         __threadfence();
         atomicAdd(&sync[0], 1u);
         uint32_t ok = 0;
@@ -351,9 +353,21 @@ __device__ __forceinline__ int dense_word(int lane, int q, int j) { return q * 1
 
 __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DenseParams d)
 {
+    // CTA group g (CTAs g, g + G, ...) works on column blocks g, g + G, ... with its own bit matrices, flags
+    // and barrier: while one group waits for its slowest warp at a level barrier, the CTAs of the other groups
+    // on the same SMs keep the memory system busy.
+    const int grp = (int)blockIdx.x % d.n_groups;
+    const int cta = (int)blockIdx.x / d.n_groups;                                   // index within the group
+    const uint32_t n_ctas = ((uint32_t)gridDim.x - (uint32_t)grp + (uint32_t)d.n_groups - 1u) / (uint32_t)d.n_groups;
+    {
+        const size_t m = (size_t)grp * d.n_max;
+        d.vis += m * kDenseRowWords; d.fr[0] += m * kDenseRowWords; d.fr[1] += m * kDenseRowWords; d.acc += m * kDenseRowWords;
+        d.acc_cnt += m; d.nonempty[0] += m; d.nonempty[1] += m; d.row_done += m;
+        d.sync += grp * 64;
+    }
     const int lane = threadIdx.x & 31;
-    const int gw = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5);
-    const int n_gw = (int)((gridDim.x * blockDim.x) >> 5);
+    const int gw = (int)((cta * blockDim.x + threadIdx.x) >> 5);
+    const int n_gw = (int)((n_ctas * blockDim.x) >> 5);
     const int32_t n = p.n_total;
     const int64_t ld = (int64_t)((n + 15) & ~15);
     const int32_t* __restrict__ rp = p.row_ptr;
@@ -399,7 +413,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
         }
     };
 
-    for (int32_t col0 = 0; col0 < (int32_t)ld; col0 += kDenseBlockBits) {
+    for (int32_t col0 = grp * kDenseBlockBits; col0 < (int32_t)ld; col0 += d.n_groups * kDenseBlockBits) {
         // ---- level 0 of this column block: every vertex has reached itself ----
         for (int s = gw; s < n; s += n_gw) {
 #pragma unroll
@@ -422,7 +436,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                 if (mine) p.spd[(int64_t)s * ld + s] = 0;
             }
         }
-        if (!dense_grid_sync(d.sync, epoch, p.header)) return;
+        if (!dense_grid_sync(d.sync, epoch, p.header, n_ctas)) return;
 
         int cur = 0;
         for (int level = 1;; ++level) {
@@ -543,9 +557,9 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                 }
               }
             }
-            if (!dense_grid_sync(d.sync, epoch, p.header)) return;
+            if (!dense_grid_sync(d.sync, epoch, p.header, n_ctas)) return;
             const uint32_t any = *(volatile uint32_t*)&d.sync[2 + flag_idx];
-            if (blockIdx.x == 0 && threadIdx.x == 0) {          // next written two levels from now
+            if (cta == 0 && threadIdx.x == 0) {                 // next written two levels from now
                 d.sync[2 + ((step + 2u) & 3u)] = 0u;
                 d.sync[8 + ((step + 2u) & 3u)] = 0u;
             }
@@ -585,6 +599,7 @@ constexpr size_t kSmemStateLimit = 200 * 1024;
 struct SpdPlan {
     bool smem_state;
     bool dense;                // single large graph: bit-matrix BFS (persistent cooperative kernel)
+    int dense_groups;
     size_t dense_off[11];      // vis, fr0, fr1, acc, acc_cnt, nonempty0, nonempty1, row_done, item_start, sync, item_vertex
     int threads;
     int grid;
@@ -624,13 +639,16 @@ SpdPlan make_plan(const gt_batch* b, int64_t nnz)
             pl.threads = 512;
             pl.grid = sms * per_sm_dense;
             const size_t n = (size_t)b->n_total;
-            const size_t mat = align_up(n * kDenseRowWords * sizeof(uint32_t), 256);
+            const int n_col_blocks = (int)((n + 15 + kDenseBlockBits - 1) / kDenseBlockBits);
+            pl.dense_groups = n_col_blocks < kDenseMaxGroups ? n_col_blocks : kDenseMaxGroups;
+            const size_t G = (size_t)pl.dense_groups;
+            const size_t mat = align_up(G * n * kDenseRowWords * sizeof(uint32_t), 256);
             size_t off = pl.scratch_off;
             for (int i = 0; i < 4; ++i) { pl.dense_off[i] = off; off += mat; }
-            pl.dense_off[4] = off; off += align_up(n * sizeof(uint32_t), 256);
-            for (int i = 5; i < 8; ++i) { pl.dense_off[i] = off; off += align_up(n, 256); }
+            pl.dense_off[4] = off; off += align_up(G * n * sizeof(uint32_t), 256);
+            for (int i = 5; i < 8; ++i) { pl.dense_off[i] = off; off += align_up(G * n, 256); }
             pl.dense_off[8] = off; off += align_up((n + 1) * sizeof(int32_t), 256);
-            pl.dense_off[9] = off; off += 256;
+            pl.dense_off[9] = off; off += 256 * kDenseMaxGroups;
             // work items: one per vertex plus one per further 64 out-edges
             pl.dense_off[10] = off; off += align_up((n + (size_t)(nnz > 0 ? nnz : 0) / kDenseChunk + 1) * sizeof(int32_t), 256);
             pl.total_bytes = off;
@@ -699,9 +717,10 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
         d.sync = (uint32_t*)(ws + pl.dense_off[9]);
         d.item_vertex = (int32_t*)(ws + pl.dense_off[10]);
         d.n_max = batch->n_total;
+        d.n_groups = pl.dense_groups;
         // accumulator rows, their counters and the barrier words start at zero
         GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[3], 0, pl.dense_off[5] - pl.dense_off[3], s));
-        GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[9], 0, 256, s));
+        GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[9], 0, 256 * kDenseMaxGroups, s));
         spd_dense_items_kernel<<<1, 1024, 0, s>>>(row_ptr, batch->n_total, d.item_start);
         GT_CUDA_TRY(cudaGetLastError());
         spd_dense_item_vertex_kernel<<<(unsigned)((batch->n_total + 255) / 256), 256, 0, s>>>(d.item_start, batch->n_total, d.item_vertex);
