@@ -575,38 +575,49 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 }
 
 // spd_t[j][i] = min(spd[i][j], n_buckets - 1) for every graph block (same offsets and pitch as the
-// source).  64 x 64 byte tiles through shared memory; reads and writes are both coalesced.
+// source).  One CTA moves a 128 x 128 byte tile: 16-byte coalesced loads into shared memory (16-byte
+// chunk c of row r at chunk c ^ (r >> 4), which makes the column reads below conflict free), then every
+// thread reads a 16-row x 4-column block as 16 words, transposes it with byte permutes and writes four
+// 16-byte pieces of four output rows; eight neighbouring lanes fill 128 contiguous bytes of a row.
 __global__ void __launch_bounds__(256) spd_transpose_clamp_kernel(const uint8_t* __restrict__ spd, uint8_t* __restrict__ spd_t,
                                                                   const int64_t* __restrict__ spd_offsets,
                                                                   const int32_t* __restrict__ cu_seqlens, int32_t n_total,
                                                                   uint32_t last_bucket)
 {
-    __shared__ uint8_t tile[64][64 + 4];
+    __shared__ __align__(16) uint32_t tile[128 * 32];
     const int g = blockIdx.z;
     const int32_t n_g = cu_seqlens ? cu_seqlens[g + 1] - cu_seqlens[g] : n_total;
-    const int32_t i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
+    const int32_t i0 = blockIdx.y * 128, j0 = blockIdx.x * 128;
     if (i0 >= n_g || j0 >= n_g) return;
     const int64_t ld = (int64_t)((n_g + 15) & ~15);
     const int64_t base = spd_offsets ? spd_offsets[g] : 0;
-    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;          // 16 x 16 threads, 4 bytes x 4 rows each
+    const uint32_t cap = last_bucket * 0x01010101u;
+    const int t = threadIdx.x;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-        const int i = i0 + ty * 4 + k, j = j0 + tx * 4;
-        uint32_t w = 0;
-        if (i < n_g && j < ld) w = *(const uint32_t*)(spd + base + (int64_t)i * ld + j);
-#pragma unroll
-        for (int b = 0; b < 4; ++b) tile[ty * 4 + k][tx * 4 + b] = (uint8_t)min((w >> (8 * b)) & 0xffu, last_bucket);
+        const int r = (t >> 3) + 32 * k, c = t & 7;
+        uint4 w = make_uint4(0u, 0u, 0u, 0u);
+        if (i0 + r < n_g && j0 + c * 16 < ld) w = *(const uint4*)(spd + base + (int64_t)(i0 + r) * ld + j0 + c * 16);
+        w.x = __vminu4(w.x, cap); w.y = __vminu4(w.y, cap); w.z = __vminu4(w.z, cap); w.w = __vminu4(w.w, cap);
+        *(uint4*)&tile[r * 32 + ((c ^ (r >> 4)) << 2)] = w;
     }
     __syncthreads();
+    const int ic = t & 7, jq = t >> 3;                // source rows 16 ic .. 16 ic + 15, source columns 4 jq .. 4 jq + 3
+    uint32_t w[16];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const int j = j0 + ty * 4 + k, i = i0 + tx * 4;               // output row j (old column), columns i..i+3
-        if (j < n_g && i < ld) {
-            uint32_t w = 0;
+    for (int m = 0; m < 16; ++m) w[m] = tile[(16 * ic + m) * 32 + (jq ^ (ic << 2))];
 #pragma unroll
-            for (int b = 0; b < 4; ++b) w |= (uint32_t)tile[tx * 4 + b][ty * 4 + k] << (8 * b);
-            *(uint32_t*)(spd_t + base + (int64_t)j * ld + i) = w;
+    for (int b = 0; b < 4; ++b) {                     // output row j0 + 4 jq + b = source column; 16 bytes = 16 source rows
+        const int j = j0 + 4 * jq + b;
+        uint32_t o[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t lo = __byte_perm(w[4 * k], w[4 * k + 1], 0x0040 + b * 0x0011);      // byte b of two words
+            const uint32_t hi = __byte_perm(w[4 * k + 2], w[4 * k + 3], 0x0040 + b * 0x0011);
+            o[k] = __byte_perm(lo, hi, 0x5410);
         }
+        if (j < n_g && i0 + 16 * ic < ld)
+            *(uint4*)(spd_t + base + (int64_t)j * ld + i0 + 16 * ic) = make_uint4(o[0], o[1], o[2], o[3]);
     }
 }
 
@@ -761,7 +772,7 @@ extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void
     GT_CUDA_TRY(cudaMemsetAsync(ws + wsp.db_off, 0, (size_t)n_db * sizeof(double), s));
     GT_CUDA_TRY(cudaMemsetAsync(ws + wsp.dq_off, 0, rows * head_dim * sizeof(float), s));
     {
-        const unsigned tiles = (unsigned)((batch->max_seqlen + 63) / 64);
+        const unsigned tiles = (unsigned)((batch->max_seqlen + 127) / 128);
         dim3 tgrid(tiles, tiles, (unsigned)batch->n_graphs);
         spd_transpose_clamp_kernel<<<tgrid, 256, 0, s>>>(spd, spd_t, p.spd_offsets, p.cu_seqlens, batch->n_total,
                                                          (uint32_t)(max_dist + 1));
