@@ -129,6 +129,38 @@ def chunk_lse(q: np.ndarray, k: np.ndarray, spd: np.ndarray, bias: np.ndarray,
 # ----------------------------------------------------------------------------------
 # Packed batches: block-diagonal attention, one shared bias table, dB summed over graphs.
 # ----------------------------------------------------------------------------------
+def backward_chunked(q: np.ndarray, k: np.ndarray, v: np.ndarray, dout: np.ndarray, out: np.ndarray,
+                     lse: np.ndarray, spd: np.ndarray, bias: np.ndarray, bounds: Sequence[Tuple[int, int]]):
+    """Backward pass of Eq. 1 taken one key/value chunk at a time, the way a ring step of the
+    paper's context parallelism sees it (Sec. GA-CP): the step holds the key rows [a, b) only, plus
+    the forward results `out` [n,H,d] and `lse` [H,n] of the WHOLE row.  With
+        P_ij = exp(S_ij - lse_i),  Delta_i = dout_i . out_i,  dS_ij = P_ij (dout_i . v_j - Delta_i)   for j in [a, b)
+    a chunk yields dK, dV of its own rows completely, and its share of dQ and dB.  One graph.
+    Returns dQ [n,H,d] (sum over chunks), dK, dV [n,H,d], dB [H,nb] (sum) and dB_c [C,H,nb]."""
+    n, H, d = q.shape
+    nb = bias.shape[1]
+    inv_sqrt_d = 1.0 / np.sqrt(float(d))
+    dq = np.zeros((n, H, d))
+    dk = np.zeros((n, H, d))
+    dv = np.zeros((n, H, d))
+    db_c = np.zeros((len(bounds), H, nb))
+    for c, (a, b) in enumerate(bounds):
+        if b <= a:
+            continue
+        idx = spd[:n, a:b].astype(np.int64).reshape(-1)
+        for h in range(H):
+            s = (q[:, h, :] @ k[a:b, h, :].T) * inv_sqrt_d + bias[h][spd[:n, a:b]]
+            p = np.exp(s - lse[h][:, None])
+            do = dout[:, h, :]
+            delta = (do * out[:, h, :]).sum(axis=1, keepdims=True)
+            ds = p * (do @ v[a:b, h, :].T - delta)
+            dv[a:b, h, :] = p.T @ do
+            dk[a:b, h, :] = (ds.T @ q[:, h, :]) * inv_sqrt_d
+            dq[:, h, :] += (ds @ k[a:b, h, :]) * inv_sqrt_d
+            db_c[c, h] = np.bincount(idx, weights=ds.reshape(-1), minlength=nb)[:nb]
+    return dq, dk, dv, db_c.sum(axis=0), db_c
+
+
 def _spd_block(spd_packed: np.ndarray, spd_offsets: np.ndarray, g: int, n_g: int) -> np.ndarray:
     ld = (n_g + 15) // 16 * 16
     a = int(spd_offsets[g])

@@ -262,3 +262,26 @@ def test_compact_spd_rows_match_full():
     gc = oattn.backward_single(q, k, v, do, np.ascontiguousarray(spd[rows]), b, rows=rows, compact_spd=True)
     for x, y in zip(ga, gc):
         np.testing.assert_array_equal(x, y)
+
+
+def test_backward_chunked_sums_to_full_and_chunks_own_their_key_rows():
+    n = 150
+    q, k, v, do, spd, b = make_case(n, 2, 32, 6, seed=23, directed=True)
+    out, lse = oattn.forward_single(q, k, v, spd, b)
+    full = oattn.backward_single(q, k, v, do, spd, b)
+    bounds = [(0, 64), (64, 128), (128, 150), (150, 150)]
+    dq, dk, dv, db, db_c = oattn.backward_chunked(q, k, v, do, out, lse, spd, b, bounds)
+    for got, ref in zip((dq, dk, dv, db), full):
+        np.testing.assert_allclose(got, ref, rtol=1e-10, atol=1e-13)
+    assert db_c.shape == (4, 2, b.shape[1]) and (db_c[3] == 0).all()
+    # a chunk's bias gradient only sees its own key columns: brute force one bucket of one chunk
+    h, c, (a_, b_) = 1, 1, bounds[1]
+    s = (q[:, h] @ k[:, h].T) / np.sqrt(32.0) + b[h][spd[:, :n].astype(int)]
+    p = np.exp(s - lse[h][:, None])
+    ds = p * (do[:, h] @ v[:, h].T - (do[:, h] * out[:, h]).sum(1, keepdims=True))
+    bucket = int(spd[3, 70])
+    mask = spd[:, a_:b_] == bucket
+    np.testing.assert_allclose(db_c[c, h, bucket], ds[:, a_:b_][mask].sum(), rtol=1e-10, atol=1e-13)
+    # rows of dS sum to zero over ALL key columns, so the per-head total of dB vanishes only once every chunk is in
+    np.testing.assert_allclose(db.sum(axis=1), 0.0, atol=1e-10)
+    assert np.abs(db_c[:3].sum(axis=2)).min() > 1e-6
