@@ -258,6 +258,25 @@ def run_cuda(args) -> int:
     value = flops_all / (fb_ms * 1e-3) / 1e12
     spd_alg_bytes = float(b.spd_bytes + 4 * (T + 1) + 4 * ci.numel())
 
+    # ---- the chunked backward (a "next" row: the ring-step view of the backward), timed on its own after the step loop ----
+    bwd_chunked = None
+    if single:
+        ws_bc = gt._workspace(gt.gt_biased_attn_bwd_chunked_workspace(batch, H, d, D, n_chunks), dev)
+        gt.gt_biased_attn_bwd_chunked(q, k, v, out, do, lse, spd, bias, batch, D, n_chunks, dq, dk, dv, dbias, None, ws_bc)
+        torch.cuda.synchronize()
+        b0, b1 = ev(), ev()
+        n_bc = max(1, min(args.steps, 3))
+        b0.record()
+        for _ in range(n_bc):
+            gt.gt_biased_attn_bwd_chunked(q, k, v, out, do, lse, spd, bias, batch, D, n_chunks, dq, dk, dv, dbias, None, ws_bc)
+        b1.record()
+        torch.cuda.synchronize()
+        gt.gt_check(ws_bc)
+        bc_ms = b0.elapsed_time(b1) / n_bc
+        bwd_chunked = {"ms": bc_ms, "tflops": f_bwd / (bc_ms * 1e-3) / 1e12, "n_kv_chunks": n_chunks, "runs": n_bc,
+                       "note": "outside the timed step; one launch of the backward kernel per key chunk"}
+        del ws_bc
+
     # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region ----
     host_in = {name: x.cpu().pin_memory() for name, x in
                (("q", q), ("k", k), ("v", v), ("do", do), ("bias", bias), ("rp", rp), ("ci", ci))}
@@ -350,6 +369,7 @@ def run_cuda(args) -> int:
         "phases_ms": {"spd_build": spd_ms, "fwd": fwd_ms, "bwd": bwd_ms, "fwd_chunked": chk_ms if single else None},
         "fwd_tflops": f_fwd / (fwd_ms * 1e-3) / 1e12, "bwd_tflops": bwd_tflops,
         "fwd_chunked_tflops": (f_fwd / (chk_ms * 1e-3) / 1e12) if single else None,
+        "bwd_chunked": bwd_chunked,
         "spd_build_gbs": roofline_spd["achieved"],
         "pct_of_bf16_peak": {"burst": 100 * value / world / float(peaks["bf16_tflops"]),
                              "sustained": 100 * value / world / peak_tf, "nominal_2250": 100 * value / world / 2250.0},

@@ -162,6 +162,28 @@ gt_status gt_biased_attn_bwd(const void* q, const void* k, const void* v, const 
                              void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------
+ * gt_biased_attn_bwd_chunked -- the backward pass taken one key/value chunk at a time, the view a
+ * ring step of graph-aware context parallelism has (Sec. GA-CP; the paper trains through it but
+ * does not spell the backward out): a step holds the key rows of one chunk, the queries, and the
+ * forward results `out` and `lse` of the WHOLE row.  With the chunks of gt_biased_attn_fwd_chunked
+ * (w = round_up(ceil(N / n_kv_chunks), 128) rows, the last may be short or empty) and
+ *     P_ij = exp(S_ij - lse_i),  dS_ij = P_ij (dout_i . v_j - dout_i . out_i)      for j in the chunk,
+ * a chunk completes dk and dv of its own rows and adds its share to dq and dbias; the chunks run
+ * one after the other in stream order.  Results equal gt_biased_attn_bwd up to rounding.
+ * Single graph only (n_graphs == 1).  dbias_chunks: optional fp32 [n_kv_chunks, n_heads,
+ * max_dist+2] receiving each chunk's share of dbias (zeros for empty chunks), or NULL.
+ * ------------------------------------------------------------------------------------- */
+size_t gt_biased_attn_bwd_chunked_workspace(const gt_batch* batch, int32_t n_heads, int32_t head_dim,
+                                            int32_t max_dist, int32_t n_kv_chunks);
+gt_status gt_biased_attn_bwd_chunked(const void* q, const void* k, const void* v, const void* out,
+                                     const void* dout, const float* lse,
+                                     const uint8_t* spd, const float* bias,
+                                     const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                     int32_t n_kv_chunks,
+                                     void* dq, void* dk, void* dv, float* dbias, float* dbias_chunks,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------
  * gt_biased_attn_fwd_chunked -- single-GPU analogue of graph-aware context parallelism
  * (Sec. GA-CP: ring steps over KV blocks; Eq. 2: the bias columns of each block are taken at
  * the block's global node indices; item 3: bias folded in before the softmax statistics).

@@ -25,7 +25,8 @@ EXPORTS = ("gt_status_string", "gt_check",
            "gt_spd_build_workspace", "gt_spd_build", "gt_spd_build_static_limit", "gt_spd_build_static",
            "gt_biased_attn_fwd_workspace", "gt_biased_attn_fwd",
            "gt_biased_attn_bwd_workspace", "gt_biased_attn_bwd",
-           "gt_biased_attn_fwd_chunked_workspace", "gt_biased_attn_fwd_chunked")
+           "gt_biased_attn_fwd_chunked_workspace", "gt_biased_attn_fwd_chunked",
+           "gt_biased_attn_bwd_chunked_workspace", "gt_biased_attn_bwd_chunked")
 
 
 class GtError(RuntimeError):
@@ -80,6 +81,10 @@ def lib() -> ctypes.CDLL:
             L.gt_biased_attn_fwd_chunked_workspace.argtypes = [bp, i32, i32, i32]
             L.gt_biased_attn_fwd_chunked.restype = ctypes.c_int
             L.gt_biased_attn_fwd_chunked.argtypes = [vp, vp, vp, vp, vp, vp, bp, i32, i32, i32, vp, vp, i32, vp, vp, sz, vp]
+            L.gt_biased_attn_bwd_chunked_workspace.restype = sz
+            L.gt_biased_attn_bwd_chunked_workspace.argtypes = [bp, i32, i32, i32, i32]
+            L.gt_biased_attn_bwd_chunked.restype = ctypes.c_int
+            L.gt_biased_attn_bwd_chunked.argtypes = [vp] * 8 + [bp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -216,4 +221,24 @@ def gt_biased_attn_fwd_chunked(q, k, v, spd, bias, batch: Batch, max_dist: int, 
                                           int(n_kv_chunks), _ptr(lse_chunks),
                                           _ptr(workspace), workspace.numel(), _stream())
     _raise(st, "gt_biased_attn_fwd_chunked")
+    return workspace
+
+
+def gt_biased_attn_bwd_chunked_workspace(batch: Batch, n_heads: int, head_dim: int, max_dist: int, n_kv_chunks: int) -> int:
+    b = batch.c_struct()
+    return int(lib().gt_biased_attn_bwd_chunked_workspace(ctypes.byref(b), n_heads, head_dim, max_dist, n_kv_chunks))
+
+
+def gt_biased_attn_bwd_chunked(q, k, v, out, dout, lse, spd, bias, batch: Batch, max_dist: int, n_kv_chunks: int,
+                               dq, dk, dv, dbias, dbias_chunks: Optional[torch.Tensor] = None,
+                               workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _, H, d = q.shape
+    if workspace is None:
+        workspace = _workspace(gt_biased_attn_bwd_chunked_workspace(batch, H, d, max_dist, n_kv_chunks), q.device)
+    b = batch.c_struct()
+    st = lib().gt_biased_attn_bwd_chunked(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(dout), _ptr(lse), _ptr(spd),
+                                          _ptr(bias), ctypes.byref(b), H, d, int(max_dist), int(n_kv_chunks),
+                                          _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dbias), _ptr(dbias_chunks),
+                                          _ptr(workspace), workspace.numel(), _stream())
+    _raise(st, "gt_biased_attn_bwd_chunked")
     return workspace

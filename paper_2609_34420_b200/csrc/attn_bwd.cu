@@ -72,6 +72,8 @@ struct BwdParams {
     int32_t n_heads;
     int32_t n_buckets;
     int32_t spd_tma;         // 1: single graph, SPD tiles come by TMA
+    int32_t kv_tile0;        // first key tile of this launch (chunked backward: one launch per key chunk)
+    int32_t kv_tile_end;     // one past its last key tile
     float c1;                // log2(e)/sqrt(d)
     float scale;             // 1/sqrt(d)
 };
@@ -142,8 +144,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     const int g = blockIdx.z;
     const int32_t node0 = p.cu_seqlens ? p.cu_seqlens[g] : 0;
     const int32_t n_g = p.cu_seqlens ? p.cu_seqlens[g + 1] - node0 : p.n_total;
-    const int32_t kv0 = (int32_t)blockIdx.y * kTile;
-    if (kv0 >= n_g) return;
+    const int32_t kv0 = ((int32_t)blockIdx.y + p.kv_tile0) * kTile;
+    if (kv0 >= n_g || (int32_t)blockIdx.y + p.kv_tile0 >= p.kv_tile_end) return;
     const int64_t ld = (int64_t)((n_g + 15) & ~15);
     const uint8_t* spd_g = p.spd_t + (p.spd_offsets ? p.spd_offsets[g] : 0);
     const int32_t n_q = (n_g + kTile - 1) / kTile;
@@ -661,12 +663,21 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ out, con
     ext[2 * idx + 1] = e1;
 }
 
-// dq = bf16(scale * dq_acc);  dbias = float(db_acc)
+// dq = bf16(scale * dq_acc);  dbias = float(sum over key chunks of db_acc), optionally each chunk's share too
 __global__ void bwd_finalize_kernel(const float* __restrict__ dq_acc, __nv_bfloat16* __restrict__ dq, size_t n_vec4,
-                                    float scale, const double* __restrict__ db_acc, float* __restrict__ dbias, int32_t n_db)
+                                    float scale, const double* __restrict__ db_acc, float* __restrict__ dbias, int32_t n_db,
+                                    int32_t n_chunks, float* __restrict__ dbias_chunks)
 {
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx < (size_t)n_db) dbias[idx] = (float)db_acc[idx];
+    if (idx < (size_t)n_db) {
+        double sum = 0.0;
+        for (int32_t c = 0; c < n_chunks; ++c) {
+            const double v = db_acc[(size_t)c * n_db + idx];
+            if (dbias_chunks) dbias_chunks[(size_t)c * n_db + idx] = (float)v;
+            sum += v;
+        }
+        dbias[idx] = (float)sum;
+    }
     if (idx >= n_vec4) return;
     const float4 v = ((const float4*)dq_acc)[idx];
     uint2 pk;
@@ -679,12 +690,12 @@ struct BwdWorkspace {
     size_t db_off, ext_off, dq_off, spdt_off, total;
 };
 
-BwdWorkspace bwd_workspace(const gt_batch* b, int32_t n_heads, int32_t head_dim, int32_t max_dist)
+BwdWorkspace bwd_workspace(const gt_batch* b, int32_t n_heads, int32_t head_dim, int32_t max_dist, int32_t n_chunks = 1)
 {
     BwdWorkspace w{};
     const size_t rows = (size_t)b->n_total * n_heads;
     w.db_off = kHeaderBytes;
-    w.ext_off = w.db_off + align_up((size_t)n_heads * (max_dist + 2) * sizeof(double), 256);
+    w.ext_off = w.db_off + align_up((size_t)n_chunks * n_heads * (max_dist + 2) * sizeof(double), 256);
     w.dq_off = w.ext_off + align_up(rows * kExtCols * 2, 256);
     w.spdt_off = w.dq_off + align_up(rows * head_dim * sizeof(float), 256);
     // transposed SPD copy: at most sum n_g * round_up(n_g,16) <= n_total * round_up(max_seqlen,16) bytes
@@ -697,7 +708,10 @@ gt_status launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtenso
                      const CUtensorMap& text, const CUtensorMap& tspd, const BwdParams& p,
                      const gt_batch* batch, cudaStream_t s)
 {
-    dim3 grid((unsigned)p.n_heads, (unsigned)((batch->max_seqlen + kTile - 1) / kTile), (unsigned)batch->n_graphs);
+    const int32_t all_tiles = (batch->max_seqlen + kTile - 1) / kTile;
+    const int32_t tile_end = p.kv_tile_end < all_tiles ? p.kv_tile_end : all_tiles;
+    if (tile_end <= p.kv_tile0) return GT_OK;                 // empty key chunk
+    dim3 grid((unsigned)p.n_heads, (unsigned)(tile_end - p.kv_tile0), (unsigned)batch->n_graphs);
     CUtensorMap tdq;
     gt_status st_map = encode_dq_map(&tdq, p.dq_acc, p.n_total, p.n_heads, D);
     if (st_map != GT_OK) return st_map;
@@ -720,12 +734,15 @@ extern "C" size_t gt_biased_attn_bwd_workspace(const gt_batch* batch, int32_t n_
     return gt::bwd_workspace(batch, n_heads, head_dim, max_dist).total;
 }
 
-extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void* v, const void* out,
-                                        const void* dout, const float* lse,
-                                        const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
-                                        const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
-                                        void* dq, void* dk, void* dv, float* dbias,
-                                        void* workspace, size_t workspace_bytes, void* stream)
+// Shared by the one-shot and the chunked entry point: pre-passes, one launch of the main kernel per key chunk
+// (the chunks run one after the other in stream order, like ring steps; dQ and dB accumulate across them,
+// dK and dV of a chunk's rows are complete when its launch ends), then the final conversion.
+static gt_status gt_bwd_run(const void* q, const void* k, const void* v, const void* out,
+                            const void* dout, const float* lse,
+                            const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
+                            const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                            void* dq, void* dk, void* dv, float* dbias, int32_t n_kv_chunks, float* dbias_chunks,
+                            void* workspace, size_t workspace_bytes, void* stream)
 {
     using namespace gt;
     gt_status st = validate_attn_common(batch, n_heads, head_dim, max_dist, spd_offsets);
@@ -735,7 +752,7 @@ extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void
         misaligned16(spd) || misaligned16(dq) || misaligned16(dk) || misaligned16(dv))
         return GT_ERR_INVALID_ARG;
     if (n_heads > 65535 || batch->n_graphs > 65535) return GT_ERR_UNSUPPORTED;
-    const BwdWorkspace wsp = bwd_workspace(batch, n_heads, head_dim, max_dist);
+    const BwdWorkspace wsp = bwd_workspace(batch, n_heads, head_dim, max_dist, n_kv_chunks);
     if (workspace == nullptr || workspace_bytes < wsp.total || misaligned16(workspace)) return GT_ERR_WORKSPACE;
     if (sm_count() <= 0) return GT_ERR_NO_DEVICE;
 
@@ -769,7 +786,7 @@ extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void
     p.scale = 1.0f / sqrtf((float)head_dim);
     p.c1 = kLog2e * p.scale;
 
-    GT_CUDA_TRY(cudaMemsetAsync(ws + wsp.db_off, 0, (size_t)n_db * sizeof(double), s));
+    GT_CUDA_TRY(cudaMemsetAsync(ws + wsp.db_off, 0, (size_t)n_kv_chunks * n_db * sizeof(double), s));
     GT_CUDA_TRY(cudaMemsetAsync(ws + wsp.dq_off, 0, rows * head_dim * sizeof(float), s));
     {
         const unsigned tiles = (unsigned)((batch->max_seqlen + 127) / 128);
@@ -789,13 +806,55 @@ extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void
     GT_CUDA_TRY(cudaGetLastError());
     CUtensorMap text;
     if ((st = encode_thd_map(&text, ext, batch->n_total, n_heads, kExtCols)) != GT_OK) return st;
-    st = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, text, tspd, p, batch, s)
-                        : launch_bwd<32>(tq, tk, tv, tdo, text, tspd, p, batch, s);
-    if (st != GT_OK) return st;
+    // key chunks of w = round_up(ceil(N / C), 128) rows, as in the chunked forward
+    const int32_t all_tiles = (batch->max_seqlen + kTile - 1) / kTile;
+    const int32_t tiles_per_chunk = ((batch->max_seqlen + n_kv_chunks - 1) / n_kv_chunks + kTile - 1) / kTile;
+    double* db_base = p.db_acc;
+    for (int32_t c = 0; c < n_kv_chunks; ++c) {
+        p.db_acc = db_base + (size_t)c * n_db;
+        p.kv_tile0 = n_kv_chunks == 1 ? 0 : c * tiles_per_chunk;
+        p.kv_tile_end = n_kv_chunks == 1 ? all_tiles : (c + 1) * tiles_per_chunk;
+        st = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, text, tspd, p, batch, s)
+                            : launch_bwd<32>(tq, tk, tv, tdo, text, tspd, p, batch, s);
+        if (st != GT_OK) return st;
+    }
+    p.db_acc = db_base;
     const size_t n_vec4 = rows * head_dim / 4;
     const size_t n_fin = n_vec4 > (size_t)n_db ? n_vec4 : (size_t)n_db;
     bwd_finalize_kernel<<<(unsigned)((n_fin + 255) / 256), 256, 0, s>>>(p.dq_acc, (__nv_bfloat16*)dq, n_vec4, p.scale,
-                                                                         p.db_acc, dbias, n_db);
+                                                                         p.db_acc, dbias, n_db, n_kv_chunks, dbias_chunks);
     GT_CUDA_TRY(cudaGetLastError());
     return GT_OK;
+}
+
+extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void* v, const void* out,
+                                        const void* dout, const float* lse,
+                                        const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
+                                        const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                        void* dq, void* dk, void* dv, float* dbias,
+                                        void* workspace, size_t workspace_bytes, void* stream)
+{
+    return gt_bwd_run(q, k, v, out, dout, lse, spd, spd_offsets, bias, batch, n_heads, head_dim, max_dist,
+                      dq, dk, dv, dbias, 1, nullptr, workspace, workspace_bytes, stream);
+}
+
+extern "C" size_t gt_biased_attn_bwd_chunked_workspace(const gt_batch* batch, int32_t n_heads, int32_t head_dim,
+                                                       int32_t max_dist, int32_t n_kv_chunks)
+{
+    if (gt::validate_batch(batch) != GT_OK || n_heads < 1 || max_dist < 1 || max_dist > 254 || n_kv_chunks < 1) return 0;
+    return gt::bwd_workspace(batch, n_heads, head_dim, max_dist, n_kv_chunks).total;
+}
+
+extern "C" gt_status gt_biased_attn_bwd_chunked(const void* q, const void* k, const void* v, const void* out,
+                                                const void* dout, const float* lse,
+                                                const uint8_t* spd, const float* bias,
+                                                const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                                int32_t n_kv_chunks,
+                                                void* dq, void* dk, void* dv, float* dbias, float* dbias_chunks,
+                                                void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (batch == nullptr || batch->n_graphs != 1) return GT_ERR_UNSUPPORTED;
+    if (n_kv_chunks < 1 || n_kv_chunks > 4096) return GT_ERR_INVALID_ARG;
+    return gt_bwd_run(q, k, v, out, dout, lse, spd, nullptr, bias, batch, n_heads, head_dim, max_dist,
+                      dq, dk, dv, dbias, n_kv_chunks, dbias_chunks, workspace, workspace_bytes, stream);
 }

@@ -80,6 +80,16 @@ class DeviceCase:
         gt.gt_check(ws)
         return out, lse, cl
 
+    def backward_chunked(self, out, lse, n_chunks, want_chunk_dbias=False):
+        dq, dk, dv = (torch.full_like(self.q, float("nan")) for _ in range(3))
+        dbias = torch.full_like(self.bias, float("nan"))
+        dbc = torch.full((n_chunks,) + tuple(self.bias.shape), float("nan"), dtype=torch.float32,
+                         device=self.q.device) if want_chunk_dbias else None
+        ws = gt.gt_biased_attn_bwd_chunked(self.q, self.k, self.v, out, self.dout, lse, self.spd, self.bias, self.batch,
+                                           self.w.max_dist, n_chunks, dq, dk, dv, dbias, dbc)
+        gt.gt_check(ws)
+        return dq, dk, dv, dbias, dbc
+
     def backward(self, out, lse, dout=None):
         dout = self.dout if dout is None else dout
         dq, dk, dv = (torch.full_like(self.q, float("nan")) for _ in range(3))

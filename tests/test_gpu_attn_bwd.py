@@ -100,3 +100,47 @@ def test_rows_with_zero_dout_do_not_contribute():
     mask = np.ones(600, bool)
     mask[rows] = False
     assert (to_f64(dq)[mask] == 0).all()
+
+
+# ---- chunked backward (one key/value chunk at a time) ----
+CHUNK_REL_L2 = 1e-3
+
+
+def chunk_bounds(n, n_chunks):
+    w = ((n + n_chunks - 1) // n_chunks + 127) // 128 * 128
+    return [(min(c * w, n), min((c + 1) * w, n)) for c in range(n_chunks)]
+
+
+@pytest.mark.parametrize("n,chunks,d", [(300, 1, 64), (300, 2, 64), (300, 3, 32), (1000, 8, 64), (129, 4, 32), (2000, 5, 64)])
+def test_chunked_backward_matches_unchunked_and_the_chunk_oracle(n, chunks, d):
+    w = wl.small_workload([n], 2, d, 6, seed=n + chunks, avg_degree=2.0, directed=True)     # asymmetric SPD
+    case = DeviceCase(w)
+    out, lse = case.forward()
+    full = case.backward(out, lse)
+    dq, dk, dv, db, dbc = case.backward_chunked(out, lse, chunks, want_chunk_dbias=True)
+    for name, got, ref in zip(("dq", "dk", "dv", "dbias"), (dq, dk, dv, db), full):
+        assert rel_l2(to_f64(got), to_f64(ref)) <= CHUNK_REL_L2, name
+    # against the oracle's chunk-by-chunk backward (fed with the oracle's own forward results)
+    q, k, v, do, b = case.host_f64()
+    spd = np.asarray(case.spd_host).reshape(n, -1)
+    ro, rl = oattn.forward_single(q, k, v, spd, b)
+    rdq, rdk, rdv, rdb, rdbc = oattn.backward_chunked(q, k, v, do, ro, rl, spd, b, chunk_bounds(n, chunks))
+    for name, got, ref in (("dq", dq, rdq), ("dk", dk, rdk), ("dv", dv, rdv), ("dbias", db, rdb)):
+        assert rel_l2(to_f64(got), ref) <= GRAD_REL_L2, name
+    g = to_f64(dbc)
+    assert np.isfinite(g).all()
+    for c, (a_, b_) in enumerate(chunk_bounds(n, chunks)):
+        if b_ <= a_:
+            assert (g[c] == 0).all()                      # empty chunk
+        else:
+            assert rel_l2(g[c], rdbc[c]) <= GRAD_REL_L2, c
+    np.testing.assert_allclose(g.sum(axis=0), to_f64(db), rtol=1e-5, atol=1e-6)
+
+
+def test_chunked_backward_is_refused_for_packed_batches():
+    from paper_2609_34420_b200 import binding as gt
+    w = wl.small_workload([100, 60], 2, 32, 4, seed=1)
+    case = DeviceCase(w)
+    out, lse = case.forward()
+    with pytest.raises(gt.GtError):
+        case.backward_chunked(out, lse, 2)

@@ -76,6 +76,16 @@ def run_large(name: str, n_slab: int, full_spd_oracle: bool):
     mask[rows_t] = False
     assert (dq[mask].float().abs().max().item() == 0.0)
 
+    # ---- chunked backward (same dO): equals the unchunked backward, chunk shares add up ----
+    C = max(w.n_kv_chunks, 2)
+    dq_c, dk_c, dv_c = (torch.empty_like(q) for _ in range(3))
+    dbias_c = torch.empty_like(bias)
+    db_chunks = torch.empty((C,) + tuple(bias.shape), device=dev)
+    gt.gt_check(gt.gt_biased_attn_bwd_chunked(q, k, v, out, do_masked, lse, spd, bias, bt, D, C, dq_c, dk_c, dv_c, dbias_c, db_chunks))
+    for got, ref_ in ((dq_c, dq), (dk_c, dk), (dv_c, dv), (dbias_c, dbias)):
+        assert rel_l2(to_f64(got), to_f64(ref_)) <= CHUNK_REL_L2
+    assert rel_l2(to_f64(db_chunks.sum(0)), to_f64(dbias_c)) <= 1e-5
+
 
 def test_powerlaw16k_full_spd_and_row_slab_attention():
     run_large("powerlaw16k", n_slab=384, full_spd_oracle=True)
