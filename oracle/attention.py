@@ -129,6 +129,44 @@ def chunk_lse(q: np.ndarray, k: np.ndarray, spd: np.ndarray, bias: np.ndarray,
 # ----------------------------------------------------------------------------------
 # Packed batches: block-diagonal attention, one shared bias table, dB summed over graphs.
 # ----------------------------------------------------------------------------------
+def attend_key_set(q: np.ndarray, k: np.ndarray, v: np.ndarray, spd: np.ndarray, bias: np.ndarray,
+                   rows: np.ndarray, keys: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Attention of the query rows `rows` over the key subset `keys` only (one graph), with the bias
+    taken at the GLOBAL key indices (Eq. 2: Score_local = Q_i K_j^T + b_i[:, Indices(K_j)]).
+    Returns the normalised output [r,H,d] and LSE [H,r] of that subset (LSE = -inf, output 0 if empty)."""
+    rows, keys = np.asarray(rows), np.asarray(keys)
+    n, H, d = q.shape
+    o = np.zeros((len(rows), H, d))
+    lse = np.full((H, len(rows)), -np.inf)
+    if len(keys) == 0:
+        return o, lse
+    inv_sqrt_d = 1.0 / np.sqrt(float(d))
+    b_idx = spd[np.ix_(rows, keys)].astype(np.int64)
+    for h in range(H):
+        s = (q[rows, h, :] @ k[keys, h, :].T) * inv_sqrt_d + bias[h][b_idx]
+        m = s.max(axis=1, keepdims=True)
+        e = np.exp(s - m)
+        l = e.sum(axis=1, keepdims=True)
+        o[:, h, :] = (e / l) @ v[keys, h, :]
+        lse[h] = (m + np.log(l))[:, 0]
+    return o, lse
+
+
+def merge_state(o_acc: np.ndarray, lse_acc: np.ndarray, o_new: np.ndarray, lse_new: np.ndarray):
+    """Online-softmax state carried between ring steps (Sec. GA-CP, item 3), in its normalised form:
+    (running_max m, running_sum l, unnormalised accumulator A) is kept as lse = m + log l and o = A / l.
+    Merging a step's result:  lse' = log(exp lse + exp lse_new),  o' = (exp(lse - lse') o + exp(lse_new - lse') o_new)."""
+    m = np.maximum(lse_acc, lse_new)
+    safe = np.where(np.isneginf(m), 0.0, m)
+    wa, wb = np.exp(lse_acc - safe), np.exp(lse_new - safe)
+    tot = wa + wb
+    lse = np.where(tot > 0, safe + np.log(np.where(tot > 0, tot, 1.0)), -np.inf)
+    fa = np.where(tot > 0, wa / np.where(tot > 0, tot, 1.0), 0.0)
+    fb = np.where(tot > 0, wb / np.where(tot > 0, tot, 1.0), 0.0)
+    o = fa.T[:, :, None] * o_acc + fb.T[:, :, None] * o_new
+    return o, lse
+
+
 def backward_chunked(q: np.ndarray, k: np.ndarray, v: np.ndarray, dout: np.ndarray, out: np.ndarray,
                      lse: np.ndarray, spd: np.ndarray, bias: np.ndarray, bounds: Sequence[Tuple[int, int]]):
     """Backward pass of Eq. 1 taken one key/value chunk at a time, the way a ring step of the

@@ -285,3 +285,31 @@ def test_backward_chunked_sums_to_full_and_chunks_own_their_key_rows():
     # rows of dS sum to zero over ALL key columns, so the per-head total of dB vanishes only once every chunk is in
     np.testing.assert_allclose(db.sum(axis=1), 0.0, atol=1e-10)
     assert np.abs(db_c[:3].sum(axis=2)).min() > 1e-6
+
+
+def test_ring_steps_with_two_part_key_slices_merge_to_the_full_forward():
+    # 3 "ranks" of regular nodes plus a block of super nodes at the end of the index range; every step's key
+    # block is a regular range plus (once only) the super-node range: two-part slicing of the bias columns
+    n, n_super = 150, 22
+    q, k, v, do, spd, b = make_case(n, 2, 32, 6, seed=31, directed=True)
+    ro, rl = oattn.forward_single(q, k, v, spd, b)
+    n_reg = n - n_super
+    shards = [(0, 48), (48, 96), (96, n_reg)]
+    rows = np.arange(16, 130)
+    o = np.zeros((len(rows), 2, 32)); lse = np.full((2, len(rows)), -np.inf)
+    for step, (a_, b_) in enumerate(shards):
+        keys = np.concatenate([np.arange(a_, b_), np.arange(n_reg, n) if step == 1 else np.arange(0)])
+        po, pl = oattn.attend_key_set(q, k, v, spd, b, rows, keys)
+        o, lse = oattn.merge_state(o, lse, po, pl)
+    np.testing.assert_allclose(o, ro[rows], rtol=1e-10, atol=1e-13)
+    np.testing.assert_allclose(lse, rl[:, rows], rtol=1e-12)
+    # a key subset's LSE by brute force, bias at the global column
+    h, i = 1, 5
+    keys = np.concatenate([np.arange(48, 96), np.arange(n_reg, n)])
+    s = (q[rows[i], h] @ k[keys, h].T) / np.sqrt(32.0) + b[h][spd[rows[i], keys].astype(int)]
+    _, pl = oattn.attend_key_set(q, k, v, spd, b, rows, keys)
+    np.testing.assert_allclose(pl[h, i], np.log(np.exp(s).sum()), rtol=1e-12)
+    # merging with an empty step changes nothing; merging into the empty state returns the step
+    eo, el = oattn.attend_key_set(q, k, v, spd, b, rows, np.arange(0))
+    o2, l2 = oattn.merge_state(o, lse, eo, el)
+    np.testing.assert_array_equal(o2, o); np.testing.assert_array_equal(l2, lse)
