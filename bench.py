@@ -277,6 +277,40 @@ def run_cuda(args) -> int:
                        "note": "outside the timed step; one launch of the backward kernel per key chunk"}
         del ws_bc
 
+    # ---- caller-driven ring steps (a "next" row): 8 ranks x 8 steps, two-part key slices, carried state ----
+    fwd_ring = None
+    if single and T >= 8192:
+        n_ranks, n_super = 8, 1024
+        n_reg = T - n_super
+        share = (n_reg // n_ranks + 15) // 16 * 16
+        shards = [(r * share, min((r + 1) * share, n_reg)) for r in range(n_ranks)]
+        o_acc = torch.zeros(T, H, d, dtype=torch.float32, device=dev)
+        lse_acc = torch.empty(H, T, dtype=torch.float32, device=dev)
+        ws_st = gt._workspace(gt.gt_biased_attn_fwd_step_workspace(batch, H, d), dev)
+
+        def ring():
+            o_acc.zero_()
+            lse_acc.fill_(float("-inf"))
+            for rank, (qa, qb) in enumerate(shards + [(n_reg, T)]):
+                for st_ in range(n_ranks):
+                    ka, kb = shards[(rank + st_) % n_ranks]
+                    gt.gt_biased_attn_fwd_step(q, k, v, spd, bias, batch, D, (qa, qb), (ka, kb),
+                                               (n_reg, T) if st_ == 0 else (0, 0), o_acc, lse_acc, None, ws_st)
+        ring()
+        torch.cuda.synchronize()
+        r0, r1 = ev(), ev()
+        r0.record()
+        ring()
+        r1.record()
+        torch.cuda.synchronize()
+        gt.gt_check(ws_st)
+        ring_ms = r0.elapsed_time(r1)
+        fwd_ring = {"ms": ring_ms, "tflops": f_fwd / (ring_ms * 1e-3) / 1e12, "ranks": n_ranks, "super_nodes": n_super,
+                    "steps": (n_ranks + 1) * n_ranks,
+                    "max_abs_vs_forward": float((o_acc - out.float()).abs().max().item()),
+                    "note": "outside the timed step; every rank's query shard (and the super nodes' rows) sees all key blocks once"}
+        del o_acc, lse_acc, ws_st
+
     # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region ----
     host_in = {name: x.cpu().pin_memory() for name, x in
                (("q", q), ("k", k), ("v", v), ("do", do), ("bias", bias), ("rp", rp), ("ci", ci))}
@@ -369,7 +403,7 @@ def run_cuda(args) -> int:
         "phases_ms": {"spd_build": spd_ms, "fwd": fwd_ms, "bwd": bwd_ms, "fwd_chunked": chk_ms if single else None},
         "fwd_tflops": f_fwd / (fwd_ms * 1e-3) / 1e12, "bwd_tflops": bwd_tflops,
         "fwd_chunked_tflops": (f_fwd / (chk_ms * 1e-3) / 1e12) if single else None,
-        "bwd_chunked": bwd_chunked,
+        "bwd_chunked": bwd_chunked, "fwd_ring_steps": fwd_ring,
         "spd_build_gbs": roofline_spd["achieved"],
         "pct_of_bf16_peak": {"burst": 100 * value / world / float(peaks["bf16_tflops"]),
                              "sustained": 100 * value / world / peak_tf, "nominal_2250": 100 * value / world / 2250.0},

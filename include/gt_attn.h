@@ -162,6 +162,31 @@ gt_status gt_biased_attn_bwd(const void* q, const void* k, const void* v, const 
                              void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------
+ * gt_biased_attn_fwd_step -- one ring step of graph-aware context parallelism driven by the caller
+ * (Sec. GA-CP, items 1-3): the query rows [q_begin, q_end) of a rank attend to ONE incoming key/value
+ * block, which is the union of a regular-node range [kv_begin0, kv_end0) and a super-node range
+ * [kv_begin1, kv_end1) (either may be empty); the bias columns are taken at those GLOBAL indices
+ * (Eq. 2, the two-part slice of the rank's bias shard) and folded in before the softmax statistics.
+ * The online-softmax state of the rows is carried in normalised form: with running max m, running
+ * sum l and unnormalised accumulator A, the caller holds  lse_acc = m + log l  (fp32 [H, N]) and
+ * o_acc = A / l  (fp32 [N, H, d]); start with lse_acc = -inf and o_acc = 0.  The step updates both
+ * for the rows of the range only:  lse' = log(exp lse + sum_r exp lse_r),  o' = the matching convex
+ * combination.  After the last step o_acc is the attention output and lse_acc its LSE.
+ * q, k, v, spd: the tensors of the whole single graph (n_graphs == 1), as for gt_biased_attn_fwd.
+ * out: optional bf16 [N, H, d]; its rows [q_begin, q_end) receive bf16(o_acc) after the step.
+ * A key range must start at a multiple of 16 (else GT_ERR_UNSUPPORTED); ranges of one row's steps
+ * must not overlap (a key seen twice is counted twice).
+ * ------------------------------------------------------------------------------------- */
+size_t gt_biased_attn_fwd_step_workspace(const gt_batch* batch, int32_t n_heads, int32_t head_dim);
+gt_status gt_biased_attn_fwd_step(const void* q, const void* k, const void* v,
+                                  const uint8_t* spd, const float* bias,
+                                  const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                  int32_t q_begin, int32_t q_end,
+                                  int32_t kv_begin0, int32_t kv_end0, int32_t kv_begin1, int32_t kv_end1,
+                                  float* o_acc, float* lse_acc, void* out,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------
  * gt_biased_attn_bwd_chunked -- the backward pass taken one key/value chunk at a time, the view a
  * ring step of graph-aware context parallelism has (Sec. GA-CP; the paper trains through it but
  * does not spell the backward out): a step holds the key rows of one chunk, the queries, and the

@@ -26,7 +26,8 @@ EXPORTS = ("gt_status_string", "gt_check",
            "gt_biased_attn_fwd_workspace", "gt_biased_attn_fwd",
            "gt_biased_attn_bwd_workspace", "gt_biased_attn_bwd",
            "gt_biased_attn_fwd_chunked_workspace", "gt_biased_attn_fwd_chunked",
-           "gt_biased_attn_bwd_chunked_workspace", "gt_biased_attn_bwd_chunked")
+           "gt_biased_attn_bwd_chunked_workspace", "gt_biased_attn_bwd_chunked",
+           "gt_biased_attn_fwd_step_workspace", "gt_biased_attn_fwd_step")
 
 
 class GtError(RuntimeError):
@@ -81,6 +82,10 @@ def lib() -> ctypes.CDLL:
             L.gt_biased_attn_fwd_chunked_workspace.argtypes = [bp, i32, i32, i32]
             L.gt_biased_attn_fwd_chunked.restype = ctypes.c_int
             L.gt_biased_attn_fwd_chunked.argtypes = [vp, vp, vp, vp, vp, vp, bp, i32, i32, i32, vp, vp, i32, vp, vp, sz, vp]
+            L.gt_biased_attn_fwd_step_workspace.restype = sz
+            L.gt_biased_attn_fwd_step_workspace.argtypes = [bp, i32, i32]
+            L.gt_biased_attn_fwd_step.restype = ctypes.c_int
+            L.gt_biased_attn_fwd_step.argtypes = [vp] * 5 + [bp, i32, i32, i32] + [i32] * 6 + [vp, vp, vp, vp, sz, vp]
             L.gt_biased_attn_bwd_chunked_workspace.restype = sz
             L.gt_biased_attn_bwd_chunked_workspace.argtypes = [bp, i32, i32, i32, i32]
             L.gt_biased_attn_bwd_chunked.restype = ctypes.c_int
@@ -241,4 +246,25 @@ def gt_biased_attn_bwd_chunked(q, k, v, out, dout, lse, spd, bias, batch: Batch,
                                           _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dbias), _ptr(dbias_chunks),
                                           _ptr(workspace), workspace.numel(), _stream())
     _raise(st, "gt_biased_attn_bwd_chunked")
+    return workspace
+
+
+def gt_biased_attn_fwd_step_workspace(batch: Batch, n_heads: int, head_dim: int) -> int:
+    b = batch.c_struct()
+    return int(lib().gt_biased_attn_fwd_step_workspace(ctypes.byref(b), n_heads, head_dim))
+
+
+def gt_biased_attn_fwd_step(q, k, v, spd, bias, batch: Batch, max_dist: int, q_range, kv_range0, kv_range1,
+                            o_acc, lse_acc, out: Optional[torch.Tensor] = None,
+                            workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _, H, d = q.shape
+    if workspace is None:
+        workspace = _workspace(gt_biased_attn_fwd_step_workspace(batch, H, d), q.device)
+    b = batch.c_struct()
+    st = lib().gt_biased_attn_fwd_step(_ptr(q), _ptr(k), _ptr(v), _ptr(spd), _ptr(bias), ctypes.byref(b), H, d,
+                                       int(max_dist), int(q_range[0]), int(q_range[1]),
+                                       int(kv_range0[0]), int(kv_range0[1]), int(kv_range1[0]), int(kv_range1[1]),
+                                       _ptr(o_acc), _ptr(lse_acc), _ptr(out),
+                                       _ptr(workspace), workspace.numel(), _stream())
+    _raise(st, "gt_biased_attn_fwd_step")
     return workspace

@@ -73,6 +73,10 @@ struct FwdParams {
     int32_t n_heads;
     int32_t n_buckets;
     int32_t kv_chunk_rows;     // chunked: keys per chunk (multiple of 128)
+    int32_t use_ranges;        // step entry point: key ranges given explicitly, one per grid z
+    int32_t range_begin[2];
+    int32_t range_end[2];
+    int32_t q_block0;          // first 256-row query block of the launch
     int32_t spd_tma;           // 1: single graph, SPD tiles come by TMA; 0: cp.async loader warp
     float c1;                  // log2(e) / sqrt(d)
 };
@@ -145,12 +149,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 
     const int32_t node0 = p.cu_seqlens ? p.cu_seqlens[g] : 0;
     const int32_t n_g = p.cu_seqlens ? p.cu_seqlens[g + 1] - node0 : p.n_total;
-    const int32_t q0 = (int32_t)blockIdx.y * kRowsPerCta;
+    const int32_t q0 = ((int32_t)blockIdx.y + p.q_block0) * kRowsPerCta;
     if (q0 >= n_g) return;
     const int64_t ld = (int64_t)((n_g + 15) & ~15);
     const uint8_t* spd_g = p.spd + (p.spd_offsets ? p.spd_offsets[g] : 0);
-    const int32_t kv_begin = kPartial ? chunk * p.kv_chunk_rows : 0;
-    const int32_t kv_end = kPartial ? min(n_g, kv_begin + p.kv_chunk_rows) : n_g;
+    const int32_t kv_begin = kPartial ? (p.use_ranges ? p.range_begin[chunk] : chunk * p.kv_chunk_rows) : 0;
+    const int32_t kv_end = kPartial ? (p.use_ranges ? p.range_end[chunk] : min(n_g, kv_begin + p.kv_chunk_rows)) : n_g;
     const int32_t n_kv = kv_end > kv_begin ? (kv_end - kv_begin + kKvTile - 1) / kKvTile : 0;
 
     if (kPartial && n_kv == 0) {            // empty chunk: weight zero in the merge
@@ -578,6 +582,57 @@ __global__ void chunk_merge_kernel(const float* __restrict__ part_o, const float
     if (v == 0) lse[(size_t)h * n_total + row] = mx + logf(den);
 }
 
+// One ring step's merge: the carried state (normalised accumulator o_acc, lse_acc) of the query rows
+// [q_begin, q_end) absorbs up to two partial results (the step's regular key range and its super-node
+// range):  lse' = log sum exp(lse_i),  o' = sum exp(lse_i - lse') o_i.  Rows with nothing to attend to yet
+// keep lse = -inf, o = 0.  One thread per (row, head, 4 channels).
+template <int D>
+__global__ void step_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse, int32_t n_parts,
+                                  float* __restrict__ o_acc, float* __restrict__ lse_acc, __nv_bfloat16* __restrict__ out,
+                                  int32_t q_begin, int32_t q_end, int32_t n_total, int32_t n_heads)
+{
+    constexpr int kVec = D / 4;
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t n_rows = (size_t)(q_end - q_begin) * n_heads;
+    if (idx >= n_rows * kVec) return;
+    const size_t rh = idx / kVec;
+    const int v = (int)(idx % kVec);
+    const int32_t row = q_begin + (int32_t)(rh / n_heads), h = (int32_t)(rh % n_heads);
+    const float l0 = lse_acc[(size_t)h * n_total + row];
+    float mx = l0;
+    for (int c = 0; c < n_parts; ++c) mx = fmaxf(mx, part_lse[((size_t)c * n_heads + h) * n_total + row]);
+    float4* acc_ptr = (float4*)(o_acc + ((size_t)row * n_heads + h) * D + v * 4);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float den = 0.f;
+    if (mx != -INFINITY) {
+        if (l0 != -INFINITY) {
+            const float w = exp2f((l0 - mx) * kLog2e);
+            const float4 o = *acc_ptr;
+            den += w;
+            acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+        }
+        for (int c = 0; c < n_parts; ++c) {
+            const float lc = part_lse[((size_t)c * n_heads + h) * n_total + row];
+            if (lc == -INFINITY) continue;
+            const float w = exp2f((lc - mx) * kLog2e);
+            const float4 o = *(const float4*)(part_o + (((size_t)c * n_total + row) * n_heads + h) * D + v * 4);
+            den += w;
+            acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+        }
+        const float inv = 1.0f / den;
+        acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+    }
+    *acc_ptr = acc;
+    if (out) {
+        uint2 pk;
+        pk.x = pack_bf16x2(acc.x, acc.y);
+        pk.y = pack_bf16x2(acc.z, acc.w);
+        *(uint2*)(out + ((size_t)row * n_heads + h) * D + v * 4) = pk;
+    }
+    __syncwarp();
+    if (v == 0) lse_acc[(size_t)h * n_total + row] = mx == -INFINITY ? -INFINITY : mx + logf(den);
+}
+
 int32_t chunk_rows(int32_t n, int32_t n_chunks)
 {
     int32_t w = (n + n_chunks - 1) / n_chunks;
@@ -586,11 +641,11 @@ int32_t chunk_rows(int32_t n, int32_t n_chunks)
 
 template <int D, bool kPartial>
 gt_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tspd,
-                     const FwdParams& p, const gt_batch* batch, int grid_z, cudaStream_t s)
+                     const FwdParams& p, const gt_batch* batch, int grid_z, cudaStream_t s, int grid_y = 0)
 {
     auto kern = p.n_buckets <= 32 ? attn_fwd_kernel<D, kPartial, true> : attn_fwd_kernel<D, kPartial, false>;
     GT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kDynamic));
-    dim3 grid((unsigned)p.n_heads, (unsigned)((batch->max_seqlen + kRowsPerCta - 1) / kRowsPerCta), (unsigned)grid_z);
+    dim3 grid((unsigned)p.n_heads, (unsigned)(grid_y > 0 ? grid_y : (batch->max_seqlen + kRowsPerCta - 1) / kRowsPerCta), (unsigned)grid_z);
     kern<<<grid, kFwdThreads, FwdSmem<D>::kDynamic, s>>>(tq, tk, tv, tspd, p);
     GT_CUDA_TRY(cudaGetLastError());
     return GT_OK;
@@ -707,6 +762,74 @@ extern "C" gt_status gt_biased_attn_fwd_chunked(const void* q, const void* k, co
     else
         chunk_merge_kernel<32><<<blocks, 256, 0, s>>>(p.part_o, p.part_lse, (__nv_bfloat16*)out, lse, lse_chunks,
                                                       batch->n_total, n_heads, n_kv_chunks);
+    GT_CUDA_TRY(cudaGetLastError());
+    return GT_OK;
+}
+
+extern "C" size_t gt_biased_attn_fwd_step_workspace(const gt_batch* batch, int32_t n_heads, int32_t head_dim)
+{
+    return gt_biased_attn_fwd_chunked_workspace(batch, n_heads, head_dim, 2);
+}
+
+extern "C" gt_status gt_biased_attn_fwd_step(const void* q, const void* k, const void* v,
+                                             const uint8_t* spd, const float* bias,
+                                             const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                             int32_t q_begin, int32_t q_end,
+                                             int32_t kv_begin0, int32_t kv_end0, int32_t kv_begin1, int32_t kv_end1,
+                                             float* o_acc, float* lse_acc, void* out,
+                                             void* workspace, size_t workspace_bytes, void* stream)
+{
+    using namespace gt;
+    gt_status st = validate_attn_common(batch, n_heads, head_dim, max_dist, nullptr);
+    if (st != GT_OK) return st;
+    if (!q || !k || !v || !spd || !bias || !o_acc || !lse_acc) return GT_ERR_INVALID_ARG;
+    if (misaligned16(q) || misaligned16(k) || misaligned16(v) || misaligned16(spd) || misaligned16(o_acc) || (out && misaligned16(out)))
+        return GT_ERR_INVALID_ARG;
+    if (batch->n_graphs != 1 || n_heads > 65535) return GT_ERR_UNSUPPORTED;
+    const int32_t n = batch->n_total;
+    if (q_begin < 0 || q_end > n || q_begin >= q_end) return GT_ERR_INVALID_ARG;
+    if (kv_begin0 < 0 || kv_end0 > n || kv_begin0 > kv_end0 || kv_begin1 < 0 || kv_end1 > n || kv_begin1 > kv_end1) return GT_ERR_INVALID_ARG;
+    // a key range starts at a multiple of 16: the SPD tile of a range is fetched by TMA from that column
+    if ((kv_begin0 & 15) || (kv_begin1 & 15)) return GT_ERR_UNSUPPORTED;
+    const size_t need = gt_biased_attn_fwd_step_workspace(batch, n_heads, head_dim);
+    if (workspace == nullptr || workspace_bytes < need || misaligned16(workspace)) return GT_ERR_WORKSPACE;
+    if (sm_count() <= 0) return GT_ERR_NO_DEVICE;
+    CUtensorMap tq, tk, tv, tspd;
+    if ((st = encode_thd_map(&tq, q, n, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&tk, k, n, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&tv, v, n, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_spd_map(&tspd, spd, n, 256)) != GT_OK) return st;
+    const size_t rows = (size_t)n * n_heads;
+    uint8_t* ws = (uint8_t*)workspace;
+    FwdParams p{};
+    p.spd_tma = 1;
+    p.spd = spd;
+    p.bias = bias;
+    p.part_lse = (float*)(ws + kHeaderBytes);
+    p.part_o = (float*)(ws + kHeaderBytes + align_up((size_t)2 * rows * sizeof(float), 256));
+    p.status = (uint32_t*)workspace;
+    p.n_total = n;
+    p.n_heads = n_heads;
+    p.n_buckets = max_dist + 2;
+    p.use_ranges = 1;
+    p.range_begin[0] = kv_begin0; p.range_end[0] = kv_end0;
+    p.range_begin[1] = kv_begin1; p.range_end[1] = kv_end1;
+    const int n_parts = kv_end1 > kv_begin1 ? 2 : 1;
+    p.q_block0 = q_begin / kRowsPerCta;
+    const int grid_y = (q_end - 1) / kRowsPerCta - p.q_block0 + 1;
+    p.c1 = kLog2e / sqrtf((float)head_dim);
+    cudaStream_t s = (cudaStream_t)stream;
+    st = head_dim == 64 ? launch_fwd<64, true>(tq, tk, tv, tspd, p, batch, n_parts, s, grid_y)
+                        : launch_fwd<32, true>(tq, tk, tv, tspd, p, batch, n_parts, s, grid_y);
+    if (st != GT_OK) return st;
+    const size_t n_thr = (size_t)(q_end - q_begin) * n_heads * (head_dim / 4);
+    const unsigned blocks = (unsigned)((n_thr + 255) / 256);
+    if (head_dim == 64)
+        step_merge_kernel<64><<<blocks, 256, 0, s>>>(p.part_o, p.part_lse, n_parts, o_acc, lse_acc, (__nv_bfloat16*)out,
+                                                     q_begin, q_end, n, n_heads);
+    else
+        step_merge_kernel<32><<<blocks, 256, 0, s>>>(p.part_o, p.part_lse, n_parts, o_acc, lse_acc, (__nv_bfloat16*)out,
+                                                     q_begin, q_end, n, n_heads);
     GT_CUDA_TRY(cudaGetLastError());
     return GT_OK;
 }

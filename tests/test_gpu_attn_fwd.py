@@ -125,3 +125,50 @@ def test_rejects_unsupported_shapes():
     with pytest.raises(gt.GtError) as e:
         gt.gt_biased_attn_fwd_chunked(multi.q, multi.k, multi.v, multi.spd, multi.bias, multi.batch, 4, o2, l2, 2)
     assert e.value.status == 2
+
+
+# ---- caller-driven ring steps: two-part key slices and carried state ----
+def test_ring_steps_with_super_nodes_reproduce_the_forward_and_the_step_oracle():
+    from paper_2609_34420_b200 import binding as gt
+    n, n_super, ranks = 1500, 60, 3                  # super nodes at the end of the index range
+    w = wl.small_workload([n], 2, 64, 6, seed=77, avg_degree=2.0, directed=True)
+    case = DeviceCase(w)
+    out_ref, lse_ref = case.forward()
+    n_reg = n - n_super
+    share = (n_reg // ranks + 15) // 16 * 16          # regular nodes per rank (ranges start at multiples of 16)
+    shards = [(r * share, min((r + 1) * share, n_reg)) for r in range(ranks)]
+    dev = case.q.device
+    o_acc = torch.zeros(n, 2, 64, dtype=torch.float32, device=dev)
+    lse_acc = torch.full((2, n), float("-inf"), dtype=torch.float32, device=dev)
+    out = torch.full_like(case.q, float("nan"))
+    q64, k64, v64, _, b64 = case.host_f64()
+    spd = np.asarray(case.spd_host).reshape(n, -1)
+    ws = None
+    for rank, (qa, qb) in enumerate(shards + [(n_reg, n)]):           # the super nodes' own rows: a fourth "rank"
+        rows = np.arange(qa, qb)
+        so = np.zeros((len(rows), 2, 64)); sl = np.full((2, len(rows)), -np.inf)
+        for step in range(ranks):                                      # KV blocks arrive round the ring
+            ka, kb = shards[(rank + step) % ranks]
+            sup = (n_reg, n) if step == 0 else (0, 0)                  # the replicated super nodes are attended to once
+            ws = gt.gt_biased_attn_fwd_step(case.q, case.k, case.v, case.spd, case.bias, case.batch, w.max_dist,
+                                            (qa, qb), (ka, kb), sup, o_acc, lse_acc, out, ws)
+            keys = np.concatenate([np.arange(ka, kb), np.arange(*sup)])
+            po, pl = oattn.attend_key_set(q64, k64, v64, spd, b64, rows, keys)
+            so, sl = oattn.merge_state(so, sl, po, pl)
+            # the carried state after every step matches the oracle's
+            assert np.abs(lse_acc[:, qa:qb].cpu().numpy().astype(np.float64) - sl).max() <= LSE_MAX_ABS
+            assert np.abs(o_acc[qa:qb].cpu().numpy().astype(np.float64) - so).max() <= O_MAX_ABS
+    gt.gt_check(ws)
+    assert rel_l2(to_f64(out), to_f64(out_ref)) <= CHUNK_REL_L2
+    assert (lse_acc - lse_ref).abs().max().item() <= LSE_MAX_ABS
+    ro, rl = oracle_forward(case)
+    assert (np.abs(to_f64(out) - ro) <= np.maximum(O_MAX_ABS, np.abs(ro) * 2.0 ** -7)).all()
+
+
+def test_step_rejects_unaligned_key_ranges_and_packed_batches():
+    from paper_2609_34420_b200 import binding as gt
+    w = wl.small_workload([300], 2, 32, 4, seed=3)
+    case = DeviceCase(w)
+    o_acc = torch.zeros(300, 2, 32, device=case.q.device); lse_acc = torch.full((2, 300), float("-inf"), device=case.q.device)
+    with pytest.raises(gt.GtError):
+        gt.gt_biased_attn_fwd_step(case.q, case.k, case.v, case.spd, case.bias, case.batch, 4, (0, 300), (8, 100), (0, 0), o_acc, lse_acc)
