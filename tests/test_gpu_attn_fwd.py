@@ -172,3 +172,26 @@ def test_step_rejects_unaligned_key_ranges_and_packed_batches():
     o_acc = torch.zeros(300, 2, 32, device=case.q.device); lse_acc = torch.full((2, 300), float("-inf"), device=case.q.device)
     with pytest.raises(gt.GtError):
         gt.gt_biased_attn_fwd_step(case.q, case.k, case.v, case.spd, case.bias, case.batch, 4, (0, 300), (8, 100), (0, 0), o_acc, lse_acc)
+
+
+def test_ring_driver_with_the_device_step_on_one_rank():
+    # world size 1: the ring degenerates to the rank's own block, which exercises the device step wrapper
+    # (block -> global rows copy, two-part key slice, state) end to end; the multi-rank schedule is tested on CPU ranks
+    from paper_2609_34420_b200 import binding as gt, ring
+    n, n_super = 700, 44
+    w = wl.small_workload([n], 2, 32, 5, seed=9, avg_degree=2.0)
+    case = DeviceCase(w)
+    out_ref, lse_ref = case.forward()
+    layout = ring.RingLayout.even(n, n_super, 1)
+    (a, b), (sa, sb) = layout.shards[0], layout.super_range
+    dev = case.q.device
+    k_full, v_full = torch.zeros_like(case.k), torch.zeros_like(case.v)       # filled by the arriving blocks only
+    k_blk = torch.cat([case.k[a:b], case.k[sa:sb]]); v_blk = torch.cat([case.v[a:b], case.v[sa:sb]])
+    o_acc = torch.zeros(n, 2, 32, dtype=torch.float32, device=dev)
+    lse_acc = torch.full((2, n), float("-inf"), dtype=torch.float32, device=dev)
+    out = torch.full_like(case.q, float("nan"))
+    step = ring.device_step(gt, case.q, k_full, v_full, case.spd, case.bias, case.batch, w.max_dist, layout, o_acc, lse_acc, out)
+    ring.ring_forward(layout, k_blk, v_blk, step, rank=0, world=1)
+    torch.cuda.synchronize()
+    assert rel_l2(to_f64(out), to_f64(out_ref)) <= CHUNK_REL_L2
+    assert (lse_acc - lse_ref).abs().max().item() <= LSE_MAX_ABS

@@ -1,0 +1,98 @@
+"""Ring schedule of graph-aware context parallelism on CPU ranks (gloo, world size 3): every rank
+drives `ring.ring_forward` with a step function built from the oracle, and the gathered result
+must equal the one-shot forward.  Checks which block is where at which step, the two-part key
+slices (super nodes once), and the carried state — not the CUDA kernels."""
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch
+import torch.multiprocessing as mp
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+N, N_SUPER, H, D_HEAD, MAX_DIST = 150, 22, 2, 32, 6
+
+
+def _case():
+    from paper_2609_34420_b200 import workloads as wl
+    w = wl.small_workload([N], H, D_HEAD, MAX_DIST, seed=5, avg_degree=2.0, directed=True)
+    t = w.tensors()
+    f = wl.bf16_bits_to_f64
+    from oracle import spd as ospd
+    spd = ospd.spd_matrix(w.batch.row_ptr, w.batch.col_idx, MAX_DIST)
+    return f(t.q), f(t.k), f(t.v), spd, t.bias.astype(np.float64)
+
+
+def _worker(rank, world, port, out_q):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    import torch.distributed as dist
+    from oracle import attention as oattn
+    from paper_2609_34420_b200 import ring
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    q, k, v, spd, bias = _case()
+    layout = ring.RingLayout.even(N, N_SUPER, world)
+    a, b = layout.shards[rank]
+    share = max(e - s for s, e in layout.shards)
+    sa, sb = layout.super_range
+
+    def block(x):                                   # own regular rows (padded to the common length) + super nodes
+        blk = np.zeros((share + N_SUPER,) + x.shape[1:])
+        blk[: b - a] = x[a:b]
+        blk[share:] = x[sa:sb]
+        return torch.from_numpy(blk)
+
+    o = np.zeros((N, H, D_HEAD)); lse = np.full((H, N), -np.inf)
+    seen = []
+
+    def step(q_range, kv_range, sup, k_blk, v_blk, owner):
+        # rebuild the key rows of this step from the ARRIVED block only (what a rank really holds)
+        ka, kb = kv_range
+        kk, vv = np.zeros_like(k), np.zeros_like(v)
+        kk[ka:kb] = k_blk.numpy()[: kb - ka]; vv[ka:kb] = v_blk.numpy()[: kb - ka]
+        kk[sa:sb] = k_blk.numpy()[share:]; vv[sa:sb] = v_blk.numpy()[share:]
+        keys = np.concatenate([np.arange(ka, kb), np.arange(*sup)])
+        rows = np.arange(*q_range)
+        po, pl = oattn.attend_key_set(q, kk, vv, spd, bias, rows, keys)
+        o[rows], lse[:, rows] = oattn.merge_state(o[rows], lse[:, rows], po, pl)
+        seen.append((q_range, owner))
+
+    ring.ring_forward(layout, block(k), block(v), step)
+    out_q.put((rank, o[a:b], lse[:, a:b], o[sa:sb], lse[:, sa:sb], seen))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_three_rank_ring_reproduces_the_forward():
+    world = 3
+    ctx = mp.get_context("spawn")
+    out_q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, out_q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted((out_q.get(timeout=180) for _ in range(world)), key=lambda r: r[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    from oracle import attention as oattn
+    from paper_2609_34420_b200 import ring
+    q, k, v, spd, bias = _case()
+    ro, rl = oattn.forward_single(q, k, v, spd, bias)
+    layout = ring.RingLayout.even(N, N_SUPER, world)
+    sa, sb = layout.super_range
+    for rank, o_sh, l_sh, o_sup, l_sup, seen in res:
+        a, b = layout.shards[rank]
+        np.testing.assert_allclose(o_sh, ro[a:b], rtol=1e-10, atol=1e-13)
+        np.testing.assert_allclose(l_sh, rl[:, a:b], rtol=1e-12)
+        np.testing.assert_allclose(o_sup, ro[sa:sb], rtol=1e-10, atol=1e-13)      # every rank's replica of the super rows
+        np.testing.assert_allclose(l_sup, rl[:, sa:sb], rtol=1e-12)
+        owners = [own for (qr, own) in seen if qr == layout.shards[rank]]
+        assert owners == [(rank - s) % world for s in range(world)]               # blocks arrive round the ring
