@@ -199,6 +199,36 @@ def backward_chunked(q: np.ndarray, k: np.ndarray, v: np.ndarray, dout: np.ndarr
     return dq, dk, dv, db_c.sum(axis=0), db_c
 
 
+def backward_block(q: np.ndarray, k: np.ndarray, v: np.ndarray, dout: np.ndarray, out: np.ndarray,
+                   lse: np.ndarray, spd: np.ndarray, bias: np.ndarray, rows: np.ndarray, keys: np.ndarray):
+    """What one rank adds at one ring step of the backward (Sec. GA-CP): the pairs (i, j) with i in `rows`
+    (the rank's queries) and j in `keys` (the block it holds), given the forward results of the whole rows:
+        P_ij = exp(S_ij - lse_i),  dS_ij = P_ij (dout_i . v_j - dout_i . out_i)
+    Returns the UNSCALED sums  dq_part [r,H,d] = sum_j dS_ij k_j,  dk_part [m,H,d] = sum_i dS_ij q_i,
+    dv_part [m,H,d] = sum_i P_ij dout_i  and db_part [H,nb]; dQ = dq / sqrt(d) and dK = dk / sqrt(d) once
+    all blocks are in.  One graph."""
+    rows, keys = np.asarray(rows), np.asarray(keys)
+    n, H, d = q.shape
+    nb = bias.shape[1]
+    dq = np.zeros((len(rows), H, d)); dk = np.zeros((len(keys), H, d)); dv = np.zeros((len(keys), H, d))
+    db = np.zeros((H, nb))
+    if len(rows) == 0 or len(keys) == 0:
+        return dq, dk, dv, db
+    inv_sqrt_d = 1.0 / np.sqrt(float(d))
+    idx = spd[np.ix_(rows, keys)].astype(np.int64)
+    for h in range(H):
+        s = (q[rows, h, :] @ k[keys, h, :].T) * inv_sqrt_d + bias[h][idx]
+        p = np.exp(s - lse[h][rows][:, None])
+        do = dout[rows, h, :]
+        delta = (do * out[rows, h, :]).sum(axis=1, keepdims=True)
+        ds = p * (do @ v[keys, h, :].T - delta)
+        dq[:, h, :] = ds @ k[keys, h, :]
+        dk[:, h, :] = ds.T @ q[rows, h, :]
+        dv[:, h, :] = p.T @ do
+        db[h] = np.bincount(idx.reshape(-1), weights=ds.reshape(-1), minlength=nb)[:nb]
+    return dq, dk, dv, db
+
+
 def _spd_block(spd_packed: np.ndarray, spd_offsets: np.ndarray, g: int, n_g: int) -> np.ndarray:
     ld = (n_g + 15) // 16 * 16
     a = int(spd_offsets[g])

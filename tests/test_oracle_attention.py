@@ -313,3 +313,27 @@ def test_ring_steps_with_two_part_key_slices_merge_to_the_full_forward():
     eo, el = oattn.attend_key_set(q, k, v, spd, b, rows, np.arange(0))
     o2, l2 = oattn.merge_state(o, lse, eo, el)
     np.testing.assert_array_equal(o2, o); np.testing.assert_array_equal(l2, lse)
+
+
+def test_backward_blocks_over_a_partition_of_rows_and_keys_sum_to_the_full_backward():
+    n = 150
+    q, k, v, do, spd, b = make_case(n, 2, 32, 6, seed=41, directed=True)
+    out, lse = oattn.forward_single(q, k, v, spd, b)
+    full = oattn.backward_single(q, k, v, do, spd, b)
+    row_parts = [np.arange(0, 48), np.arange(48, 128), np.arange(128, 150)]
+    key_parts = [np.arange(0, 64), np.concatenate([np.arange(64, 100), np.arange(130, 150)]), np.arange(100, 130)]
+    dq = np.zeros_like(q); dk = np.zeros_like(q); dv = np.zeros_like(q); db = np.zeros_like(b)
+    for rows in row_parts:
+        for keys in key_parts:
+            pq, pk, pv, pb = oattn.backward_block(q, k, v, do, out, lse, spd, b, rows, keys)
+            dq[rows] += pq; dk[keys] += pk; dv[keys] += pv; db += pb
+    s = 1.0 / np.sqrt(32.0)
+    for got, ref in zip((dq * s, dk * s, dv, db), full):
+        np.testing.assert_allclose(got, ref, rtol=1e-10, atol=1e-13)
+    # one block's dv by brute force
+    rows, keys = row_parts[1], key_parts[1]
+    _, _, pv, _ = oattn.backward_block(q, k, v, do, out, lse, spd, b, rows, keys)
+    h, jj = 1, 40                                   # key 130 + (40 - 36)
+    j = keys[jj]
+    sc = (q[rows, h] @ k[j, h]) / np.sqrt(32.0) + b[h][spd[rows, j].astype(int)]
+    np.testing.assert_allclose(pv[jj, h], (np.exp(sc - lse[h][rows])[:, None] * do[rows, h]).sum(0), rtol=1e-10, atol=1e-13)
