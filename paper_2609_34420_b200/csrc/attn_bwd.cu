@@ -72,8 +72,12 @@ struct BwdParams {
     int32_t n_heads;
     int32_t n_buckets;
     int32_t spd_tma;         // 1: single graph, SPD tiles come by TMA
-    int32_t kv_tile0;        // first key tile of this launch (chunked backward: one launch per key chunk)
-    int32_t kv_tile_end;     // one past its last key tile
+    int32_t kv_row0;         // key rows [kv_row0, kv_row_end) of a graph are this launch's (chunked / step entry points)
+    int32_t kv_row_end;
+    int32_t q_row0;          // query rows [q_row0, q_row_end) take part (step entry point; else the whole graph)
+    int32_t q_row_end;
+    float* dk_acc;           // step entry point: unscaled fp32 sums [T,H,D] that this launch ADDS to (else dk / dv are written)
+    float* dv_acc;
     float c1;                // log2(e)/sqrt(d)
     float scale;             // 1/sqrt(d)
 };
@@ -144,11 +148,14 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     const int g = blockIdx.z;
     const int32_t node0 = p.cu_seqlens ? p.cu_seqlens[g] : 0;
     const int32_t n_g = p.cu_seqlens ? p.cu_seqlens[g + 1] - node0 : p.n_total;
-    const int32_t kv0 = ((int32_t)blockIdx.y + p.kv_tile0) * kTile;
-    if (kv0 >= n_g || (int32_t)blockIdx.y + p.kv_tile0 >= p.kv_tile_end) return;
+    const int32_t kv0 = p.kv_row0 + (int32_t)blockIdx.y * kTile;
+    const int32_t kv_lim = min(n_g, p.kv_row_end);
+    if (kv0 >= kv_lim) return;
+    const int32_t q_lo = p.q_row0, q_hi = min(n_g, p.q_row_end);
+    if (q_hi <= q_lo) return;
     const int64_t ld = (int64_t)((n_g + 15) & ~15);
     const uint8_t* spd_g = p.spd_t + (p.spd_offsets ? p.spd_offsets[g] : 0);
-    const int32_t n_q = (n_g + kTile - 1) / kTile;
+    const int32_t n_q = (q_hi - q_lo + kTile - 1) / kTile;
 
     uint64_t* bars = (uint64_t*)(smem + L::kBars);
     uint32_t* misc = (uint32_t*)(smem + L::kMisc);
@@ -217,7 +224,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 const int s = i & 1;
                 mbar_wait(bar(kBarStageEmpty + s), ((i >> 1) & 1) ^ 1, abort_flag, p.status, 110);
                 if (lane == 0) {
-                    const int32_t row = node0 + i * kTile;
+                    const int32_t row = node0 + q_lo + i * kTile;
                     mbar_arrive_expect_tx(bar(kBarQdoFull + s), 2 * L::kTileBytes + kExtTileBytes);
                     tma_load_3d(smem_u32(smem + L::kQ + s * L::kStageBytes), &tmap_q, bar(kBarQdoFull + s), 0, h, row);
                     tma_load_3d(smem_u32(smem + L::kDo + s * L::kStageBytes), &tmap_do, bar(kBarQdoFull + s), 0, h, row);
@@ -228,13 +235,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 if (p.spd_tma) {
                     if (lane == 0) {
                         mbar_arrive_expect_tx(bar(kBarSpdFull), L::kSpdBytes);
-                        tma_load_2d(smem_u32(smem + L::kSpd), &tmap_spd, bar(kBarSpdFull), i * kTile, kv0);
+                        tma_load_2d(smem_u32(smem + L::kSpd), &tmap_spd, bar(kBarSpdFull), q_lo + i * kTile, kv0);
                     }
                     __syncwarp();
                 } else {
                     // packed batch (per-graph pitch): cp.async in the layout of the TMA 128-byte swizzle,
                     // 16-byte chunk c of row r at chunk c ^ (r & 7)
-                    const int32_t q0 = i * kTile;
+                    const int32_t q0 = q_lo + i * kTile;
                     const uint32_t dst0 = smem_u32(smem + L::kSpd);
 #pragma unroll 4
                     for (int it = 0; it < (kTile * 8) / 32; ++it) {
@@ -343,7 +350,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + half * 128 + (grp & 1) * 32 + lane_off;
         const uint32_t tDp = tS + kHalf;
-        const bool kv_valid = kv0 + r < n_g;
+        const bool kv_valid = kv0 + r < kv_lim;
         const uint64_t c1c1 = pack_f32x2(p.c1, p.c1);
         const float tbl = s_bias[lane];
         float* my_bins = s_bins + (kPrivateBins ? st : lane);
@@ -410,7 +417,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     pr[c + 1] = ex2_approx(hi);
                 }
             }
-            const int nq_valid = n_g - i * kTile - grp * 32;      // valid query columns of this group
+            const int nq_valid = q_hi - q_lo - i * kTile - grp * 32;      // valid query columns of this group
             if (!kv_valid || nq_valid < 32) {
 #pragma unroll
                 for (int c = 0; c < 32; ++c)
@@ -498,7 +505,19 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             uint32_t o[kOC];
             if constexpr (kOC == 32) tmem_ld32(tacc, o); else tmem_ld16(tacc, o);
             tmem_wait_ld();
-            if (kv_valid) {
+            float* acc_base = half == 0 ? p.dv_acc : p.dk_acc;
+            if (kv_valid && acc_base != nullptr) {
+                // step entry point: this launch's share is added to the caller's unscaled fp32 sums (a key row belongs
+                // to one CTA of the launch, launches are ordered by the stream: plain read-modify-write)
+                float4* dst = (float4*)(acc_base + ((size_t)(node0 + kv0 + r) * p.n_heads + h) * D + ch * kOC);
+#pragma unroll
+                for (int k = 0; k < kOC / 4; ++k) {
+                    float4 v = dst[k];
+                    v.x += __uint_as_float(o[4 * k]); v.y += __uint_as_float(o[4 * k + 1]);
+                    v.z += __uint_as_float(o[4 * k + 2]); v.w += __uint_as_float(o[4 * k + 3]);
+                    dst[k] = v;
+                }
+            } else if (kv_valid) {
                 uint4* dst = (uint4*)dst_base;
 #pragma unroll
                 for (int k = 0; k < kOC / 8; ++k) {
@@ -560,7 +579,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 named_barrier_sync(kNbDqStaged, 128);
                 if (warp == 20) {
                     if (elect_one()) {
-                        tma_reduce_add_2d(&tmap_dq, smem_u32(stg), h * D + c * 32, node0 + i * kTile);
+                        tma_reduce_add_2d(&tmap_dq, smem_u32(stg), h * D + c * 32, node0 + q_lo + i * kTile);
                         bulk_commit_group();
                     }
                     __syncwarp();
@@ -708,10 +727,9 @@ gt_status launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtenso
                      const CUtensorMap& text, const CUtensorMap& tspd, const BwdParams& p,
                      const gt_batch* batch, cudaStream_t s)
 {
-    const int32_t all_tiles = (batch->max_seqlen + kTile - 1) / kTile;
-    const int32_t tile_end = p.kv_tile_end < all_tiles ? p.kv_tile_end : all_tiles;
-    if (tile_end <= p.kv_tile0) return GT_OK;                 // empty key chunk
-    dim3 grid((unsigned)p.n_heads, (unsigned)(tile_end - p.kv_tile0), (unsigned)batch->n_graphs);
+    const int32_t kv_end = p.kv_row_end < batch->max_seqlen ? p.kv_row_end : batch->max_seqlen;
+    if (kv_end <= p.kv_row0 || p.q_row_end <= p.q_row0) return GT_OK;      // empty key chunk / no queries
+    dim3 grid((unsigned)p.n_heads, (unsigned)((kv_end - p.kv_row0 + kTile - 1) / kTile), (unsigned)batch->n_graphs);
     CUtensorMap tdq;
     gt_status st_map = encode_dq_map(&tdq, p.dq_acc, p.n_total, p.n_heads, D);
     if (st_map != GT_OK) return st_map;
@@ -812,8 +830,10 @@ static gt_status gt_bwd_run(const void* q, const void* k, const void* v, const v
     double* db_base = p.db_acc;
     for (int32_t c = 0; c < n_kv_chunks; ++c) {
         p.db_acc = db_base + (size_t)c * n_db;
-        p.kv_tile0 = n_kv_chunks == 1 ? 0 : c * tiles_per_chunk;
-        p.kv_tile_end = n_kv_chunks == 1 ? all_tiles : (c + 1) * tiles_per_chunk;
+        p.kv_row0 = n_kv_chunks == 1 ? 0 : c * tiles_per_chunk * kTile;
+        p.kv_row_end = n_kv_chunks == 1 ? all_tiles * kTile : (c + 1) * tiles_per_chunk * kTile;
+        p.q_row0 = 0;
+        p.q_row_end = all_tiles * kTile;
         st = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, text, tspd, p, batch, s)
                             : launch_bwd<32>(tq, tk, tv, tdo, text, tspd, p, batch, s);
         if (st != GT_OK) return st;
