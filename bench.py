@@ -311,6 +311,49 @@ def run_cuda(args) -> int:
                     "note": "outside the timed step; every rank's query shard (and the super nodes' rows) sees all key blocks once"}
         del o_acc, lse_acc, ws_st
 
+    # ---- the backward of the same ring (a "next" row): prepare + 8 x 8 + 8 step calls + finish ----
+    bwd_ring = None
+    if single and T >= 8192:
+        n_ranks, n_super = 8, 1024
+        n_reg = T - n_super
+        share = (n_reg // n_ranks + 15) // 16 * 16
+        shards = [(r * share, min((r + 1) * share, n_reg)) for r in range(n_ranks)]
+        accs = [torch.zeros(T, H, d, dtype=torch.float32, device=dev) for _ in range(3)]
+        db_acc = torch.zeros(H, D + 2, dtype=torch.float64, device=dev)
+        ctx = gt._workspace(gt.gt_biased_attn_bwd_step_context_bytes(batch, H, d), dev)
+        dq_r, dk_r, dv_r = (torch.empty_like(q) for _ in range(3))
+        dbias_r = torch.empty_like(bias)
+
+        def bwd_ring_pass():
+            for a_ in accs:
+                a_.zero_()
+            db_acc.zero_()
+            gt.gt_biased_attn_bwd_step_prepare(out, do, lse, spd, batch, D, ctx)
+            for rank, qr in enumerate(shards):
+                for st_ in range(n_ranks):
+                    gt.gt_biased_attn_bwd_step(q, k, v, do, bias, batch, D, qr, shards[(rank - st_) % n_ranks],
+                                               (n_reg, T) if st_ == 0 else (0, 0), accs[0], accs[1], accs[2], db_acc, ctx)
+                gt.gt_biased_attn_bwd_step(q, k, v, do, bias, batch, D, (n_reg, T), qr, (n_reg, T) if rank == 0 else (0, 0),
+                                           accs[0], accs[1], accs[2], db_acc, ctx)
+            gt.gt_biased_attn_bwd_step_finish(accs[0], accs[1], accs[2], db_acc, batch, D, dq_r, dk_r, dv_r, dbias_r)
+        bwd_ring_pass()
+        torch.cuda.synchronize()
+        r0, r1 = ev(), ev()
+        r0.record()
+        bwd_ring_pass()
+        r1.record()
+        torch.cuda.synchronize()
+        gt.gt_check(ctx)
+        ring_ms = r0.elapsed_time(r1)
+        gt.gt_biased_attn_bwd(q, k, v, out, do, lse, spd, bias, batch, D, dq, dk, dv, dbias, ws_bwd)
+        torch.cuda.synchronize()
+        rel = lambda x, y: float(((x.float() - y.float()).norm() / y.float().norm()).item())
+        bwd_ring = {"ms": ring_ms, "tflops": f_bwd / (ring_ms * 1e-3) / 1e12, "ranks": n_ranks, "super_nodes": n_super,
+                    "steps": n_ranks * n_ranks + n_ranks,
+                    "rel_l2_vs_backward": {"dq": rel(dq_r, dq), "dk": rel(dk_r, dk), "dv": rel(dv_r, dv), "dbias": rel(dbias_r, dbias)},
+                    "note": "outside the timed step; includes the prepare pass (SPD transpose) and the final conversion"}
+        del accs, ctx, dq_r, dk_r, dv_r
+
     # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region ----
     host_in = {name: x.cpu().pin_memory() for name, x in
                (("q", q), ("k", k), ("v", v), ("do", do), ("bias", bias), ("rp", rp), ("ci", ci))}
@@ -403,7 +446,7 @@ def run_cuda(args) -> int:
         "phases_ms": {"spd_build": spd_ms, "fwd": fwd_ms, "bwd": bwd_ms, "fwd_chunked": chk_ms if single else None},
         "fwd_tflops": f_fwd / (fwd_ms * 1e-3) / 1e12, "bwd_tflops": bwd_tflops,
         "fwd_chunked_tflops": (f_fwd / (chk_ms * 1e-3) / 1e12) if single else None,
-        "bwd_chunked": bwd_chunked, "fwd_ring_steps": fwd_ring,
+        "bwd_chunked": bwd_chunked, "fwd_ring_steps": fwd_ring, "bwd_ring_steps": bwd_ring,
         "spd_build_gbs": roofline_spd["achieved"],
         "pct_of_bf16_peak": {"burst": 100 * value / world / float(peaks["bf16_tflops"]),
                              "sustained": 100 * value / world / peak_tf, "nominal_2250": 100 * value / world / 2250.0},

@@ -209,6 +209,40 @@ gt_status gt_biased_attn_bwd_chunked(const void* q, const void* k, const void* v
                                      void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------
+ * gt_biased_attn_bwd_step_* -- the backward of one ring step of graph-aware context parallelism,
+ * driven by the caller (Sec. GA-CP; counterpart of gt_biased_attn_fwd_step).  A backward pass is
+ *   prepare  once: from the forward results of the whole rows (`out` bf16, `lse`) and `dout` it writes
+ *            the per-(query, head) terms and a transposed copy of `spd` into `context`
+ *            (gt_biased_attn_bwd_step_context_bytes bytes, device memory, kept until finish);
+ *   step     once per (query rows [q_begin, q_end), arriving key/value block = regular range
+ *            [kv_begin0, kv_end0) united with super-node range [kv_begin1, kv_end1), either may be
+ *            empty): for the pairs (i, j) of that block it ADDS, unscaled and in fp32,
+ *                dq_acc[i] += sum_j dS_ij k_j    dk_acc[j] += sum_i dS_ij q_i    dv_acc[j] += sum_i P_ij dout_i
+ *            ([N, H, d] each) and dbias_acc[h][b] += sum of dS over the block's pairs in bucket b
+ *            (fp64 [n_heads, max_dist+2]); the accumulators start at zero, dk_acc / dv_acc are the ones
+ *            that travel with the block, every pair must be visited exactly once;
+ *   finish   once: dq = bf16(dq_acc / sqrt(d)), dk = bf16(dk_acc / sqrt(d)), dv = bf16(dv_acc),
+ *            dbias = float(dbias_acc).
+ * q, k, v, dout: the tensors of the whole single graph (n_graphs == 1) at their global rows.
+ * q_begin must be a multiple of 16 (else GT_ERR_UNSUPPORTED).  The status word of the step calls
+ * lives in `context` (gt_check(context, stream)).
+ * ------------------------------------------------------------------------------------- */
+size_t gt_biased_attn_bwd_step_context_bytes(const gt_batch* batch, int32_t n_heads, int32_t head_dim);
+gt_status gt_biased_attn_bwd_step_prepare(const void* out, const void* dout, const float* lse, const uint8_t* spd,
+                                          const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                          void* context, size_t context_bytes, void* stream);
+gt_status gt_biased_attn_bwd_step(const void* q, const void* k, const void* v, const void* dout, const float* bias,
+                                  const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                  int32_t q_begin, int32_t q_end,
+                                  int32_t kv_begin0, int32_t kv_end0, int32_t kv_begin1, int32_t kv_end1,
+                                  float* dq_acc, float* dk_acc, float* dv_acc, double* dbias_acc,
+                                  void* context, size_t context_bytes, void* stream);
+gt_status gt_biased_attn_bwd_step_finish(const float* dq_acc, const float* dk_acc, const float* dv_acc,
+                                         const double* dbias_acc,
+                                         const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                         void* dq, void* dk, void* dv, float* dbias, void* stream);
+
+/* ---------------------------------------------------------------------------------------
  * gt_biased_attn_fwd_chunked -- single-GPU analogue of graph-aware context parallelism
  * (Sec. GA-CP: ring steps over KV blocks; Eq. 2: the bias columns of each block are taken at
  * the block's global node indices; item 3: bias folded in before the softmax statistics).

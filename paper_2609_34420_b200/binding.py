@@ -27,7 +27,9 @@ EXPORTS = ("gt_status_string", "gt_check",
            "gt_biased_attn_bwd_workspace", "gt_biased_attn_bwd",
            "gt_biased_attn_fwd_chunked_workspace", "gt_biased_attn_fwd_chunked",
            "gt_biased_attn_bwd_chunked_workspace", "gt_biased_attn_bwd_chunked",
-           "gt_biased_attn_fwd_step_workspace", "gt_biased_attn_fwd_step")
+           "gt_biased_attn_fwd_step_workspace", "gt_biased_attn_fwd_step",
+           "gt_biased_attn_bwd_step_context_bytes", "gt_biased_attn_bwd_step_prepare",
+           "gt_biased_attn_bwd_step", "gt_biased_attn_bwd_step_finish")
 
 
 class GtError(RuntimeError):
@@ -86,6 +88,14 @@ def lib() -> ctypes.CDLL:
             L.gt_biased_attn_fwd_step_workspace.argtypes = [bp, i32, i32]
             L.gt_biased_attn_fwd_step.restype = ctypes.c_int
             L.gt_biased_attn_fwd_step.argtypes = [vp] * 5 + [bp, i32, i32, i32] + [i32] * 6 + [vp, vp, vp, vp, sz, vp]
+            L.gt_biased_attn_bwd_step_context_bytes.restype = sz
+            L.gt_biased_attn_bwd_step_context_bytes.argtypes = [bp, i32, i32]
+            L.gt_biased_attn_bwd_step_prepare.restype = ctypes.c_int
+            L.gt_biased_attn_bwd_step_prepare.argtypes = [vp, vp, vp, vp, bp, i32, i32, i32, vp, sz, vp]
+            L.gt_biased_attn_bwd_step.restype = ctypes.c_int
+            L.gt_biased_attn_bwd_step.argtypes = [vp] * 5 + [bp, i32, i32, i32] + [i32] * 6 + [vp, vp, vp, vp, vp, sz, vp]
+            L.gt_biased_attn_bwd_step_finish.restype = ctypes.c_int
+            L.gt_biased_attn_bwd_step_finish.argtypes = [vp, vp, vp, vp, bp, i32, i32, i32, vp, vp, vp, vp, vp]
             L.gt_biased_attn_bwd_chunked_workspace.restype = sz
             L.gt_biased_attn_bwd_chunked_workspace.argtypes = [bp, i32, i32, i32, i32]
             L.gt_biased_attn_bwd_chunked.restype = ctypes.c_int
@@ -268,3 +278,40 @@ def gt_biased_attn_fwd_step(q, k, v, spd, bias, batch: Batch, max_dist: int, q_r
                                        _ptr(workspace), workspace.numel(), _stream())
     _raise(st, "gt_biased_attn_fwd_step")
     return workspace
+
+
+def gt_biased_attn_bwd_step_context_bytes(batch: Batch, n_heads: int, head_dim: int) -> int:
+    b = batch.c_struct()
+    return int(lib().gt_biased_attn_bwd_step_context_bytes(ctypes.byref(b), n_heads, head_dim))
+
+
+def gt_biased_attn_bwd_step_prepare(out, dout, lse, spd, batch: Batch, max_dist: int,
+                                    context: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _, H, d = out.shape
+    if context is None:
+        context = _workspace(gt_biased_attn_bwd_step_context_bytes(batch, H, d), out.device)
+    b = batch.c_struct()
+    st = lib().gt_biased_attn_bwd_step_prepare(_ptr(out), _ptr(dout), _ptr(lse), _ptr(spd), ctypes.byref(b), H, d,
+                                               int(max_dist), _ptr(context), context.numel(), _stream())
+    _raise(st, "gt_biased_attn_bwd_step_prepare")
+    return context
+
+
+def gt_biased_attn_bwd_step(q, k, v, dout, bias, batch: Batch, max_dist: int, q_range, kv_range0, kv_range1,
+                            dq_acc, dk_acc, dv_acc, dbias_acc, context: torch.Tensor) -> None:
+    _, H, d = q.shape
+    b = batch.c_struct()
+    st = lib().gt_biased_attn_bwd_step(_ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(bias), ctypes.byref(b), H, d, int(max_dist),
+                                       int(q_range[0]), int(q_range[1]), int(kv_range0[0]), int(kv_range0[1]),
+                                       int(kv_range1[0]), int(kv_range1[1]),
+                                       _ptr(dq_acc), _ptr(dk_acc), _ptr(dv_acc), _ptr(dbias_acc),
+                                       _ptr(context), context.numel(), _stream())
+    _raise(st, "gt_biased_attn_bwd_step")
+
+
+def gt_biased_attn_bwd_step_finish(dq_acc, dk_acc, dv_acc, dbias_acc, batch: Batch, max_dist: int, dq, dk, dv, dbias) -> None:
+    _, H, d = dq_acc.shape
+    b = batch.c_struct()
+    st = lib().gt_biased_attn_bwd_step_finish(_ptr(dq_acc), _ptr(dk_acc), _ptr(dv_acc), _ptr(dbias_acc), ctypes.byref(b), H, d,
+                                              int(max_dist), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dbias), _stream())
+    _raise(st, "gt_biased_attn_bwd_step_finish")

@@ -878,3 +878,169 @@ extern "C" gt_status gt_biased_attn_bwd_chunked(const void* q, const void* k, co
     return gt_bwd_run(q, k, v, out, dout, lse, spd, nullptr, bias, batch, n_heads, head_dim, max_dist,
                       dq, dk, dv, dbias, n_kv_chunks, dbias_chunks, workspace, workspace_bytes, stream);
 }
+
+// ------------------------------------------------------------------------------------------
+// Backward ring step (caller-driven): prepare once per backward pass, one step call per
+// (query shard, arriving key/value block), finish once.
+// ------------------------------------------------------------------------------------------
+namespace gt {
+namespace {
+
+struct StepContext {
+    size_t ext_off, spdt_off, total;
+};
+
+StepContext step_context(const gt_batch* b, int32_t n_heads)
+{
+    StepContext c{};
+    const size_t rows = (size_t)b->n_total * n_heads;
+    c.ext_off = kHeaderBytes;
+    c.spdt_off = c.ext_off + align_up(rows * kExtCols * 2, 256);
+    c.total = c.spdt_off + align_up((size_t)b->n_total * (size_t)((b->n_total + 15) & ~15), 256);
+    return c;
+}
+
+// dq = bf16(scale dq_acc), dk = bf16(scale dk_acc), dv = bf16(dv_acc), dbias = float(dbias_acc)
+__global__ void bwd_step_finish_kernel(const float* __restrict__ dq_acc, const float* __restrict__ dk_acc,
+                                       const float* __restrict__ dv_acc, const double* __restrict__ db_acc,
+                                       __nv_bfloat16* __restrict__ dq, __nv_bfloat16* __restrict__ dk, __nv_bfloat16* __restrict__ dv,
+                                       float* __restrict__ dbias, size_t n_vec4, int32_t n_db, float scale)
+{
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < (size_t)n_db) dbias[idx] = (float)db_acc[idx];
+    if (idx >= n_vec4) return;
+    const float* src[3] = {dq_acc, dk_acc, dv_acc};
+    __nv_bfloat16* dst[3] = {dq, dk, dv};
+    const float mul[3] = {scale, scale, 1.0f};
+#pragma unroll
+    for (int t = 0; t < 3; ++t) {
+        const float4 v = ((const float4*)src[t])[idx];
+        uint2 pk;
+        pk.x = pack_bf16x2(v.x * mul[t], v.y * mul[t]);
+        pk.y = pack_bf16x2(v.z * mul[t], v.w * mul[t]);
+        ((uint2*)dst[t])[idx] = pk;
+    }
+}
+
+}  // namespace
+}  // namespace gt
+
+extern "C" size_t gt_biased_attn_bwd_step_context_bytes(const gt_batch* batch, int32_t n_heads, int32_t head_dim)
+{
+    (void)head_dim;
+    if (gt::validate_batch(batch) != GT_OK || n_heads < 1 || batch->n_graphs != 1) return 0;
+    return gt::step_context(batch, n_heads).total;
+}
+
+extern "C" gt_status gt_biased_attn_bwd_step_prepare(const void* out, const void* dout, const float* lse, const uint8_t* spd,
+                                                     const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                                     void* context, size_t context_bytes, void* stream)
+{
+    using namespace gt;
+    gt_status st = validate_attn_common(batch, n_heads, head_dim, max_dist, nullptr);
+    if (st != GT_OK) return st;
+    if (batch->n_graphs != 1) return GT_ERR_UNSUPPORTED;
+    if (!out || !dout || !lse || !spd || misaligned16(out) || misaligned16(dout) || misaligned16(spd)) return GT_ERR_INVALID_ARG;
+    const StepContext cx = step_context(batch, n_heads);
+    if (context == nullptr || context_bytes < cx.total || misaligned16(context)) return GT_ERR_WORKSPACE;
+    if (sm_count() <= 0) return GT_ERR_NO_DEVICE;
+    cudaStream_t s = (cudaStream_t)stream;
+    uint8_t* ws = (uint8_t*)context;
+    GT_CUDA_TRY(cudaMemsetAsync(ws, 0, kHeaderBytes, s));
+    const unsigned tiles = (unsigned)((batch->n_total + 127) / 128);
+    spd_transpose_clamp_kernel<<<dim3(tiles, tiles, 1), 256, 0, s>>>(spd, ws + cx.spdt_off, nullptr, nullptr, batch->n_total,
+                                                                    (uint32_t)(max_dist + 1));
+    GT_CUDA_TRY(cudaGetLastError());
+    const size_t rows = (size_t)batch->n_total * n_heads;
+    const unsigned pre_blocks = (unsigned)((rows + 255) / 256);
+    uint4* ext = (uint4*)(ws + cx.ext_off);
+    if (head_dim == 64)
+        bwd_preprocess_kernel<64><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse, ext,
+                                                             batch->n_total, n_heads, sqrtf(64.f));
+    else
+        bwd_preprocess_kernel<32><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse, ext,
+                                                             batch->n_total, n_heads, sqrtf(32.f));
+    GT_CUDA_TRY(cudaGetLastError());
+    return GT_OK;
+}
+
+extern "C" gt_status gt_biased_attn_bwd_step(const void* q, const void* k, const void* v, const void* dout, const float* bias,
+                                             const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                             int32_t q_begin, int32_t q_end,
+                                             int32_t kv_begin0, int32_t kv_end0, int32_t kv_begin1, int32_t kv_end1,
+                                             float* dq_acc, float* dk_acc, float* dv_acc, double* dbias_acc,
+                                             void* context, size_t context_bytes, void* stream)
+{
+    using namespace gt;
+    gt_status st = validate_attn_common(batch, n_heads, head_dim, max_dist, nullptr);
+    if (st != GT_OK) return st;
+    if (batch->n_graphs != 1 || n_heads > 65535) return GT_ERR_UNSUPPORTED;
+    if (!q || !k || !v || !dout || !bias || !dq_acc || !dk_acc || !dv_acc || !dbias_acc) return GT_ERR_INVALID_ARG;
+    if (misaligned16(q) || misaligned16(k) || misaligned16(v) || misaligned16(dout) || misaligned16(dq_acc) ||
+        misaligned16(dk_acc) || misaligned16(dv_acc))
+        return GT_ERR_INVALID_ARG;
+    const int32_t n = batch->n_total;
+    if (q_begin < 0 || q_end > n || q_begin >= q_end) return GT_ERR_INVALID_ARG;
+    if (kv_begin0 < 0 || kv_end0 > n || kv_begin0 > kv_end0 || kv_begin1 < 0 || kv_end1 > n || kv_begin1 > kv_end1) return GT_ERR_INVALID_ARG;
+    if (q_begin & 15) return GT_ERR_UNSUPPORTED;          // the SPD^T tile of a query tile is fetched by TMA from that column
+    const StepContext cx = step_context(batch, n_heads);
+    if (context == nullptr || context_bytes < cx.total || misaligned16(context)) return GT_ERR_WORKSPACE;
+    if (sm_count() <= 0) return GT_ERR_NO_DEVICE;
+    uint8_t* ws = (uint8_t*)context;
+    CUtensorMap tq, tk, tv, tdo, text, tspd;
+    if ((st = encode_thd_map(&tq, q, n, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&tk, k, n, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&tv, v, n, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&tdo, dout, n, n_heads, head_dim)) != GT_OK) return st;
+    if ((st = encode_thd_map(&text, ws + cx.ext_off, n, n_heads, kExtCols)) != GT_OK) return st;
+    if ((st = encode_spd_map(&tspd, ws + cx.spdt_off, n, 128)) != GT_OK) return st;
+    BwdParams p{};
+    p.spd_tma = 1;
+    p.spd_t = ws + cx.spdt_off;
+    p.bias = bias;
+    p.dq_acc = dq_acc;
+    p.db_acc = dbias_acc;
+    p.dk_acc = dk_acc;
+    p.dv_acc = dv_acc;
+    p.status = (uint32_t*)context;
+    p.n_total = n;
+    p.n_heads = n_heads;
+    p.n_buckets = max_dist + 2;
+    p.scale = 1.0f / sqrtf((float)head_dim);
+    p.c1 = kLog2e * p.scale;
+    p.q_row0 = q_begin;
+    p.q_row_end = q_end;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int32_t ranges[2][2] = {{kv_begin0, kv_end0}, {kv_begin1, kv_end1}};
+    for (int r = 0; r < 2; ++r) {
+        if (ranges[r][1] <= ranges[r][0]) continue;
+        p.kv_row0 = ranges[r][0];
+        p.kv_row_end = ranges[r][1];
+        st = head_dim == 64 ? launch_bwd<64>(tq, tk, tv, tdo, text, tspd, p, batch, s)
+                            : launch_bwd<32>(tq, tk, tv, tdo, text, tspd, p, batch, s);
+        if (st != GT_OK) return st;
+    }
+    return GT_OK;
+}
+
+extern "C" gt_status gt_biased_attn_bwd_step_finish(const float* dq_acc, const float* dk_acc, const float* dv_acc,
+                                                    const double* dbias_acc,
+                                                    const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                                    void* dq, void* dk, void* dv, float* dbias, void* stream)
+{
+    using namespace gt;
+    gt_status st = validate_attn_common(batch, n_heads, head_dim, max_dist, nullptr);
+    if (st != GT_OK) return st;
+    if (!dq_acc || !dk_acc || !dv_acc || !dbias_acc || !dq || !dk || !dv || !dbias) return GT_ERR_INVALID_ARG;
+    if (misaligned16(dq_acc) || misaligned16(dk_acc) || misaligned16(dv_acc) || misaligned16(dq) || misaligned16(dk) || misaligned16(dv))
+        return GT_ERR_INVALID_ARG;
+    if (sm_count() <= 0) return GT_ERR_NO_DEVICE;
+    const size_t n_vec4 = (size_t)batch->n_total * n_heads * head_dim / 4;
+    const int32_t n_db = n_heads * (max_dist + 2);
+    const size_t n_thr = n_vec4 > (size_t)n_db ? n_vec4 : (size_t)n_db;
+    bwd_step_finish_kernel<<<(unsigned)((n_thr + 255) / 256), 256, 0, (cudaStream_t)stream>>>(
+        dq_acc, dk_acc, dv_acc, dbias_acc, (__nv_bfloat16*)dq, (__nv_bfloat16*)dk, (__nv_bfloat16*)dv, dbias, n_vec4, n_db,
+        1.0f / sqrtf((float)head_dim));
+    GT_CUDA_TRY(cudaGetLastError());
+    return GT_OK;
+}

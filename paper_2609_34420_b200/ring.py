@@ -100,3 +100,48 @@ def device_step(binding, q, k_full, v_full, spd, bias, batch, max_dist: int, lay
                                                       o_acc, lse_acc, out, state["ws"])
 
     return step
+
+
+# bwd_step(q_range, kv_range, super_range_or_empty, k_block, v_block, dk_block, dv_block, block_owner) -> None
+BwdStepFn = Callable[[Range, Range, Range, torch.Tensor, torch.Tensor, torch.Tensor, torch.Tensor, int], None]
+
+
+def ring_backward(layout: RingLayout, k_own: torch.Tensor, v_own: torch.Tensor, step: BwdStepFn,
+                  group: Optional[dist.ProcessGroup] = None, rank: Optional[int] = None,
+                  world: Optional[int] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """One context-parallel backward on this rank; returns (dk_own, dv_own), the unscaled sums of this rank's
+    own regular key rows after they have been round the ring.
+
+    k_own, v_own: the rank's REGULAR key/value rows only ([shard_len, H, d], same shape on all ranks; the
+    super nodes' K/V are replicated and do not travel).  A block travels together with its dk / dv sums:
+    at step s the rank holds the block of rank (r - s) mod P, adds what its queries contribute, and passes
+    it on; after P hops the block is home again.  Pairs are visited exactly once:
+      * the rank's regular queries see every regular block once, and the super-node keys at step 0;
+      * the super-node QUERY rows are handled at a block's home rank (step 0) for its regular keys, and on
+        rank 0 for the super-node keys.
+    What is replicated ends up as per-rank partial sums — dq of the super rows, dk / dv of the super keys,
+    dbias — and is summed by the caller (all-reduce) after this function: the step function owns those
+    accumulators, this function only moves the blocks."""
+    if world is None:
+        world = dist.get_world_size(group) if dist.is_initialized() else 1
+    if rank is None:
+        rank = dist.get_rank(group) if dist.is_initialized() else 0
+    assert len(layout.shards) == world
+    cur = [k_own, v_own, torch.zeros_like(k_own), torch.zeros_like(v_own)]
+    bufs = [[torch.empty_like(k_own) for _ in range(4)] for _ in range(2)] if world > 1 else []
+    empty: Range = (0, 0)
+    has_super = layout.super_range[1] > layout.super_range[0]
+    for s in range(world):
+        owner = (rank - s) % world
+        step(layout.shards[rank], layout.shards[owner], layout.super_range if s == 0 else empty, *cur, owner)
+        if has_super and s == 0:
+            step(layout.super_range, layout.shards[owner], layout.super_range if rank == 0 else empty, *cur, owner)
+        if world > 1:                           # the sums always move on (the last hop takes them home), K and V only while needed
+            nxt = bufs[s % 2]
+            dst, src = (rank + 1) % world, (rank - 1) % world
+            which = range(4) if s + 1 < world else range(2, 4)
+            ops = [dist.P2POp(dist.isend, cur[t], dst, group) for t in which] + [dist.P2POp(dist.irecv, nxt[t], src, group) for t in which]
+            for r in dist.batch_isend_irecv(ops):
+                r.wait()
+            cur = [nxt[t] if t in which else cur[t] for t in range(4)]
+    return cur[2], cur[3]

@@ -164,3 +164,51 @@ def test_dbias_given_the_same_bf16_output_matches_to_rounding(n, D, deg, directe
     assert rel_l2(to_f64(db), rdb) <= 1e-3
     for got, ref in ((dq, rdq), (dk, rdk), (dv, rdv)):
         assert rel_l2(to_f64(got), ref) <= GRAD_REL_L2
+
+
+# ---- caller-driven ring steps of the backward ----
+@pytest.mark.parametrize("n,n_super,ranks,d", [(1500, 60, 3, 64), (700, 0, 2, 32), (900, 37, 4, 64)])
+def test_backward_ring_steps_reproduce_the_backward_and_the_block_oracle(n, n_super, ranks, d):
+    from paper_2609_34420_b200 import binding as gt
+    w = wl.small_workload([n], 2, d, 6, seed=n + ranks, avg_degree=2.0, directed=True)
+    case = DeviceCase(w)
+    out, lse = case.forward()
+    full = case.backward(out, lse)
+    dev = case.q.device
+    n_reg = n - n_super
+    share = (n_reg // ranks + 15) // 16 * 16
+    shards = [(min(r * share, n_reg), min((r + 1) * share, n_reg)) for r in range(ranks)]
+    sup_q = (n_reg // 16 * 16, n) if n_super else (0, 0)       # query ranges start at multiples of 16 ...
+    if n_super and sup_q[0] != n_reg:                          # ... so the last shard cedes its tail rows to the super range
+        shards[-1] = (shards[-1][0], sup_q[0])
+    sup_k = (n_reg, n)
+    acc = [torch.zeros(n, 2, d, dtype=torch.float32, device=dev) for _ in range(3)]
+    db_acc = torch.zeros(2, w.max_dist + 2, dtype=torch.float64, device=dev)
+    ctx = gt.gt_biased_attn_bwd_step_prepare(out, case.dout, lse, case.spd, case.batch, w.max_dist)
+    q64, k64, v64, do64, b64 = case.host_f64()
+    spd = np.asarray(case.spd_host).reshape(n, -1)
+    ro, rl = oattn.forward_single(q64, k64, v64, spd, b64)
+    o_dq = np.zeros((n, 2, d)); o_dk = np.zeros((n, 2, d)); o_dv = np.zeros((n, 2, d)); o_db = np.zeros((2, w.max_dist + 2))
+    q_ranges = shards + ([sup_q] if n_super else [])
+    key_of = lambda a, b: np.arange(a, b)
+    for qi, (qa, qb) in enumerate(q_ranges):
+        for step in range(ranks):
+            # key blocks are the plain split of the regular rows (the query shards above may differ in the last rows)
+            kreg = (min(((qi + step) % ranks) * share, n_reg), min((((qi + step) % ranks) + 1) * share, n_reg))
+            sup = sup_k if (step == 0 and n_super) else (0, 0)
+            gt.gt_biased_attn_bwd_step(case.q, case.k, case.v, case.dout, case.bias, case.batch, w.max_dist,
+                                       (qa, qb), kreg, sup, acc[0], acc[1], acc[2], db_acc, ctx)
+            rows = np.arange(qa, qb)
+            keys = np.concatenate([key_of(*kreg), key_of(*sup)])
+            pq, pk, pv, pb = oattn.backward_block(q64, k64, v64, do64, ro, rl, spd, b64, rows, keys)
+            o_dq[rows] += pq; o_dk[keys] += pk; o_dv[keys] += pv; o_db += pb
+    gt.gt_check(ctx)
+    dq, dk, dv = (torch.full_like(case.q, float("nan")) for _ in range(3))
+    dbias = torch.full_like(case.bias, float("nan"))
+    gt.gt_biased_attn_bwd_step_finish(acc[0], acc[1], acc[2], db_acc, case.batch, w.max_dist, dq, dk, dv, dbias)
+    torch.cuda.synchronize()
+    for name, got, ref in zip(("dq", "dk", "dv", "dbias"), (dq, dk, dv, dbias), full):
+        assert rel_l2(to_f64(got), to_f64(ref)) <= CHUNK_REL_L2, name
+    s_ = 1.0 / np.sqrt(float(d))
+    for name, got, ref in (("dq", acc[0], o_dq), ("dk", acc[1], o_dk), ("dv", acc[2], o_dv), ("db", db_acc, o_db)):
+        assert rel_l2(got.cpu().numpy().astype(np.float64), ref) <= GRAD_REL_L2, name

@@ -96,3 +96,80 @@ def test_three_rank_ring_reproduces_the_forward():
         np.testing.assert_allclose(l_sup, rl[:, sa:sb], rtol=1e-12)
         owners = [own for (qr, own) in seen if qr == layout.shards[rank]]
         assert owners == [(rank - s) % world for s in range(world)]               # blocks arrive round the ring
+
+
+def _bwd_worker(rank, world, port, out_q):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    import torch.distributed as dist
+    from oracle import attention as oattn
+    from paper_2609_34420_b200 import ring, workloads as wl
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    q, k, v, spd, bias = _case()
+    w = wl.small_workload([N], H, D_HEAD, MAX_DIST, seed=5, avg_degree=2.0, directed=True)
+    do = wl.bf16_bits_to_f64(w.tensors().dout)
+    out, lse = oattn.forward_single(q, k, v, spd, bias)
+    layout = ring.RingLayout.even(N, N_SUPER, world)
+    a, b = layout.shards[rank]
+    share = max(e - s for s, e in layout.shards)
+    sa, sb = layout.super_range
+
+    def block(x):
+        blk = np.zeros((share,) + x.shape[1:]); blk[: b - a] = x[a:b]
+        return torch.from_numpy(blk)
+
+    # accumulators this rank owns: dq of its rows (and its share for the super rows), super-key dk / dv, dbias
+    dq = np.zeros_like(q); dk_sup = np.zeros((N_SUPER, H, D_HEAD)); dv_sup = np.zeros((N_SUPER, H, D_HEAD)); db = np.zeros_like(bias)
+
+    def step(q_range, kv_range, sup, k_blk, v_blk, dk_blk, dv_blk, owner):
+        ka, kb = kv_range
+        kk, vv = np.zeros_like(k), np.zeros_like(v)
+        kk[ka:kb] = k_blk.numpy()[: kb - ka]; vv[ka:kb] = v_blk.numpy()[: kb - ka]       # the arrived block ...
+        kk[sa:sb] = k[sa:sb]; vv[sa:sb] = v[sa:sb]                                      # ... and the local super-node replica
+        rows = np.arange(*q_range); keys = np.concatenate([np.arange(ka, kb), np.arange(*sup)])
+        pq, pk, pv, pb = oattn.backward_block(q, kk, vv, do, out, lse, spd, bias, rows, keys)
+        dq[rows] += pq
+        dk_blk.numpy()[: kb - ka] += pk[: kb - ka]; dv_blk.numpy()[: kb - ka] += pv[: kb - ka]
+        if sup[1] > sup[0]:
+            dk_sup[:] += pk[kb - ka:]; dv_sup[:] += pv[kb - ka:]
+        db[:] += pb
+
+    dk_own, dv_own = ring.ring_backward(layout, block(k), block(v), step)
+    red = [torch.from_numpy(x) for x in (dq[sa:sb].copy(), dk_sup, dv_sup, db)]
+    for t in red:
+        dist.all_reduce(t)
+    out_q.put((rank, dq[a:b], dk_own.numpy()[: b - a], dv_own.numpy()[: b - a], [t.numpy() for t in red]))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_three_rank_backward_ring_reproduces_the_backward():
+    world = 3
+    ctx = mp.get_context("spawn")
+    out_q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_bwd_worker, args=(r, world, port, out_q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted((out_q.get(timeout=180) for _ in range(world)), key=lambda r: r[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    from oracle import attention as oattn
+    from paper_2609_34420_b200 import ring, workloads as wl
+    q, k, v, spd, bias = _case()
+    w = wl.small_workload([N], H, D_HEAD, MAX_DIST, seed=5, avg_degree=2.0, directed=True)
+    do = wl.bf16_bits_to_f64(w.tensors().dout)
+    rdq, rdk, rdv, rdb = oattn.backward_single(q, k, v, do, spd, bias)
+    layout = ring.RingLayout.even(N, N_SUPER, world)
+    sa, sb = layout.super_range
+    s_ = 1.0 / np.sqrt(float(D_HEAD))
+    for rank, dq_sh, dk_sh, dv_sh, (dq_sup, dk_sup, dv_sup, db) in res:
+        a, b = layout.shards[rank]
+        np.testing.assert_allclose(dq_sh * s_, rdq[a:b], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(dk_sh * s_, rdk[a:b], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(dv_sh, rdv[a:b], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(dq_sup * s_, rdq[sa:sb], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(dk_sup * s_, rdk[sa:sb], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(dv_sup, rdv[sa:sb], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(db, rdb, rtol=1e-9, atol=1e-12)
