@@ -247,7 +247,7 @@ struct DenseParams {
     uint8_t* nonempty[2];   // [n_max] frontier row of that buffer has a bit set
     uint8_t* row_done;      // [n_max] every valid target of the block is visited
     int32_t* item_start;    // [n_max + 1] prefix sum of chunks per vertex (of the current graph)
-    int32_t* item_vertex;   // [n_items] vertex of a work item
+    int4* item_rec;         // [n_items] {vertex, first edge, one past the last edge, chunks of the vertex} of a work item
     uint32_t* sync;         // [0] barrier counter, [1] abort, [2..5] "some frontier bit" and [8..11] work counter, by level mod 4
     int32_t n_max;
     int32_t n_groups;       // CTA groups that work on different column blocks at the same time (own state each)
@@ -283,11 +283,15 @@ __global__ void spd_dense_items_kernel(const int32_t* __restrict__ rp, int32_t n
     if (threadIdx.x == 0) item_start[n] = carry;
 }
 
-__global__ void spd_dense_item_vertex_kernel(const int32_t* __restrict__ item_start, int32_t n, int32_t* __restrict__ item_vertex)
+__global__ void spd_dense_item_rec_kernel(const int32_t* __restrict__ rp, const int32_t* __restrict__ item_start, int32_t n,
+                                          int4* __restrict__ item_rec)
 {
     const int v = blockIdx.x * blockDim.x + threadIdx.x;
     if (v >= n) return;
-    for (int32_t i = item_start[v]; i < item_start[v + 1]; ++i) item_vertex[i] = v;
+    const int32_t first = item_start[v], n_chunks = item_start[v + 1] - first;
+    const int32_t e0 = rp[v], e1 = rp[v + 1];
+    for (int32_t c = 0; c < n_chunks; ++c)
+        item_rec[first + c] = make_int4(v, e0 + c * kDenseChunk, min(e1, e0 + (c + 1) * kDenseChunk), n_chunks);
 }
 
 // Grid barrier with a bounded wait (the kernel is launched cooperatively, so all CTAs are resident).
@@ -370,7 +374,6 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
     const int n_gw = (int)((n_ctas * blockDim.x) >> 5);
     const int32_t n = p.n_total;
     const int64_t ld = (int64_t)((n + 15) & ~15);
-    const int32_t* __restrict__ rp = p.row_ptr;
     const int32_t* __restrict__ ci = p.col_idx;
     const int32_t n_items = d.item_start[n];
     const uint32_t unreach = (uint32_t)(p.max_dist + 1);
@@ -458,11 +461,12 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                 const int batch = __shfl_sync(0xffffffffu, batch_next, 0);
                 if (batch >= n_batches) break;
                 if (lane == 0) batch_next = (int)atomicAdd(counter, 1u);
+              int4 rec_next = d.item_rec[batch];
               for (int item = batch; item < n_items; item += n_batches) {
-                const int s = d.item_vertex[item];
-                const int32_t first = d.item_start[s];
-                const int32_t n_chunks = d.item_start[s + 1] - first;
-                const int32_t c = item - first;
+                const int4 rec = rec_next;                                  // one 16-byte record per item, fetched an item ahead
+                if (item + n_batches < n_items) rec_next = d.item_rec[item + n_batches];
+                const int s = rec.x;
+                const int32_t n_chunks = rec.w;
                 uint32_t acc[kDenseVecs][4];
 #pragma unroll
                 for (int q = 0; q < kDenseVecs; ++q)
@@ -489,8 +493,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                         }
                     }
                     bool covered = false;
-                    const int32_t e0 = rp[s] + c * kDenseChunk;
-                    const int32_t e1 = min(rp[s + 1], e0 + kDenseChunk);
+                    const int32_t e0 = rec.y, e1 = rec.z;
 #pragma unroll
                     for (int part = 0; part < kDenseChunk / 32 && !covered; ++part) {
                         const int32_t e = e0 + part * 32 + lane;
@@ -600,7 +603,7 @@ struct SpdPlan {
     bool smem_state;
     bool dense;                // single large graph: bit-matrix BFS (persistent cooperative kernel)
     int dense_groups;
-    size_t dense_off[11];      // vis, fr0, fr1, acc, acc_cnt, nonempty0, nonempty1, row_done, item_start, sync, item_vertex
+    size_t dense_off[11];      // vis, fr0, fr1, acc, acc_cnt, nonempty0, nonempty1, row_done, item_start, sync, item_rec
     int threads;
     int grid;
     size_t smem_bytes;
@@ -650,7 +653,7 @@ SpdPlan make_plan(const gt_batch* b, int64_t nnz)
             pl.dense_off[8] = off; off += align_up((n + 1) * sizeof(int32_t), 256);
             pl.dense_off[9] = off; off += 256 * kDenseMaxGroups;
             // work items: one per vertex plus one per further 64 out-edges
-            pl.dense_off[10] = off; off += align_up((n + (size_t)(nnz > 0 ? nnz : 0) / kDenseChunk + 1) * sizeof(int32_t), 256);
+            pl.dense_off[10] = off; off += align_up((n + (size_t)(nnz > 0 ? nnz : 0) / kDenseChunk + 1) * sizeof(int4), 256);
             pl.total_bytes = off;
         } else {
             cudaGetLastError();
@@ -715,7 +718,7 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
         d.row_done = ws + pl.dense_off[7];
         d.item_start = (int32_t*)(ws + pl.dense_off[8]);
         d.sync = (uint32_t*)(ws + pl.dense_off[9]);
-        d.item_vertex = (int32_t*)(ws + pl.dense_off[10]);
+        d.item_rec = (int4*)(ws + pl.dense_off[10]);
         d.n_max = batch->n_total;
         d.n_groups = pl.dense_groups;
         // accumulator rows, their counters and the barrier words start at zero
@@ -723,7 +726,7 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
         GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[9], 0, 256 * kDenseMaxGroups, s));
         spd_dense_items_kernel<<<1, 1024, 0, s>>>(row_ptr, batch->n_total, d.item_start);
         GT_CUDA_TRY(cudaGetLastError());
-        spd_dense_item_vertex_kernel<<<(unsigned)((batch->n_total + 255) / 256), 256, 0, s>>>(d.item_start, batch->n_total, d.item_vertex);
+        spd_dense_item_rec_kernel<<<(unsigned)((batch->n_total + 255) / 256), 256, 0, s>>>(row_ptr, d.item_start, batch->n_total, d.item_rec);
         GT_CUDA_TRY(cudaGetLastError());
         void* args[] = {(void*)&p, (void*)&d};
         GT_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)spd_dense_kernel, dim3((unsigned)pl.grid), dim3((unsigned)pl.threads), args, 0, s));
