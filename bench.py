@@ -39,6 +39,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the backward kernel, from the ncu
 # capture summarised in profiles/attn_bwd_kernel_powerlaw16k.md (16 384-node graph, scaled by N^2).
 BWD_KERNEL_DRAM_BYTES_PER_N2 = 1036.5e6 / (16384.0 ** 2)
+# the same for the forward kernel (profiles/attn_fwd_kernel_powerlaw16k.md) and for the bit-matrix SPD build
+# (profiles/spd_dense_kernel_pl24000.md: 24 000-node graph; its traffic grows with N^2 x levels, so this is an estimate)
+FWD_KERNEL_DRAM_BYTES_PER_N2 = 438.7e6 / (16384.0 ** 2)
+SPD_DENSE_DRAM_BYTES_PER_N2 = 6.26e9 / (24000.0 ** 2)
 
 
 def load_peaks():
@@ -420,11 +424,19 @@ def run_cuda(args) -> int:
         "traffic": None if BWD_KERNEL_DRAM_BYTES_PER_N2 is None else BWD_KERNEL_DRAM_BYTES_PER_N2 * sum_n2,
         "flops_per_launch": f_bwd, "ms_per_launch": bwd_ms,
     }
+    fwd_tflops_ = f_fwd / (fwd_ms * 1e-3) / 1e12
+    roofline_fwd = {
+        "kernel": "attn_fwd_kernel", "bound": "tensor", "achieved": fwd_tflops_, "peak": peak_tf, "unit": "TFLOP/s",
+        "frac": fwd_tflops_ / peak_tf, "peak_kind": f"bf16_tflops_sustained of {peak_kind} (kernel timed inside a long step)",
+        "frac_of_burst_peak": fwd_tflops_ / float(peaks["bf16_tflops"]),
+        "traffic": FWD_KERNEL_DRAM_BYTES_PER_N2 * sum_n2, "flops_per_launch": f_fwd, "ms_per_launch": fwd_ms,
+    }
     roofline_spd = {
         "kernel": "spd_dense_kernel" if dense_spd else "spd_bfs_kernel", "bound": "hbm", "achieved": spd_alg_bytes / (spd_ms * 1e-3) / 1e9,
         "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
         "frac": spd_alg_bytes / (spd_ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"]), "peak_kind": f"hbm_gbs of {peak_kind}",
-        "bytes_per_launch": spd_alg_bytes, "ms_per_launch": spd_ms, "traffic": None,
+        "bytes_per_launch": spd_alg_bytes, "ms_per_launch": spd_ms,
+        "traffic": SPD_DENSE_DRAM_BYTES_PER_N2 * sum_n2 if dense_spd else None,
     }
 
     cpu_baseline = None
@@ -450,7 +462,7 @@ def run_cuda(args) -> int:
         "spd_build_gbs": roofline_spd["achieved"],
         "pct_of_bf16_peak": {"burst": 100 * value / world / float(peaks["bf16_tflops"]),
                              "sustained": 100 * value / world / peak_tf, "nominal_2250": 100 * value / world / 2250.0},
-        "roofline": roofline, "roofline_spd": roofline_spd, "cpu_baseline": cpu_baseline,
+        "roofline": roofline, "roofline_fwd": roofline_fwd, "roofline_spd": roofline_spd, "cpu_baseline": cpu_baseline,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "ms_per_step": e2e_ms, "steps": n_e2e, "includes": "H2D of Q,K,V,dO,bias,CSR; spd_build+fwd+bwd; D2H of O,LSE,dQ,dK,dV,dBias (input copies overlap the SPD build, O/LSE copies the backward, on a second stream)"},
         "gpu_launches": kernels_per_step * args.steps, "clocks": clocks,
