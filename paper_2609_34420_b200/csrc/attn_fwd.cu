@@ -77,6 +77,10 @@ struct FwdParams {
     int32_t range_begin[2];
     int32_t range_end[2];
     int32_t q_block0;          // first 256-row query block of the launch
+    float* state_o;            // step entry point, one key range: carried state merged in the epilogue
+    float* state_lse;          //   ([T,H,D] fp32, [H,T]); rows [state_q_begin, state_q_end) only
+    int32_t state_q_begin;
+    int32_t state_q_end;
     int32_t spd_tma;           // 1: single graph, SPD tiles come by TMA; 0: cp.async loader warp
     float c1;                  // log2(e) / sqrt(d)
 };
@@ -508,6 +512,40 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const int32_t q = q0 + t * kRowsPerTile + r;
         const float inv_l = 1.0f / l;
         const float lse_nat = (m + log2f(l)) * kLn2;
+        if (kPartial && p.state_o != nullptr) {
+            // Merge into the carried state: lse' = log(e^lse0 + e^lse), o' = e^(lse0-lse') o0 + e^(lse-lse') o.
+            const bool mine = q >= p.state_q_begin && q < p.state_q_end;
+            float* lse_ptr = p.state_lse + (size_t)h * p.n_total + q;
+            const float l0 = mine ? *lse_ptr : -INFINITY;
+            named_barrier_sync(pair_bar, 64);   // both column halves have read lse0 before it is rewritten
+            const float mx = fmaxf(l0, lse_nat);
+            const float e0 = l0 == -INFINITY ? 0.f : exp2f((l0 - mx) * kLog2e);
+            const float e1 = exp2f((lse_nat - mx) * kLog2e);
+            const float inv = 1.0f / (e0 + e1);
+            const float w0 = e0 * inv, w1 = e1 * inv * inv_l;
+#pragma unroll
+            for (int c = 0; c < kOC / kOP; ++c) {
+                uint32_t o[kOP];
+                tmem_ld<kOP>(tO + c * kOP, o);
+                tmem_wait_ld();
+                if (mine) {
+                    float4* st = (float4*)(p.state_o + ((size_t)q * p.n_heads + h) * D + hf * kOC + c * kOP);
+                    uint2* ob = p.out ? (uint2*)(p.out + ((size_t)q * p.n_heads + h) * D + hf * kOC + c * kOP) : nullptr;
+#pragma unroll
+                    for (int i = 0; i < kOP / 4; ++i) {
+                        float4 a = make_float4(__uint_as_float(o[4 * i]) * w1, __uint_as_float(o[4 * i + 1]) * w1,
+                                               __uint_as_float(o[4 * i + 2]) * w1, __uint_as_float(o[4 * i + 3]) * w1);
+                        if (e0 != 0.f) {
+                            const float4 b = st[i];
+                            a.x += w0 * b.x; a.y += w0 * b.y; a.z += w0 * b.z; a.w += w0 * b.w;
+                        }
+                        st[i] = a;
+                        if (ob) ob[i] = make_uint2(pack_bf16x2(a.x, a.y), pack_bf16x2(a.z, a.w));
+                    }
+                }
+            }
+            if (mine && hf == 0) *lse_ptr = mx + log2f(e0 + e1) * kLn2;
+        } else {
 #pragma unroll
         for (int c = 0; c < kOC / kOP; ++c) {
             uint32_t o[kOP];
@@ -537,6 +575,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         if (q < n_g && hf == 0) {
             if (kPartial) p.part_lse[((size_t)chunk * p.n_heads + h) * p.n_total + q] = lse_nat;
             else p.lse[(size_t)h * p.n_total + node0 + q] = lse_nat;
+        }
         }
     }
 
@@ -819,9 +858,16 @@ extern "C" gt_status gt_biased_attn_fwd_step(const void* q, const void* k, const
     const int grid_y = (q_end - 1) / kRowsPerCta - p.q_block0 + 1;
     p.c1 = kLog2e / sqrtf((float)head_dim);
     cudaStream_t s = (cudaStream_t)stream;
+    // One non-empty key range: the kernel's epilogue merges into the carried state itself.
+    const bool fused = n_parts == 1 && kv_end0 > kv_begin0;
+    if (fused) {
+        p.state_o = o_acc; p.state_lse = lse_acc;
+        p.state_q_begin = q_begin; p.state_q_end = q_end;
+        p.out = (__nv_bfloat16*)out;
+    }
     st = head_dim == 64 ? launch_fwd<64, true>(tq, tk, tv, tspd, p, batch, n_parts, s, grid_y)
                         : launch_fwd<32, true>(tq, tk, tv, tspd, p, batch, n_parts, s, grid_y);
-    if (st != GT_OK) return st;
+    if (st != GT_OK || fused) return st;
     const size_t n_thr = (size_t)(q_end - q_begin) * n_heads * (head_dim / 4);
     const unsigned blocks = (unsigned)((n_thr + 255) / 256);
     if (head_dim == 64)
