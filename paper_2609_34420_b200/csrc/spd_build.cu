@@ -237,14 +237,16 @@ constexpr int kDenseVecs = kDenseRowWords / 128;         // 16-byte vectors per 
 constexpr int kDenseChunk = 32;                          // out-edges per work item
 constexpr int kDenseBatch = 4;                           // work items a warp takes at a time
 constexpr int kDenseMaxGroups = 4;                       // CTA groups working on different column blocks at once
+constexpr int kDenseHist = 12;                           // levels whose frontier matrices are kept for the output pass
+constexpr int kDensePlanes = kDenseHist + 1;             // frontier matrices per group (level 0 .. kDenseHist)
 constexpr uint32_t kGridWaitIterations = 1u << 24;
 
 struct DenseParams {
     uint32_t* vis;          // [n_max][kDenseRowWords]
-    uint32_t* fr[2];        // [n_max][kDenseRowWords] current / next frontier
+    uint32_t* fr;           // [kDensePlanes][n_max][kDenseRowWords] frontier of level l in plane l (later levels: planes 0 / 1 in turn)
     uint32_t* acc;          // [n_max][kDenseRowWords] accumulator rows of split vertices (all zero between uses)
     uint32_t* acc_cnt;      // [n_max] finished chunks of a split vertex
-    uint8_t* nonempty[2];   // [n_max] frontier row of that buffer has a bit set
+    uint8_t* nonempty;      // [kDensePlanes][n_max] the row of that plane is valid and has a bit set (rows without the flag are never read)
     uint8_t* row_done;      // [n_max] every valid target of the block is visited
     int32_t* item_start;    // [n_max + 1] prefix sum of chunks per vertex (of the current graph)
     int4* item_rec;         // [n_items] {vertex, first edge, one past the last edge, chunks of the vertex} of a work item
@@ -334,9 +336,9 @@ __device__ __forceinline__ uint4 dense_blend16(uint4 old, uint32_t m16, uint32_t
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
-// bytes of word `w` (32 targets from t0) of output row `row`: bits of `set` take `code`; bytes whose bit is in
-// `keep` are final already and are preserved (the row is only read when there are any)
-__device__ __forceinline__ void dense_write_word(uint8_t* row, int32_t t0, uint32_t set, uint32_t keep, uint32_t code)
+// bytes of a word (32 targets from t0) of an output row that the output pass has written: the bytes whose bit
+// is in `set` take `code`, the others stay (final already, or the provisional unreachable code, or padding)
+__device__ __forceinline__ void dense_blend_word(uint8_t* row, int32_t t0, uint32_t set, uint32_t code)
 {
     const uint32_t code4 = code * 0x01010101u;
 #pragma unroll
@@ -344,9 +346,7 @@ __device__ __forceinline__ void dense_write_word(uint8_t* row, int32_t t0, uint3
         const uint32_t m = (set >> (16 * hlf)) & 0xFFFFu;
         if (m) {
             uint4* ptr = (uint4*)(row + t0 + 16 * hlf);
-            uint4 old = make_uint4(0u, 0u, 0u, 0u);
-            if ((keep >> (16 * hlf)) & 0xFFFFu) old = __ldcg(ptr);      // written by another SM in an earlier level
-            *ptr = dense_blend16(old, m, code4);
+            *ptr = dense_blend16(__ldcg(ptr), m, code4);      // written by another SM in an earlier level
         }
     }
 }
@@ -365,8 +365,8 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
     const uint32_t n_ctas = ((uint32_t)gridDim.x - (uint32_t)grp + (uint32_t)d.n_groups - 1u) / (uint32_t)d.n_groups;
     {
         const size_t m = (size_t)grp * d.n_max;
-        d.vis += m * kDenseRowWords; d.fr[0] += m * kDenseRowWords; d.fr[1] += m * kDenseRowWords; d.acc += m * kDenseRowWords;
-        d.acc_cnt += m; d.nonempty[0] += m; d.nonempty[1] += m; d.row_done += m;
+        d.vis += m * kDenseRowWords; d.fr += m * kDensePlanes * kDenseRowWords; d.acc += m * kDenseRowWords;
+        d.acc_cnt += m; d.nonempty += m * kDensePlanes; d.row_done += m;
         d.sync += grp * 64;
     }
     const int lane = threadIdx.x & 31;
@@ -380,35 +380,39 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
     uint32_t epoch = 0;
     uint32_t step = 0;                         // levels over all column blocks: index of the rotating "any" flags
 
-    // finalise vertex s for this level: new bits, visited, next frontier row, flags, output bytes
-    auto finalise = [&](int s, const uint32_t (&acc)[kDenseVecs][4], int32_t col0, uint32_t* vis_row, uint32_t* next_row,
-                        uint8_t* next_nonempty, uint32_t code, uint32_t flag_idx) {
+    // finalise vertex s for this level: new bits (left in acc), visited, next frontier row, flags.  While the
+    // levels still have a plane each (blend == false) no output byte is written here: the output pass reads the
+    // planes once.  Later levels blend their bytes into the rows that pass has written.
+    auto finalise = [&](int s, uint32_t (&acc)[kDenseVecs][4], int32_t col0, uint32_t* vis_row, uint32_t* next_row,
+                        uint8_t* next_nonempty, uint32_t code, uint32_t flag_idx, bool blend) {
         bool any_new = false, full = true;
-        const bool rewrite = __ldcg(&next_nonempty[s]) != 0;      // the row this level overwrites has bits set
 #pragma unroll
         for (int q = 0; q < kDenseVecs; ++q) {
             const uint4 v4 = __ldcg((const uint4*)&vis_row[dense_word(lane, q, 0)]);   // written by other SMs earlier: from L2
             const uint32_t v[4] = {v4.x, v4.y, v4.z, v4.w};
-            uint32_t nw[4];
             bool vec_new = false;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int32_t t0 = col0 + dense_word(lane, q, j) * 32;
                 const int32_t nv = n - t0;
                 const uint32_t vm = nv >= 32 ? 0xffffffffu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
-                nw[j] = acc[q][j] & ~v[j] & vm;
-                if (nw[j]) {
-                    dense_write_word(p.spd + (int64_t)s * ld, t0, nw[j], v[j], code);
+                acc[q][j] &= ~v[j] & vm;
+                if (acc[q][j]) {
+                    if (blend) dense_blend_word(p.spd + (int64_t)s * ld, t0, acc[q][j], code);
                     vec_new = true;
                 }
-                full = full && (((v[j] | nw[j]) & vm) == vm);
+                full = full && (((v[j] | acc[q][j]) & vm) == vm);
             }
-            if (vec_new || rewrite) *(uint4*)&next_row[dense_word(lane, q, 0)] = make_uint4(nw[0], nw[1], nw[2], nw[3]);
-            if (vec_new) *(uint4*)&vis_row[dense_word(lane, q, 0)] = make_uint4(v[0] | nw[0], v[1] | nw[1], v[2] | nw[2], v[3] | nw[3]);
+            if (vec_new) *(uint4*)&vis_row[dense_word(lane, q, 0)] = make_uint4(v[0] | acc[q][0], v[1] | acc[q][1], v[2] | acc[q][2], v[3] | acc[q][3]);
             any_new = any_new || vec_new;
         }
         const bool row_new = __any_sync(0xffffffffu, any_new);
         const bool row_full = __all_sync(0xffffffffu, full);
+        if (row_new) {                 // the whole row, zeros included: a flagged row is read in full
+#pragma unroll
+            for (int q = 0; q < kDenseVecs; ++q)
+                *(uint4*)&next_row[dense_word(lane, q, 0)] = make_uint4(acc[q][0], acc[q][1], acc[q][2], acc[q][3]);
+        }
         if (lane == 0) {
             next_nonempty[s] = row_new ? 1 : 0;
             if (row_new) d.sync[2 + flag_idx] = 1u;
@@ -416,9 +420,71 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
         }
     };
 
+    // Output pass of a column block: every byte of the block's columns is written once, from the frontier planes
+    // of levels 1..n_levels (a pair is in at most one of them): its level, clamped; 0 on the diagonal; the
+    // unreachable code where no plane has the pair (later levels, if any, overwrite that); 255 in the padding.
+    auto emit_rows = [&](int32_t col0, int n_levels) {
+        static_assert(kDenseHist <= 15, "four bit slices hold the level codes");
+        for (int s = gw; s < n; s += n_gw) {
+            uint8_t* row = p.spd + (int64_t)s * ld;
+            const uint32_t fl = (lane >= 1 && lane <= n_levels) ? (uint32_t)__ldcg(&d.nonempty[(size_t)lane * d.n_max + s]) : 0u;
+            const uint32_t valid = __ballot_sync(0xffffffffu, fl != 0u);
+#pragma unroll
+            for (int q = 0; q < kDenseVecs; ++q) {
+                uint32_t cb[4][4], found[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { found[j] = 0u; cb[0][j] = cb[1][j] = cb[2][j] = cb[3][j] = 0u; }
+                for (uint32_t m = valid; m;) {                      // two planes in flight
+                    const int l0 = __ffs(m) - 1;
+                    m &= m - 1;
+                    int l1 = 0;
+                    if (m) { l1 = __ffs(m) - 1; m &= m - 1; }
+                    const uint4 x = __ldcg((const uint4*)&d.fr[((size_t)l0 * d.n_max + s) * kDenseRowWords + dense_word(lane, q, 0)]);
+                    uint4 y = make_uint4(0u, 0u, 0u, 0u);
+                    if (l1) y = __ldcg((const uint4*)&d.fr[((size_t)l1 * d.n_max + s) * kDenseRowWords + dense_word(lane, q, 0)]);
+                    const uint32_t c0 = (uint32_t)min(l0, p.max_dist), c1 = (uint32_t)min(l1, p.max_dist);
+                    const uint32_t xw[4] = {x.x, x.y, x.z, x.w}, yw[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) {
+                        const uint32_t m0 = 0u - ((c0 >> b) & 1u), m1 = 0u - ((c1 >> b) & 1u);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) cb[b][j] |= (xw[j] & m0) | (yw[j] & m1);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) found[j] |= xw[j] | yw[j];
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int32_t t0 = col0 + dense_word(lane, q, j) * 32;
+                    if (t0 >= (int32_t)ld) continue;
+                    const int32_t nv = n - t0, np = (int32_t)ld - t0, rel = s - t0;
+                    const uint32_t vm = nv >= 32 ? 0xffffffffu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
+                    const uint32_t pm = (np >= 32 ? 0xffffffffu : ((1u << np) - 1u)) & ~vm;       // padding columns
+                    const uint32_t self = (rel >= 0 && rel < 32) ? (1u << rel) : 0u;
+                    const uint32_t miss = ~found[j] & ~self & vm;
+#pragma unroll
+                    for (int hlf = 0; hlf < 2; ++hlf) {
+                        if (t0 + 16 * hlf >= (int32_t)ld) continue;
+                        uint32_t o[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const int sh = 16 * hlf + 4 * k;
+                            auto spread = [&](uint32_t w) { return (((w >> sh) & 0xFu) * 0x00204081u) & 0x01010101u; };   // bit i of the nibble -> byte i
+                            o[k] = spread(cb[0][j]) | (spread(cb[1][j]) << 1) | (spread(cb[2][j]) << 2) | (spread(cb[3][j]) << 3);
+                            o[k] |= spread(miss) * unreach;
+                            if (pm) o[k] |= spread(pm) * 255u;
+                        }
+                        *(uint4*)(row + t0 + 16 * hlf) = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                }
+            }
+        }
+    };
+
     for (int32_t col0 = grp * kDenseBlockBits; col0 < (int32_t)ld; col0 += d.n_groups * kDenseBlockBits) {
         // ---- level 0 of this column block: every vertex has reached itself ----
         for (int s = gw; s < n; s += n_gw) {
+            const bool mine = s >= col0 && s < col0 + kDenseBlockBits;
 #pragma unroll
             for (int q = 0; q < kDenseVecs; ++q) {
                 uint32_t bit[4];
@@ -429,26 +495,24 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                 }
                 const uint4 b4 = make_uint4(bit[0], bit[1], bit[2], bit[3]);
                 *(uint4*)&d.vis[(size_t)s * kDenseRowWords + dense_word(lane, q, 0)] = b4;
-                *(uint4*)&d.fr[0][(size_t)s * kDenseRowWords + dense_word(lane, q, 0)] = b4;
+                if (mine) *(uint4*)&d.fr[(size_t)s * kDenseRowWords + dense_word(lane, q, 0)] = b4;      // plane 0
             }
-            if (lane == 0) {
-                const bool mine = s >= col0 && s < col0 + kDenseBlockBits;
-                d.nonempty[0][s] = mine ? 1 : 0;
-                d.nonempty[1][s] = 1;                  // the other buffer holds stale bits: level 1 rewrites every row
-                d.row_done[s] = 0;
-                if (mine) p.spd[(int64_t)s * ld + s] = 0;
-            }
+            if (lane < kDensePlanes) d.nonempty[(size_t)lane * d.n_max + s] = (lane == 0 && mine) ? 1 : 0;
+            if (lane == 0) d.row_done[s] = 0;
         }
         if (!dense_grid_sync(d.sync, epoch, p.header, n_ctas)) return;
 
-        int cur = 0;
+        bool emitted = false;                  // the output pass of this column block has run
         for (int level = 1;; ++level) {
             const uint32_t code = (uint32_t)min(level, p.max_dist);
             const uint32_t flag_idx = step & 3u;
-            const uint32_t* fcur = d.fr[cur];
-            uint32_t* fnext = d.fr[cur ^ 1];
-            const uint8_t* ne_cur = d.nonempty[cur];
-            uint8_t* ne_next = d.nonempty[cur ^ 1];
+            // level l <= kDenseHist writes plane l; later levels take planes 0 and 1 in turn (free after the output pass)
+            const int pl_cur = level - 1 <= kDenseHist ? level - 1 : ((level - kDenseHist) & 1);
+            const int pl_next = level <= kDenseHist ? level : ((level - kDenseHist - 1) & 1);
+            const uint32_t* fcur = d.fr + (size_t)pl_cur * d.n_max * kDenseRowWords;
+            uint32_t* fnext = d.fr + (size_t)pl_next * d.n_max * kDenseRowWords;
+            const uint8_t* ne_cur = d.nonempty + (size_t)pl_cur * d.n_max;
+            uint8_t* ne_next = d.nonempty + (size_t)pl_next * d.n_max;
             // Items cost between one flag read and tens of KB of row reads, so warps take them in batches of four
             // from a counter (one per level, four in rotation) and ask for the next batch before working.  The
             // four items of a batch lie a quarter of the list apart: the chunks of one high-degree vertex are
@@ -533,7 +597,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                 }
                 uint32_t* next_row = fnext + (size_t)s * kDenseRowWords;
                 if (n_chunks == 1) {
-                    finalise(s, acc, col0, vis_row, next_row, ne_next, code, flag_idx);
+                    finalise(s, acc, col0, vis_row, next_row, ne_next, code, flag_idx, emitted);
                 } else {
                     uint32_t* acc_row = d.acc + (size_t)s * kDenseRowWords;
 #pragma unroll
@@ -555,7 +619,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                             if (a4.x | a4.y | a4.z | a4.w) *(uint4*)&acc_row[dense_word(lane, q, 0)] = make_uint4(0u, 0u, 0u, 0u);
                         }
                         if (lane == 0) d.acc_cnt[s] = 0u;
-                        finalise(s, acc, col0, vis_row, next_row, ne_next, code, flag_idx);
+                        finalise(s, acc, col0, vis_row, next_row, ne_next, code, flag_idx, emitted);
                     }
                 }
               }
@@ -567,29 +631,13 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                 d.sync[8 + ((step + 2u) & 3u)] = 0u;
             }
             ++step;
-            cur ^= 1;
-            if (!any) break;
-        }
-
-        // ---- unreachable pairs and row padding of this column block ----
-        for (int s = gw; s < n; s += n_gw) {
-            uint8_t* row = p.spd + (int64_t)s * ld;
-#pragma unroll
-            for (int q = 0; q < kDenseVecs; ++q) {
-                const uint4 v4 = __ldcg((const uint4*)&d.vis[(size_t)s * kDenseRowWords + dense_word(lane, q, 0)]);
-                const uint32_t v[4] = {v4.x, v4.y, v4.z, v4.w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int32_t t0 = col0 + dense_word(lane, q, j) * 32;
-                    if (t0 >= (int32_t)ld) continue;
-                    const int32_t nv = n - t0, np = (int32_t)ld - t0;
-                    const uint32_t vm = nv >= 32 ? 0xffffffffu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
-                    const uint32_t pm = (np >= 32 ? 0xffffffffu : ((1u << np) - 1u)) & ~vm;       // padding columns
-                    const uint32_t miss = ~v[j] & vm;
-                    if (miss) dense_write_word(row, t0, miss, v[j] | pm, unreach);
-                    if (pm) dense_write_word(row, t0, pm, vm, 255u);
-                }
+            if (!emitted && (!any || level == kDenseHist)) {
+                emit_rows(col0, level);
+                emitted = true;
+                // levels that follow blend into rows this pass wrote from other SMs
+                if (any && !dense_grid_sync(d.sync, epoch, p.header, n_ctas)) return;
             }
+            if (!any) break;
         }
         // the same warps own the same vertices in the next block's level 0, and nothing else touches the
         // bit matrices until the barrier behind it
@@ -603,7 +651,7 @@ struct SpdPlan {
     bool smem_state;
     bool dense;                // single large graph: bit-matrix BFS (persistent cooperative kernel)
     int dense_groups;
-    size_t dense_off[11];      // vis, fr0, fr1, acc, acc_cnt, nonempty0, nonempty1, row_done, item_start, sync, item_rec
+    size_t dense_off[9];       // vis, frontier planes, acc, acc_cnt, nonempty flags, row_done, item_start, sync, item_rec
     int threads;
     int grid;
     size_t smem_bytes;
@@ -647,13 +695,16 @@ SpdPlan make_plan(const gt_batch* b, int64_t nnz)
             const size_t G = (size_t)pl.dense_groups;
             const size_t mat = align_up(G * n * kDenseRowWords * sizeof(uint32_t), 256);
             size_t off = pl.scratch_off;
-            for (int i = 0; i < 4; ++i) { pl.dense_off[i] = off; off += mat; }
-            pl.dense_off[4] = off; off += align_up(G * n * sizeof(uint32_t), 256);
-            for (int i = 5; i < 8; ++i) { pl.dense_off[i] = off; off += align_up(G * n, 256); }
-            pl.dense_off[8] = off; off += align_up((n + 1) * sizeof(int32_t), 256);
-            pl.dense_off[9] = off; off += 256 * kDenseMaxGroups;
-            // work items: one per vertex plus one per further 64 out-edges
-            pl.dense_off[10] = off; off += align_up((n + (size_t)(nnz > 0 ? nnz : 0) / kDenseChunk + 1) * sizeof(int4), 256);
+            pl.dense_off[0] = off; off += mat;
+            pl.dense_off[1] = off; off += mat * kDensePlanes;
+            pl.dense_off[2] = off; off += mat;
+            pl.dense_off[3] = off; off += align_up(G * n * sizeof(uint32_t), 256);
+            pl.dense_off[4] = off; off += align_up(G * n * kDensePlanes, 256);
+            pl.dense_off[5] = off; off += align_up(G * n, 256);
+            pl.dense_off[6] = off; off += align_up((n + 1) * sizeof(int32_t), 256);
+            pl.dense_off[7] = off; off += 256 * kDenseMaxGroups;
+            // work items: one per vertex plus one per further chunk of out-edges
+            pl.dense_off[8] = off; off += align_up((n + (size_t)(nnz > 0 ? nnz : 0) / kDenseChunk + 1) * sizeof(int4), 256);
             pl.total_bytes = off;
         } else {
             cudaGetLastError();
@@ -709,21 +760,19 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
     if (pl.dense) {
         DenseParams d{};
         d.vis = (uint32_t*)(ws + pl.dense_off[0]);
-        d.fr[0] = (uint32_t*)(ws + pl.dense_off[1]);
-        d.fr[1] = (uint32_t*)(ws + pl.dense_off[2]);
-        d.acc = (uint32_t*)(ws + pl.dense_off[3]);
-        d.acc_cnt = (uint32_t*)(ws + pl.dense_off[4]);
-        d.nonempty[0] = ws + pl.dense_off[5];
-        d.nonempty[1] = ws + pl.dense_off[6];
-        d.row_done = ws + pl.dense_off[7];
-        d.item_start = (int32_t*)(ws + pl.dense_off[8]);
-        d.sync = (uint32_t*)(ws + pl.dense_off[9]);
-        d.item_rec = (int4*)(ws + pl.dense_off[10]);
+        d.fr = (uint32_t*)(ws + pl.dense_off[1]);
+        d.acc = (uint32_t*)(ws + pl.dense_off[2]);
+        d.acc_cnt = (uint32_t*)(ws + pl.dense_off[3]);
+        d.nonempty = ws + pl.dense_off[4];
+        d.row_done = ws + pl.dense_off[5];
+        d.item_start = (int32_t*)(ws + pl.dense_off[6]);
+        d.sync = (uint32_t*)(ws + pl.dense_off[7]);
+        d.item_rec = (int4*)(ws + pl.dense_off[8]);
         d.n_max = batch->n_total;
         d.n_groups = pl.dense_groups;
         // accumulator rows, their counters and the barrier words start at zero
-        GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[3], 0, pl.dense_off[5] - pl.dense_off[3], s));
-        GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[9], 0, 256 * kDenseMaxGroups, s));
+        GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[2], 0, pl.dense_off[4] - pl.dense_off[2], s));
+        GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[7], 0, 256 * kDenseMaxGroups, s));
         spd_dense_items_kernel<<<1, 1024, 0, s>>>(row_ptr, batch->n_total, d.item_start);
         GT_CUDA_TRY(cudaGetLastError());
         spd_dense_item_rec_kernel<<<(unsigned)((batch->n_total + 255) / 256), 256, 0, s>>>(row_ptr, d.item_start, batch->n_total, d.item_rec);
