@@ -86,8 +86,8 @@ gt_status gt_check(void* workspace, void* stream);
  * distinct from unreachable pairs (bucket max_dist+1).  Bit-exact and deterministic.
  * Out-of-range col_idx entries are undefined behaviour.
  * Workspace: 256 bytes + 4(G+1) when every graph has at most 17 066 nodes; a single larger graph
- * needs about 4.1 KB per node for each of min(4, ceil(n/8192)) groups of thread blocks (four bit
- * matrices of 1 KB rows per group; 1.07 GB at 65 536 nodes) plus 4 bytes per 32 edges, and a
+ * needs about 15 KB per node for each of min(4, ceil(n/8192)) groups of thread blocks (fifteen bit
+ * matrices of 1 KB rows per group; 3.9 GB at 65 536 nodes) plus 16 bytes per 32 edges, and a
  * device that supports cooperative launches; a batch that contains a larger graph needs 12 bytes
  * per node of the largest graph for each of up to 2 x (number of SMs) thread blocks.
  * ------------------------------------------------------------------------------------- */
