@@ -542,28 +542,32 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                 // (every chunk of a split vertex sees the same two flags, so they all skip together)
                 if (done && !__ldcg(&ne_next[s])) continue;
                 if (!done) {
-                    // bits this vertex still misses: once the neighbours read so far cover them all, the rest
-                    // of the edge list cannot add anything (at the dense levels a few rows are enough)
-                    uint32_t need[kDenseVecs][4];
-#pragma unroll
-                    for (int q = 0; q < kDenseVecs; ++q) {
-                        const uint4 v4 = __ldcg((const uint4*)&vis_row[dense_word(lane, q, 0)]);
-                        const uint32_t v[4] = {v4.x, v4.y, v4.z, v4.w};
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const int32_t nv = n - (col0 + dense_word(lane, q, j) * 32);
-                            const uint32_t vm = nv >= 32 ? 0xffffffffu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
-                            need[q][j] = ~v[j] & vm;
-                        }
+                    static_assert(kDenseChunk == 32, "one edge per lane");
+                    // the neighbours whose frontier row has a bit set; with none of them nothing can be new
+                    // here, and the visited row need not even be read (most items at the first and last levels)
+                    const int32_t e = rec.y + lane;
+                    int32_t u = e < rec.z ? ci[e] : -1;
+                    if (u >= 0 && !__ldcg(&ne_cur[u])) u = -1;
+                    uint32_t m = __ballot_sync(0xffffffffu, u >= 0);
+                    if (m == 0u && n_chunks == 1) {
+                        if (emitted && lane == 0) ne_next[s] = 0;      // planes in turn: the flag may be stale
+                        continue;
                     }
-                    bool covered = false;
-                    const int32_t e0 = rec.y, e1 = rec.z;
+                    if (m) {
+                        // bits this vertex still misses: once the neighbours read so far cover them all, the rest
+                        // of the edge list cannot add anything (at the dense levels a few rows are enough)
+                        uint32_t need[kDenseVecs][4];
 #pragma unroll
-                    for (int part = 0; part < kDenseChunk / 32 && !covered; ++part) {
-                        const int32_t e = e0 + part * 32 + lane;
-                        int32_t u = e < e1 ? ci[e] : -1;
-                        if (u >= 0 && !__ldcg(&ne_cur[u])) u = -1;     // empty frontier row: nothing to OR
-                        uint32_t m = __ballot_sync(0xffffffffu, u >= 0);
+                        for (int q = 0; q < kDenseVecs; ++q) {
+                            const uint4 v4 = __ldcg((const uint4*)&vis_row[dense_word(lane, q, 0)]);
+                            const uint32_t v[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const int32_t nv = n - (col0 + dense_word(lane, q, j) * 32);
+                                const uint32_t vm = nv >= 32 ? 0xffffffffu : (nv <= 0 ? 0u : ((1u << nv) - 1u));
+                                need[q][j] = ~v[j] & vm;
+                            }
+                        }
                         while (m) {                                   // two frontier rows (2 x 1 KB) in flight
                             const int b0 = __ffs(m) - 1;
                             m &= m - 1;
@@ -591,7 +595,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                             for (int q = 0; q < kDenseVecs; ++q)
 #pragma unroll
                                 for (int j = 0; j < 4; ++j) left |= need[q][j] & ~acc[q][j];
-                            if (__all_sync(0xffffffffu, left == 0u)) { covered = true; break; }
+                            if (__all_sync(0xffffffffu, left == 0u)) break;
                         }
                     }
                 }
