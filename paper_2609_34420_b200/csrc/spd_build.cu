@@ -239,6 +239,7 @@ constexpr int kDenseBatch = 4;                           // work items a warp ta
 constexpr int kDenseMaxGroups = 4;                       // CTA groups working on different column blocks at once
 constexpr int kDenseHist = 12;                           // levels whose frontier matrices are kept for the output pass
 constexpr int kDensePlanes = kDenseHist + 1;             // frontier matrices per group (level 0 .. kDenseHist)
+constexpr int kDenseFlagWords = 8192;                    // row flags of a level kept as a bitmap in shared memory (graphs up to 262 144 vertices)
 constexpr uint32_t kGridWaitIterations = 1u << 24;
 
 struct DenseParams {
@@ -246,12 +247,13 @@ struct DenseParams {
     uint32_t* fr;           // [kDensePlanes][n_max][kDenseRowWords] frontier of level l in plane l (later levels: planes 0 / 1 in turn)
     uint32_t* acc;          // [n_max][kDenseRowWords] accumulator rows of split vertices (all zero between uses)
     uint32_t* acc_cnt;      // [n_max] finished chunks of a split vertex
-    uint8_t* nonempty;      // [kDensePlanes][n_max] the row of that plane is valid and has a bit set (rows without the flag are never read)
+    uint8_t* nonempty;      // [kDensePlanes][n_pad] the row of that plane is valid and has a bit set (rows without the flag are never read)
     uint8_t* row_done;      // [n_max] every valid target of the block is visited
     int32_t* item_start;    // [n_max + 1] prefix sum of chunks per vertex (of the current graph)
     int4* item_rec;         // [n_items] {vertex, first edge, one past the last edge, chunks of the vertex} of a work item
     uint32_t* sync;         // [0] barrier counter, [1] abort, [2..5] "some frontier bit" and [8..11] work counter, by level mod 4
     int32_t n_max;
+    int32_t n_pad;          // n_max rounded up to 32: pitch of the flag arrays
     int32_t n_groups;       // CTA groups that work on different column blocks at the same time (own state each)
 };
 
@@ -366,7 +368,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
     {
         const size_t m = (size_t)grp * d.n_max;
         d.vis += m * kDenseRowWords; d.fr += m * kDensePlanes * kDenseRowWords; d.acc += m * kDenseRowWords;
-        d.acc_cnt += m; d.nonempty += m * kDensePlanes; d.row_done += m;
+        d.acc_cnt += m; d.nonempty += (size_t)grp * d.n_pad * kDensePlanes; d.row_done += m;
         d.sync += grp * 64;
     }
     const int lane = threadIdx.x & 31;
@@ -377,6 +379,8 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
     const int32_t* __restrict__ ci = p.col_idx;
     const int32_t n_items = d.item_start[n];
     const uint32_t unreach = (uint32_t)(p.max_dist + 1);
+    __shared__ uint32_t s_flags[kDenseFlagWords];
+    const bool flags_in_smem = n <= kDenseFlagWords * 32;
     uint32_t epoch = 0;
     uint32_t step = 0;                         // levels over all column blocks: index of the rotating "any" flags
 
@@ -427,7 +431,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
         static_assert(kDenseHist <= 15, "four bit slices hold the level codes");
         for (int s = gw; s < n; s += n_gw) {
             uint8_t* row = p.spd + (int64_t)s * ld;
-            const uint32_t fl = (lane >= 1 && lane <= n_levels) ? (uint32_t)__ldcg(&d.nonempty[(size_t)lane * d.n_max + s]) : 0u;
+            const uint32_t fl = (lane >= 1 && lane <= n_levels) ? (uint32_t)__ldcg(&d.nonempty[(size_t)lane * d.n_pad + s]) : 0u;
             const uint32_t valid = __ballot_sync(0xffffffffu, fl != 0u);
 #pragma unroll
             for (int q = 0; q < kDenseVecs; ++q) {
@@ -497,7 +501,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                 *(uint4*)&d.vis[(size_t)s * kDenseRowWords + dense_word(lane, q, 0)] = b4;
                 if (mine) *(uint4*)&d.fr[(size_t)s * kDenseRowWords + dense_word(lane, q, 0)] = b4;      // plane 0
             }
-            if (lane < kDensePlanes) d.nonempty[(size_t)lane * d.n_max + s] = (lane == 0 && mine) ? 1 : 0;
+            if (lane < kDensePlanes) d.nonempty[(size_t)lane * d.n_pad + s] = (lane == 0 && mine) ? 1 : 0;
             if (lane == 0) d.row_done[s] = 0;
         }
         if (!dense_grid_sync(d.sync, epoch, p.header, n_ctas)) return;
@@ -511,8 +515,22 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
             const int pl_next = level <= kDenseHist ? level : ((level - kDenseHist - 1) & 1);
             const uint32_t* fcur = d.fr + (size_t)pl_cur * d.n_max * kDenseRowWords;
             uint32_t* fnext = d.fr + (size_t)pl_next * d.n_max * kDenseRowWords;
-            const uint8_t* ne_cur = d.nonempty + (size_t)pl_cur * d.n_max;
-            uint8_t* ne_next = d.nonempty + (size_t)pl_next * d.n_max;
+            const uint8_t* ne_cur = d.nonempty + (size_t)pl_cur * d.n_pad;
+            uint8_t* ne_next = d.nonempty + (size_t)pl_next * d.n_pad;
+            // The flags of the current frontier as a bitmap in shared memory: an item looks up one per out-edge, and
+            // at the first and last levels that look-up is all an item does.
+            if (flags_in_smem) {
+                for (int w = (int)threadIdx.x; w < (n + 31) / 32; w += (int)blockDim.x) {
+                    const uint4 a = __ldcg((const uint4*)(ne_cur + 32 * (size_t)w)), b = __ldcg((const uint4*)(ne_cur + 32 * (size_t)w + 16));
+                    const uint32_t x[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+                    uint32_t bits = 0u;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)          // four flag bytes (0 / 1) -> four bits
+                        bits |= ((x[k] & 1u) | ((x[k] >> 7) & 2u) | ((x[k] >> 14) & 4u) | ((x[k] >> 21) & 8u)) << (4 * k);
+                    s_flags[w] = bits;
+                }
+                __syncthreads();
+            }
             // Items cost between one flag read and tens of KB of row reads, so warps take them in batches of four
             // from a counter (one per level, four in rotation) and ask for the next batch before working.  The
             // four items of a batch lie a quarter of the list apart: the chunks of one high-degree vertex are
@@ -547,7 +565,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                     // here, and the visited row need not even be read (most items at the first and last levels)
                     const int32_t e = rec.y + lane;
                     int32_t u = e < rec.z ? ci[e] : -1;
-                    if (u >= 0 && !__ldcg(&ne_cur[u])) u = -1;
+                    if (u >= 0 && !(flags_in_smem ? ((s_flags[u >> 5] >> (u & 31)) & 1u) : (uint32_t)__ldcg(&ne_cur[u]))) u = -1;
                     uint32_t m = __ballot_sync(0xffffffffu, u >= 0);
                     if (m == 0u && n_chunks == 1) {
                         if (emitted && lane == 0) ne_next[s] = 0;      // planes in turn: the flag may be stale
@@ -703,7 +721,7 @@ SpdPlan make_plan(const gt_batch* b, int64_t nnz)
             pl.dense_off[1] = off; off += mat * kDensePlanes;
             pl.dense_off[2] = off; off += mat;
             pl.dense_off[3] = off; off += align_up(G * n * sizeof(uint32_t), 256);
-            pl.dense_off[4] = off; off += align_up(G * n * kDensePlanes, 256);
+            pl.dense_off[4] = off; off += align_up(G * align_up(n, 32) * kDensePlanes, 256);
             pl.dense_off[5] = off; off += align_up(G * n, 256);
             pl.dense_off[6] = off; off += align_up((n + 1) * sizeof(int32_t), 256);
             pl.dense_off[7] = off; off += 256 * kDenseMaxGroups;
@@ -773,6 +791,7 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
         d.sync = (uint32_t*)(ws + pl.dense_off[7]);
         d.item_rec = (int4*)(ws + pl.dense_off[8]);
         d.n_max = batch->n_total;
+        d.n_pad = (int32_t)align_up((size_t)batch->n_total, 32);
         d.n_groups = pl.dense_groups;
         // accumulator rows, their counters and the barrier words start at zero
         GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[2], 0, pl.dense_off[4] - pl.dense_off[2], s));
