@@ -42,7 +42,7 @@ BWD_KERNEL_DRAM_BYTES_PER_N2 = 1036.5e6 / (16384.0 ** 2)
 # the same for the forward kernel (profiles/attn_fwd_kernel_powerlaw16k.md) and for the bit-matrix SPD build
 # (profiles/spd_dense_kernel_pl24000.md: 24 000-node graph; its traffic grows with N^2 x levels, so this is an estimate)
 FWD_KERNEL_DRAM_BYTES_PER_N2 = 438.7e6 / (16384.0 ** 2)
-SPD_DENSE_DRAM_BYTES_PER_N2 = 2.84e9 / (24000.0 ** 2)
+SPD_DENSE_DRAM_BYTES_PER_N2 = 2.71e9 / (24000.0 ** 2)
 
 
 def load_peaks():
