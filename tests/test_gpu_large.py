@@ -123,6 +123,32 @@ def test_bit_matrix_build_directed_ragged_with_hub_and_isolated_vertices():
     np.testing.assert_array_equal(got, exp)
 
 
+@pytest.mark.parametrize("chain", [6, 7])
+def test_bit_matrix_build_depth_around_the_kept_levels(chain):
+    """Chains of `chain` vertices hanging off one centre: the longest path has 2 * chain hops.  With 12
+    levels kept for the output pass, chain = 6 ends exactly there (the pass runs while the last level still
+    found pairs, the level after finds none) and chain = 7 adds two levels that blend into written rows.
+    Directed extras make the matrix asymmetric; a few vertices stay isolated."""
+    n_chains = 17200 // chain
+    n = 1 + n_chains * chain + 37               # 37 isolated vertices at the end
+    src, dst = [], []
+    for c in range(n_chains):
+        first = 1 + c * chain
+        src.append(0); dst.append(first)
+        for t in range(chain - 1):
+            src.append(first + t); dst.append(first + t + 1)
+    src, dst = np.array(src), np.array(dst)
+    both_src, both_dst = np.concatenate([src, dst]), np.concatenate([dst, src])
+    # one-way shortcuts from chain ends back to the centre's first neighbour of the next chain
+    ends = 1 + np.arange(0, n_chains - 1, 97) * chain + (chain - 1)
+    both_src = np.concatenate([both_src, ends]); both_dst = np.concatenate([both_dst, ends + 1])
+    csr = wl.csr_from_edges(n, both_src, both_dst, symmetric=False)
+    w, got = _spd_of(csr, 24)
+    exp = ospd.spd_matrix(w.batch.row_ptr, w.batch.col_idx, 24)
+    assert int(exp[exp <= 24].max()) == 2 * chain
+    np.testing.assert_array_equal(got, exp)
+
+
 def test_bit_matrix_build_ring_runs_thousands_of_levels_and_clips():
     n = 17500
     i = np.arange(n)
