@@ -23,7 +23,12 @@
  *    enqueue work and return; they never synchronise.  Errors detected on the host are
  *    returned immediately.  Errors detected on the device (a bounded wait that ran out)
  *    are recorded in a status word at the start of the workspace and are reported by
- *    gt_check(), which synchronises the stream.
+ *    gt_check(), which synchronises the stream.  The first 256 bytes of a workspace (or step
+ *    context) hold that status word and a few counters: they must be ZERO when the buffer is
+ *    first handed to the library (one cudaMemset after allocation); the calls do not clear the
+ *    status themselves, so that one gt_check() after a sequence of calls on the same workspace
+ *    reports a failure of any of them, and gt_check() clears it after reporting.  A workspace
+ *    with a dirty header makes gt_check() report an error that no kernel raised.
  *  - Node features are packed: a batch of G graphs with n_g nodes each is stored as
  *    T = sum n_g consecutive rows; Q, K, V, O and their gradients are bf16 [T, H, d]
  *    (row-major, d contiguous); graph g owns rows cu_seqlens[g] .. cu_seqlens[g+1]-1 and
@@ -32,8 +37,11 @@
  *  - SPD layout: graph g's block starts at byte spd_offsets[g] (int64, device) and holds
  *    n_g rows of pitch ld_g = round_up(n_g, 16) bytes; spd[i*ld_g + j] is the bucket of the
  *    ordered pair (i -> j): min(hops, max_dist), or max_dist+1 if j is unreachable from i.
- *    There are n_buckets = max_dist + 2 buckets.  Values >= n_buckets found in the matrix
- *    are clamped to n_buckets-1 on the device.  Padding bytes (j >= n_g) are ignored.
+ *    There are n_buckets = max_dist + 2 buckets.  A value >= n_buckets is invalid input: no kernel
+ *    reads out of bounds on it, but WHICH valid bucket it is taken for is unspecified and differs
+ *    between kernels (the forward may use the value modulo 32, the backward the last bucket), so
+ *    forward and backward need not agree on such a matrix.  gt_spd_build never writes one;
+ *    gt_spd_validate checks a matrix that came from elsewhere.  Padding bytes (j >= n_g) are ignored.
  *  - Supported shapes: head_dim in {32, 64}; 1 <= max_dist <= 254; n_heads >= 1;
  *    anything else returns GT_ERR_UNSUPPORTED / GT_ERR_INVALID_ARG without launching.
  */
@@ -54,7 +62,8 @@ typedef enum gt_status {
     GT_ERR_WORKSPACE = 3,      /* workspace NULL or smaller than the *_workspace() query       */
     GT_ERR_CUDA = 4,           /* a CUDA runtime/driver call failed (launch, descriptor)       */
     GT_ERR_DEVICE_TIMEOUT = 5, /* a bounded device-side wait expired (reported by gt_check)    */
-    GT_ERR_NO_DEVICE = 6       /* no sm_100 device is current                                  */
+    GT_ERR_NO_DEVICE = 6,      /* no sm_100 device is current                                  */
+    GT_ERR_BAD_SPD = 7         /* gt_spd_validate found entries >= max_dist+2 (reported by gt_check) */
 } gt_status;
 
 /* Packed batch description (host struct; cu_seqlens is a device pointer). */
@@ -120,11 +129,39 @@ gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx, int64_t n
  *    call clears the words that must start at zero), and two calls whose GPU work overlaps --
  *    different streams, or different host threads -- race on it.  Serialise them, or give the
  *    concurrent ones their own workspace through gt_spd_build.
+ *  - No device status: the caller has no workspace pointer to hand to gt_check().  Nothing is lost by
+ *    that: the builds that fit the built-in array contain no bounded device-side wait, so the only
+ *    errors this call can have are the ones it returns.
  * ------------------------------------------------------------------------------------- */
 size_t gt_spd_build_static_limit(void);
 gt_status gt_spd_build_static(const int32_t* row_ptr, const int32_t* col_idx, int64_t nnz,
                               const gt_batch* batch, int32_t max_dist,
                               const int64_t* spd_offsets, uint8_t* spd_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------
+ * gt_spd_validate -- checks an SPD index matrix that gt_spd_build did not write (the paper's bias
+ * matrix is built by the data loader, Sec. "Preliminaries"; a caller may bring its own): counts the
+ * entries of the valid n_g x n_g regions that are >= max_dist + 2.  If there are any, the status
+ * word of `workspace` (gt_spd_validate_workspace() bytes, header zeroed as for every workspace) is
+ * set to GT_ERR_BAD_SPD, which gt_check(workspace, stream) then returns; gt_spd_validate_count
+ * synchronises the stream and copies the number of such entries to *count_host (host pointer).
+ * ------------------------------------------------------------------------------------- */
+size_t gt_spd_validate_workspace(void);
+gt_status gt_spd_validate(const uint8_t* spd, const int64_t* spd_offsets, const gt_batch* batch, int32_t max_dist,
+                          void* workspace, size_t workspace_bytes, void* stream);
+gt_status gt_spd_validate_count(void* workspace, void* stream, int64_t* count_host);
+
+/* ---------------------------------------------------------------------------------------
+ * gt_test_hook_barrier_overcount -- test hook of the device-timeout path (no counterpart in the
+ * paper).  Every device-side wait of this library is bounded; one that runs out makes its kernel
+ * return and gt_check() report GT_ERR_DEVICE_TIMEOUT.  After gt_test_hook_barrier_overcount(k), k > 0,
+ * the NEXT bit-matrix build of this process (gt_spd_build on a single graph beyond 17 066 nodes) waits
+ * at its grid barriers for k arrivals more than there are thread blocks, with a shortened limit, so the
+ * wait runs out within a second; the kernel issues no asynchronous copies, so nothing is in flight when
+ * it returns, the context stays usable and the next build is normal.  The output of the hooked build
+ * is undefined.  Not thread-safe; meant for tests only.
+ * ------------------------------------------------------------------------------------- */
+void gt_test_hook_barrier_overcount(int32_t extra);
 
 /* ---------------------------------------------------------------------------------------
  * gt_biased_attn_fwd -- Eq. 1, forward.  For every graph, head h and query row i:
@@ -141,6 +178,19 @@ gt_status gt_biased_attn_fwd(const void* q, const void* k, const void* v,
                              const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
                              void* out, float* lse,
                              void* workspace, size_t workspace_bytes, void* stream);
+
+/* gt_biased_attn_fwd_ex -- gt_biased_attn_fwd that can also return the output BEFORE its rounding to
+ * bf16: out_f32, fp32 [T,H,d], or NULL (then the call is gt_biased_attn_fwd).  It exists for the
+ * backward: Delta_i = dout_i . out_i of Eq. 1's gradient is formed from the stored output, and where a
+ * few distance buckets hold nearly all pairs (max_dist 1-3, a hub or global node joined to every node,
+ * mostly unreachable pairs) dbias is a small residue of large cancelling sums, so the 2^-9 relative
+ * rounding of a bf16 `out` alone moves it by several per cent.  Pass the same out_f32 to
+ * gt_biased_attn_bwd_ex and dbias keeps the accuracy of the other gradients. */
+gt_status gt_biased_attn_fwd_ex(const void* q, const void* k, const void* v,
+                                const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
+                                const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                void* out, float* lse, float* out_f32,
+                                void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------
  * gt_biased_attn_bwd -- gradient of Eq. 1 for upstream gradient `dout` (bf16 [T,H,d]).
@@ -160,6 +210,16 @@ gt_status gt_biased_attn_bwd(const void* q, const void* k, const void* v, const 
                              const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
                              void* dq, void* dk, void* dv, float* dbias,
                              void* workspace, size_t workspace_bytes, void* stream);
+/* gt_biased_attn_bwd_ex -- gt_biased_attn_bwd with Delta_i = dout_i . out_f32_i taken from the fp32
+ * forward output of gt_biased_attn_fwd_ex (out_f32 fp32 [T,H,d]; NULL: Delta from the bf16 `out`, i.e.
+ * gt_biased_attn_bwd).  Same workspace query.  With the bf16 `out` alone dbias can miss the 2e-2
+ * relative-L2 bound on graphs whose pairs sit in very few buckets; with out_f32 it does not. */
+gt_status gt_biased_attn_bwd_ex(const void* q, const void* k, const void* v, const void* out,
+                                const void* dout, const float* lse,
+                                const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
+                                const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                void* dq, void* dk, void* dv, float* dbias, const float* out_f32,
+                                void* workspace, size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------
  * gt_biased_attn_fwd_step -- one ring step of graph-aware context parallelism driven by the caller
@@ -231,6 +291,12 @@ size_t gt_biased_attn_bwd_step_context_bytes(const gt_batch* batch, int32_t n_he
 gt_status gt_biased_attn_bwd_step_prepare(const void* out, const void* dout, const float* lse, const uint8_t* spd,
                                           const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
                                           void* context, size_t context_bytes, void* stream);
+/* prepare_ex: the same with the fp32 forward output (the o_acc that gt_biased_attn_fwd_step leaves after its
+ * last step) for the per-query term dout_i . out_i; `out` (bf16) may then be NULL. */
+gt_status gt_biased_attn_bwd_step_prepare_ex(const void* out, const float* out_f32, const void* dout,
+                                             const float* lse, const uint8_t* spd,
+                                             const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                             void* context, size_t context_bytes, void* stream);
 gt_status gt_biased_attn_bwd_step(const void* q, const void* k, const void* v, const void* dout, const float* bias,
                                   const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
                                   int32_t q_begin, int32_t q_end,

@@ -19,16 +19,17 @@ LIB_PATH = os.environ.get("GT_ATTN_LIB", os.path.join(_HERE, "libgtattn.so"))
 
 GT_OK = 0
 STATUS_NAMES = {0: "GT_OK", 1: "GT_ERR_INVALID_ARG", 2: "GT_ERR_UNSUPPORTED", 3: "GT_ERR_WORKSPACE",
-                4: "GT_ERR_CUDA", 5: "GT_ERR_DEVICE_TIMEOUT", 6: "GT_ERR_NO_DEVICE"}
+                4: "GT_ERR_CUDA", 5: "GT_ERR_DEVICE_TIMEOUT", 6: "GT_ERR_NO_DEVICE", 7: "GT_ERR_BAD_SPD"}
 
 EXPORTS = ("gt_status_string", "gt_check",
            "gt_spd_build_workspace", "gt_spd_build", "gt_spd_build_static_limit", "gt_spd_build_static",
-           "gt_biased_attn_fwd_workspace", "gt_biased_attn_fwd",
-           "gt_biased_attn_bwd_workspace", "gt_biased_attn_bwd",
+           "gt_spd_validate_workspace", "gt_spd_validate", "gt_spd_validate_count", "gt_test_hook_barrier_overcount",
+           "gt_biased_attn_fwd_workspace", "gt_biased_attn_fwd", "gt_biased_attn_fwd_ex",
+           "gt_biased_attn_bwd_workspace", "gt_biased_attn_bwd", "gt_biased_attn_bwd_ex",
            "gt_biased_attn_fwd_chunked_workspace", "gt_biased_attn_fwd_chunked",
            "gt_biased_attn_bwd_chunked_workspace", "gt_biased_attn_bwd_chunked",
            "gt_biased_attn_fwd_step_workspace", "gt_biased_attn_fwd_step",
-           "gt_biased_attn_bwd_step_context_bytes", "gt_biased_attn_bwd_step_prepare",
+           "gt_biased_attn_bwd_step_context_bytes", "gt_biased_attn_bwd_step_prepare", "gt_biased_attn_bwd_step_prepare_ex",
            "gt_biased_attn_bwd_step", "gt_biased_attn_bwd_step_finish")
 
 
@@ -64,42 +65,52 @@ def lib() -> ctypes.CDLL:
         L.gt_spd_build_workspace.argtypes = [bp, i64, i32]
         L.gt_spd_build.restype = ctypes.c_int
         L.gt_spd_build.argtypes = [vp, vp, i64, bp, i32, vp, vp, vp, sz, vp]
-        if hasattr(L, "gt_spd_build_static"):
-            L.gt_spd_build_static_limit.restype = sz
-            L.gt_spd_build_static_limit.argtypes = []
-            L.gt_spd_build_static.restype = ctypes.c_int
-            L.gt_spd_build_static.argtypes = [vp, vp, i64, bp, i32, vp, vp, vp]
-        if hasattr(L, "gt_biased_attn_fwd"):
-            L.gt_biased_attn_fwd_workspace.restype = sz
-            L.gt_biased_attn_fwd_workspace.argtypes = [bp, i32, i32]
-            L.gt_biased_attn_fwd.restype = ctypes.c_int
-            L.gt_biased_attn_fwd.argtypes = [vp, vp, vp, vp, vp, vp, bp, i32, i32, i32, vp, vp, vp, sz, vp]
-        if hasattr(L, "gt_biased_attn_bwd"):
-            L.gt_biased_attn_bwd_workspace.restype = sz
-            L.gt_biased_attn_bwd_workspace.argtypes = [bp, i32, i32, i32]
-            L.gt_biased_attn_bwd.restype = ctypes.c_int
-            L.gt_biased_attn_bwd.argtypes = [vp] * 9 + [bp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
-        if hasattr(L, "gt_biased_attn_fwd_chunked"):
-            L.gt_biased_attn_fwd_chunked_workspace.restype = sz
-            L.gt_biased_attn_fwd_chunked_workspace.argtypes = [bp, i32, i32, i32]
-            L.gt_biased_attn_fwd_chunked.restype = ctypes.c_int
-            L.gt_biased_attn_fwd_chunked.argtypes = [vp, vp, vp, vp, vp, vp, bp, i32, i32, i32, vp, vp, i32, vp, vp, sz, vp]
-            L.gt_biased_attn_fwd_step_workspace.restype = sz
-            L.gt_biased_attn_fwd_step_workspace.argtypes = [bp, i32, i32]
-            L.gt_biased_attn_fwd_step.restype = ctypes.c_int
-            L.gt_biased_attn_fwd_step.argtypes = [vp] * 5 + [bp, i32, i32, i32] + [i32] * 6 + [vp, vp, vp, vp, sz, vp]
-            L.gt_biased_attn_bwd_step_context_bytes.restype = sz
-            L.gt_biased_attn_bwd_step_context_bytes.argtypes = [bp, i32, i32]
-            L.gt_biased_attn_bwd_step_prepare.restype = ctypes.c_int
-            L.gt_biased_attn_bwd_step_prepare.argtypes = [vp, vp, vp, vp, bp, i32, i32, i32, vp, sz, vp]
-            L.gt_biased_attn_bwd_step.restype = ctypes.c_int
-            L.gt_biased_attn_bwd_step.argtypes = [vp] * 5 + [bp, i32, i32, i32] + [i32] * 6 + [vp, vp, vp, vp, vp, sz, vp]
-            L.gt_biased_attn_bwd_step_finish.restype = ctypes.c_int
-            L.gt_biased_attn_bwd_step_finish.argtypes = [vp, vp, vp, vp, bp, i32, i32, i32, vp, vp, vp, vp, vp]
-            L.gt_biased_attn_bwd_chunked_workspace.restype = sz
-            L.gt_biased_attn_bwd_chunked_workspace.argtypes = [bp, i32, i32, i32, i32]
-            L.gt_biased_attn_bwd_chunked.restype = ctypes.c_int
-            L.gt_biased_attn_bwd_chunked.argtypes = [vp] * 8 + [bp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.gt_spd_build_static_limit.restype = sz
+        L.gt_spd_build_static_limit.argtypes = []
+        L.gt_spd_build_static.restype = ctypes.c_int
+        L.gt_spd_build_static.argtypes = [vp, vp, i64, bp, i32, vp, vp, vp]
+        L.gt_spd_validate_workspace.restype = sz
+        L.gt_spd_validate_workspace.argtypes = []
+        L.gt_spd_validate.restype = ctypes.c_int
+        L.gt_spd_validate.argtypes = [vp, vp, bp, i32, vp, sz, vp]
+        L.gt_spd_validate_count.restype = ctypes.c_int
+        L.gt_spd_validate_count.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int64)]
+        L.gt_test_hook_barrier_overcount.restype = None
+        L.gt_test_hook_barrier_overcount.argtypes = [i32]
+        L.gt_biased_attn_fwd_workspace.restype = sz
+        L.gt_biased_attn_fwd_workspace.argtypes = [bp, i32, i32]
+        L.gt_biased_attn_fwd.restype = ctypes.c_int
+        L.gt_biased_attn_fwd.argtypes = [vp, vp, vp, vp, vp, vp, bp, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.gt_biased_attn_fwd_ex.restype = ctypes.c_int
+        L.gt_biased_attn_fwd_ex.argtypes = [vp, vp, vp, vp, vp, vp, bp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+        L.gt_biased_attn_bwd_workspace.restype = sz
+        L.gt_biased_attn_bwd_workspace.argtypes = [bp, i32, i32, i32]
+        L.gt_biased_attn_bwd.restype = ctypes.c_int
+        L.gt_biased_attn_bwd.argtypes = [vp] * 9 + [bp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.gt_biased_attn_bwd_ex.restype = ctypes.c_int
+        L.gt_biased_attn_bwd_ex.argtypes = [vp] * 9 + [bp, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.gt_biased_attn_fwd_chunked_workspace.restype = sz
+        L.gt_biased_attn_fwd_chunked_workspace.argtypes = [bp, i32, i32, i32]
+        L.gt_biased_attn_fwd_chunked.restype = ctypes.c_int
+        L.gt_biased_attn_fwd_chunked.argtypes = [vp, vp, vp, vp, vp, vp, bp, i32, i32, i32, vp, vp, i32, vp, vp, sz, vp]
+        L.gt_biased_attn_fwd_step_workspace.restype = sz
+        L.gt_biased_attn_fwd_step_workspace.argtypes = [bp, i32, i32]
+        L.gt_biased_attn_fwd_step.restype = ctypes.c_int
+        L.gt_biased_attn_fwd_step.argtypes = [vp] * 5 + [bp, i32, i32, i32] + [i32] * 6 + [vp, vp, vp, vp, sz, vp]
+        L.gt_biased_attn_bwd_step_context_bytes.restype = sz
+        L.gt_biased_attn_bwd_step_context_bytes.argtypes = [bp, i32, i32]
+        L.gt_biased_attn_bwd_step_prepare.restype = ctypes.c_int
+        L.gt_biased_attn_bwd_step_prepare.argtypes = [vp, vp, vp, vp, bp, i32, i32, i32, vp, sz, vp]
+        L.gt_biased_attn_bwd_step_prepare_ex.restype = ctypes.c_int
+        L.gt_biased_attn_bwd_step_prepare_ex.argtypes = [vp, vp, vp, vp, vp, bp, i32, i32, i32, vp, sz, vp]
+        L.gt_biased_attn_bwd_step.restype = ctypes.c_int
+        L.gt_biased_attn_bwd_step.argtypes = [vp] * 5 + [bp, i32, i32, i32] + [i32] * 6 + [vp, vp, vp, vp, vp, sz, vp]
+        L.gt_biased_attn_bwd_step_finish.restype = ctypes.c_int
+        L.gt_biased_attn_bwd_step_finish.argtypes = [vp, vp, vp, vp, bp, i32, i32, i32, vp, vp, vp, vp, vp]
+        L.gt_biased_attn_bwd_chunked_workspace.restype = sz
+        L.gt_biased_attn_bwd_chunked_workspace.argtypes = [bp, i32, i32, i32, i32]
+        L.gt_biased_attn_bwd_chunked.restype = ctypes.c_int
+        L.gt_biased_attn_bwd_chunked.argtypes = [vp] * 8 + [bp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -200,6 +211,20 @@ def gt_biased_attn_fwd(q, k, v, spd, bias, batch: Batch, max_dist: int, out, lse
     return workspace
 
 
+def gt_biased_attn_fwd_ex(q, k, v, spd, bias, batch: Batch, max_dist: int, out, lse, out_f32: Optional[torch.Tensor],
+                          workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Forward that also writes the fp32 output (before its rounding to bf16) into ``out_f32``."""
+    _, H, d = q.shape
+    if workspace is None:
+        workspace = _workspace(gt_biased_attn_fwd_workspace(batch, H, d), q.device)
+    b = batch.c_struct()
+    st = lib().gt_biased_attn_fwd_ex(_ptr(q), _ptr(k), _ptr(v), _ptr(spd), _ptr(batch.spd_offsets), _ptr(bias),
+                                     ctypes.byref(b), H, d, int(max_dist), _ptr(out), _ptr(lse), _ptr(out_f32),
+                                     _ptr(workspace), workspace.numel(), _stream())
+    _raise(st, "gt_biased_attn_fwd_ex")
+    return workspace
+
+
 def gt_biased_attn_bwd_workspace(batch: Batch, n_heads: int, head_dim: int, max_dist: int) -> int:
     b = batch.c_struct()
     return int(lib().gt_biased_attn_bwd_workspace(ctypes.byref(b), n_heads, head_dim, max_dist))
@@ -217,6 +242,44 @@ def gt_biased_attn_bwd(q, k, v, out, dout, lse, spd, bias, batch: Batch, max_dis
                                   _ptr(workspace), workspace.numel(), _stream())
     _raise(st, "gt_biased_attn_bwd")
     return workspace
+
+
+def gt_biased_attn_bwd_ex(q, k, v, out, dout, lse, spd, bias, batch: Batch, max_dist: int, dq, dk, dv, dbias,
+                          out_f32: Optional[torch.Tensor], workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Backward whose per-query term dout . out is formed from the fp32 forward output ``out_f32``."""
+    _, H, d = q.shape
+    if workspace is None:
+        workspace = _workspace(gt_biased_attn_bwd_workspace(batch, H, d, max_dist), q.device)
+    b = batch.c_struct()
+    st = lib().gt_biased_attn_bwd_ex(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(dout), _ptr(lse), _ptr(spd),
+                                     _ptr(batch.spd_offsets), _ptr(bias), ctypes.byref(b), H, d, int(max_dist),
+                                     _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dbias), _ptr(out_f32),
+                                     _ptr(workspace), workspace.numel(), _stream())
+    _raise(st, "gt_biased_attn_bwd_ex")
+    return workspace
+
+
+def gt_spd_validate(spd, batch: Batch, max_dist: int, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Enqueue the check of an SPD matrix for entries that name no bucket; ``gt_check`` on the returned
+    workspace raises GtError(GT_ERR_BAD_SPD) if there are any, ``gt_spd_validate_count`` gives their number."""
+    if workspace is None:
+        workspace = _workspace(int(lib().gt_spd_validate_workspace()), spd.device)
+    b = batch.c_struct()
+    st = lib().gt_spd_validate(_ptr(spd), _ptr(batch.spd_offsets), ctypes.byref(b), int(max_dist),
+                               _ptr(workspace), workspace.numel(), _stream())
+    _raise(st, "gt_spd_validate")
+    return workspace
+
+
+def gt_spd_validate_count(workspace: torch.Tensor) -> int:
+    c = ctypes.c_int64(0)
+    _raise(lib().gt_spd_validate_count(_ptr(workspace), _stream(), ctypes.byref(c)), "gt_spd_validate_count")
+    return int(c.value)
+
+
+def gt_test_hook_barrier_overcount(extra: int) -> None:
+    """Test hook: the next bit-matrix SPD build waits for ``extra`` thread blocks that do not exist."""
+    lib().gt_test_hook_barrier_overcount(int(extra))
 
 
 def gt_biased_attn_fwd_chunked_workspace(batch: Batch, n_heads: int, head_dim: int, n_kv_chunks: int) -> int:
@@ -286,13 +349,20 @@ def gt_biased_attn_bwd_step_context_bytes(batch: Batch, n_heads: int, head_dim: 
 
 
 def gt_biased_attn_bwd_step_prepare(out, dout, lse, spd, batch: Batch, max_dist: int,
-                                    context: Optional[torch.Tensor] = None) -> torch.Tensor:
-    _, H, d = out.shape
+                                    context: Optional[torch.Tensor] = None,
+                                    out_f32: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """``out_f32`` (the fp32 o_acc of the forward steps) selects gt_biased_attn_bwd_step_prepare_ex."""
+    _, H, d = dout.shape
     if context is None:
-        context = _workspace(gt_biased_attn_bwd_step_context_bytes(batch, H, d), out.device)
+        context = _workspace(gt_biased_attn_bwd_step_context_bytes(batch, H, d), dout.device)
     b = batch.c_struct()
-    st = lib().gt_biased_attn_bwd_step_prepare(_ptr(out), _ptr(dout), _ptr(lse), _ptr(spd), ctypes.byref(b), H, d,
-                                               int(max_dist), _ptr(context), context.numel(), _stream())
+    if out_f32 is None:
+        st = lib().gt_biased_attn_bwd_step_prepare(_ptr(out), _ptr(dout), _ptr(lse), _ptr(spd), ctypes.byref(b), H, d,
+                                                   int(max_dist), _ptr(context), context.numel(), _stream())
+    else:
+        st = lib().gt_biased_attn_bwd_step_prepare_ex(_ptr(out), _ptr(out_f32), _ptr(dout), _ptr(lse), _ptr(spd),
+                                                      ctypes.byref(b), H, d, int(max_dist),
+                                                      _ptr(context), context.numel(), _stream())
     _raise(st, "gt_biased_attn_bwd_step_prepare")
     return context
 

@@ -32,6 +32,7 @@ extern "C" const char* gt_status_string(gt_status s)
         case GT_ERR_CUDA: return "GT_ERR_CUDA";
         case GT_ERR_DEVICE_TIMEOUT: return "GT_ERR_DEVICE_TIMEOUT";
         case GT_ERR_NO_DEVICE: return "GT_ERR_NO_DEVICE";
+        case GT_ERR_BAD_SPD: return "GT_ERR_BAD_SPD";
     }
     return "GT_ERR_UNKNOWN";
 }
@@ -46,7 +47,7 @@ extern "C" gt_status gt_check(void* workspace, void* stream)
     if (words[0] != 0u) {
         if (getenv("GT_DEBUG")) fprintf(stderr, "[gt_attn] device status %u at wait site %u\n", words[0], words[1]);
         GT_CUDA_TRY(cudaMemset(workspace, 0, sizeof(words)));
-        return words[0] <= (uint32_t)GT_ERR_NO_DEVICE ? (gt_status)words[0] : GT_ERR_CUDA;
+        return words[0] <= (uint32_t)GT_ERR_BAD_SPD ? (gt_status)words[0] : GT_ERR_CUDA;
     }
     return GT_OK;
 }

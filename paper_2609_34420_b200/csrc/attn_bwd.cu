@@ -643,7 +643,8 @@ __global__ void __launch_bounds__(256) spd_transpose_clamp_kernel(const uint8_t*
 }
 
 // For every (t, h): ext[t][h][0..2] = three-term bf16 split of -lse * sqrt(d), ext[t][h][8..10] = split of
-// -Delta with Delta = sum_c dO[t,h,c] * O[t,h,c], zeros elsewhere.
+// -Delta with Delta = sum_c dO[t,h,c] * O[t,h,c], zeros elsewhere.  O is taken from `out_f32` (the forward
+// output before its rounding to bf16) when the caller has it, else from the bf16 `out`.
 __device__ __forceinline__ void split3_bf16(float v, uint32_t& w01, uint32_t& w2)
 {
     const __nv_bfloat16 hi = __float2bfloat16_rn(v);
@@ -655,24 +656,38 @@ __device__ __forceinline__ void split3_bf16(float v, uint32_t& w01, uint32_t& w2
 }
 
 template <int D>
-__global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
+__global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ out, const float* __restrict__ out_f32,
+                                      const __nv_bfloat16* __restrict__ dout,
                                       const float* __restrict__ lse, uint4* __restrict__ ext,
                                       int32_t n_total, int32_t n_heads, float sqrt_d)
 {
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;      // = t * H + h
     if (idx >= (size_t)n_total * n_heads) return;
     const int32_t t = (int32_t)(idx / n_heads), h = (int32_t)(idx % n_heads);
-    const uint4* o4 = (const uint4*)(out + idx * D);
     const uint4* d4 = (const uint4*)(dout + idx * D);
     float acc = 0.f;
+    if (out_f32 != nullptr) {
+        const float4* o4 = (const float4*)(out_f32 + idx * D);
 #pragma unroll
-    for (int i = 0; i < D / 8; ++i) {
-        const uint4 a = o4[i], b = d4[i];
-        const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+        for (int i = 0; i < D / 8; ++i) {
+            const float4 a0 = o4[2 * i], a1 = o4[2 * i + 1];
+            const uint4 b = d4[i];
+            acc += a0.x * __uint_as_float(b.x << 16) + a0.y * __uint_as_float(b.x & 0xffff0000u);
+            acc += a0.z * __uint_as_float(b.y << 16) + a0.w * __uint_as_float(b.y & 0xffff0000u);
+            acc += a1.x * __uint_as_float(b.z << 16) + a1.y * __uint_as_float(b.z & 0xffff0000u);
+            acc += a1.z * __uint_as_float(b.w << 16) + a1.w * __uint_as_float(b.w & 0xffff0000u);
+        }
+    } else {
+        const uint4* o4 = (const uint4*)(out + idx * D);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            acc += __uint_as_float(aw[k] << 16) * __uint_as_float(bw[k] << 16);
-            acc += __uint_as_float(aw[k] & 0xffff0000u) * __uint_as_float(bw[k] & 0xffff0000u);
+        for (int i = 0; i < D / 8; ++i) {
+            const uint4 a = o4[i], b = d4[i];
+            const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                acc += __uint_as_float(aw[k] << 16) * __uint_as_float(bw[k] << 16);
+                acc += __uint_as_float(aw[k] & 0xffff0000u) * __uint_as_float(bw[k] & 0xffff0000u);
+            }
         }
     }
     uint4 e0 = make_uint4(0u, 0u, 0u, 0u), e1 = make_uint4(0u, 0u, 0u, 0u);
@@ -755,7 +770,7 @@ extern "C" size_t gt_biased_attn_bwd_workspace(const gt_batch* batch, int32_t n_
 // Shared by the one-shot and the chunked entry point: pre-passes, one launch of the main kernel per key chunk
 // (the chunks run one after the other in stream order, like ring steps; dQ and dB accumulate across them,
 // dK and dV of a chunk's rows are complete when its launch ends), then the final conversion.
-static gt_status gt_bwd_run(const void* q, const void* k, const void* v, const void* out,
+static gt_status gt_bwd_run(const void* q, const void* k, const void* v, const void* out, const float* out_f32,
                             const void* dout, const float* lse,
                             const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
                             const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
@@ -767,7 +782,7 @@ static gt_status gt_bwd_run(const void* q, const void* k, const void* v, const v
     if (st != GT_OK) return st;
     if (!q || !k || !v || !out || !dout || !lse || !spd || !bias || !dq || !dk || !dv || !dbias) return GT_ERR_INVALID_ARG;
     if (misaligned16(q) || misaligned16(k) || misaligned16(v) || misaligned16(out) || misaligned16(dout) ||
-        misaligned16(spd) || misaligned16(dq) || misaligned16(dk) || misaligned16(dv))
+        misaligned16(spd) || misaligned16(dq) || misaligned16(dk) || misaligned16(dv) || (out_f32 && misaligned16(out_f32)))
         return GT_ERR_INVALID_ARG;
     if (n_heads > 65535 || batch->n_graphs > 65535) return GT_ERR_UNSUPPORTED;
     const BwdWorkspace wsp = bwd_workspace(batch, n_heads, head_dim, max_dist, n_kv_chunks);
@@ -816,10 +831,10 @@ static gt_status gt_bwd_run(const void* q, const void* k, const void* v, const v
     const unsigned pre_blocks = (unsigned)((rows + 255) / 256);
     uint4* ext = (uint4*)(ws + wsp.ext_off);
     if (head_dim == 64)
-        bwd_preprocess_kernel<64><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse,
+        bwd_preprocess_kernel<64><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, out_f32, (const __nv_bfloat16*)dout, lse,
                                                              ext, batch->n_total, n_heads, sqrtf(64.f));
     else
-        bwd_preprocess_kernel<32><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse,
+        bwd_preprocess_kernel<32><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, out_f32, (const __nv_bfloat16*)dout, lse,
                                                              ext, batch->n_total, n_heads, sqrtf(32.f));
     GT_CUDA_TRY(cudaGetLastError());
     CUtensorMap text;
@@ -854,7 +869,18 @@ extern "C" gt_status gt_biased_attn_bwd(const void* q, const void* k, const void
                                         void* dq, void* dk, void* dv, float* dbias,
                                         void* workspace, size_t workspace_bytes, void* stream)
 {
-    return gt_bwd_run(q, k, v, out, dout, lse, spd, spd_offsets, bias, batch, n_heads, head_dim, max_dist,
+    return gt_bwd_run(q, k, v, out, nullptr, dout, lse, spd, spd_offsets, bias, batch, n_heads, head_dim, max_dist,
+                      dq, dk, dv, dbias, 1, nullptr, workspace, workspace_bytes, stream);
+}
+
+extern "C" gt_status gt_biased_attn_bwd_ex(const void* q, const void* k, const void* v, const void* out,
+                                           const void* dout, const float* lse,
+                                           const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
+                                           const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                           void* dq, void* dk, void* dv, float* dbias, const float* out_f32,
+                                           void* workspace, size_t workspace_bytes, void* stream)
+{
+    return gt_bwd_run(q, k, v, out, out_f32, dout, lse, spd, spd_offsets, bias, batch, n_heads, head_dim, max_dist,
                       dq, dk, dv, dbias, 1, nullptr, workspace, workspace_bytes, stream);
 }
 
@@ -875,7 +901,7 @@ extern "C" gt_status gt_biased_attn_bwd_chunked(const void* q, const void* k, co
 {
     if (batch == nullptr || batch->n_graphs != 1) return GT_ERR_UNSUPPORTED;
     if (n_kv_chunks < 1 || n_kv_chunks > 4096) return GT_ERR_INVALID_ARG;
-    return gt_bwd_run(q, k, v, out, dout, lse, spd, nullptr, bias, batch, n_heads, head_dim, max_dist,
+    return gt_bwd_run(q, k, v, out, nullptr, dout, lse, spd, nullptr, bias, batch, n_heads, head_dim, max_dist,
                       dq, dk, dv, dbias, n_kv_chunks, dbias_chunks, workspace, workspace_bytes, stream);
 }
 
@@ -936,11 +962,22 @@ extern "C" gt_status gt_biased_attn_bwd_step_prepare(const void* out, const void
                                                      const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
                                                      void* context, size_t context_bytes, void* stream)
 {
+    return gt_biased_attn_bwd_step_prepare_ex(out, nullptr, dout, lse, spd, batch, n_heads, head_dim, max_dist,
+                                              context, context_bytes, stream);
+}
+
+extern "C" gt_status gt_biased_attn_bwd_step_prepare_ex(const void* out, const float* out_f32, const void* dout,
+                                                        const float* lse, const uint8_t* spd,
+                                                        const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                                        void* context, size_t context_bytes, void* stream)
+{
     using namespace gt;
     gt_status st = validate_attn_common(batch, n_heads, head_dim, max_dist, nullptr);
     if (st != GT_OK) return st;
     if (batch->n_graphs != 1) return GT_ERR_UNSUPPORTED;
-    if (!out || !dout || !lse || !spd || misaligned16(out) || misaligned16(dout) || misaligned16(spd)) return GT_ERR_INVALID_ARG;
+    if ((!out && !out_f32) || !dout || !lse || !spd || (out && misaligned16(out)) || (out_f32 && misaligned16(out_f32)) ||
+        misaligned16(dout) || misaligned16(spd))
+        return GT_ERR_INVALID_ARG;
     const StepContext cx = step_context(batch, n_heads);
     if (context == nullptr || context_bytes < cx.total || misaligned16(context)) return GT_ERR_WORKSPACE;
     if (sm_count() <= 0) return GT_ERR_NO_DEVICE;
@@ -955,10 +992,10 @@ extern "C" gt_status gt_biased_attn_bwd_step_prepare(const void* out, const void
     const unsigned pre_blocks = (unsigned)((rows + 255) / 256);
     uint4* ext = (uint4*)(ws + cx.ext_off);
     if (head_dim == 64)
-        bwd_preprocess_kernel<64><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse, ext,
+        bwd_preprocess_kernel<64><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, out_f32, (const __nv_bfloat16*)dout, lse, ext,
                                                              batch->n_total, n_heads, sqrtf(64.f));
     else
-        bwd_preprocess_kernel<32><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, (const __nv_bfloat16*)dout, lse, ext,
+        bwd_preprocess_kernel<32><<<pre_blocks, 256, 0, s>>>((const __nv_bfloat16*)out, out_f32, (const __nv_bfloat16*)dout, lse, ext,
                                                              batch->n_total, n_heads, sqrtf(32.f));
     GT_CUDA_TRY(cudaGetLastError());
     return GT_OK;

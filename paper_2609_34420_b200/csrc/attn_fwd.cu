@@ -65,6 +65,7 @@ struct FwdParams {
     const int32_t* cu_seqlens;
     const float* bias;
     __nv_bfloat16* out;        // [T,H,D]          (unchunked)
+    float* out_f32;            // [T,H,D] fp32     (unchunked, optional: the output before its rounding to bf16)
     float* lse;                // [H,T]            (unchunked)
     float* part_o;             // [C,T,H,D] fp32   (chunked)
     float* part_lse;           // [C,H,T]          (chunked)
@@ -132,7 +133,12 @@ __device__ __forceinline__ void tmem_st(uint32_t taddr, const uint32_t (&r)[N])
     if constexpr (N == 32) tmem_st32(taddr, r); else tmem_st16(taddr, r);
 }
 
-template <int D, bool kPartial, bool kShflBias>
+// kPrecise (the fp32-output entry point): P goes to the P V MMA as TWO bf16 terms, P = hi + lo with
+// lo = bf16(P - hi) (16 mantissa bits instead of 8), so that the output is accurate to fp32 accumulation
+// instead of to the 2^-9 relative rounding of a bf16 P.  The two terms of a 16-key chunk overwrite that
+// chunk's own score columns ([0,8) hi, [8,16) lo) as soon as the chunk has been read, which needs the
+// tile's maximum first: the precise variant always takes the classical two-pass way.
+template <int D, bool kPartial, bool kShflBias, bool kPrecise = false>
 __global__ void __launch_bounds__(kFwdThreads, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_spd,
@@ -279,10 +285,19 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     mbar_wait(bar(kBarPFull + 2 * t + (j & 1)), (j >> 1) & 1, abort_flag, p.status, 24);
                     tc_fence_after();
                     if (elect_one()) {
+                        if constexpr (kPrecise) {
+#pragma unroll
+                            for (int k = 0; k < kKvTile / 16; ++k) {    // hi and lo term of key chunk k at the start of its own 16 score columns
+                                const uint32_t a = tm + b * 128 + (k / (kCols / 16)) * kCols + (k % (kCols / 16)) * 16;
+                                mma_ts(tm + 384 + t * 64, a, advance_desc(dv, k * 16 * L::kRowBytes), idesc_o, k > 0 ? 1u : acc0);
+                                mma_ts(tm + 384 + t * 64, a + 8, advance_desc(dv, k * 16 * L::kRowBytes), idesc_o, 1u);
+                            }
+                        } else {
 #pragma unroll
                         for (int k = 0; k < kKvTile / 16; ++k)      // P of key half hf sits at the start of that half's score columns
                             mma_ts(tm + 384 + t * 64, tm + b * 128 + (k / (kCols / 16)) * kCols + (k % (kCols / 16)) * 8,
                                    advance_desc(dv, k * 16 * L::kRowBytes), idesc_o, k > 0 ? 1u : acc0);
+                        }
                         mma_commit(bar(kBarODone + 2 * t + (j & 1)));
                         mma_commit(bar(kBarBufFree + b));
                         if (t == 1) mma_commit(bar(kBarVEmpty + vs));
@@ -378,7 +393,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             uint32_t pk[kCols / 64][32];           // P of this thread's columns, bf16 pairs
             float tile_sum = 0.f;
             bool loaded = true;                    // chunk 0 is already on its way
-            bool exact = (j == 0);                 // take the tile maximum first
+            bool exact = kPrecise || (j == 0);     // take the tile maximum first
 
             for (;;) {
                 if (exact) {
@@ -438,6 +453,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 const uint64_t neg_m = pack_f32x2(-m, -m);
                 uint64_t sum2 = pack_f32x2(0.f, 0.f);
                 auto exp_chunk = [&](int c, const uint32_t (&sr)[kCW], const uint4 (&ws)[kCW / 16], auto rag) {
+                    [[maybe_unused]] uint32_t hl[kCW];   // precise variant: hi terms of the chunk, then its lo terms
 #pragma unroll
                     for (int q = 0; q < kCW / 8; ++q) {
                         const uint4& ww = ws[q >> 1];
@@ -456,9 +472,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                             lo = ex2_approx(lo);
                             hi = ex2_approx(hi);
                             sum2 = add_f32x2(sum2, pack_f32x2(lo, hi));
-                            pk[(c * (kCW / 2) + q * 4 + i) >> 5][(c * (kCW / 2) + q * 4 + i) & 31] = pack_bf16x2(lo, hi);
+                            const uint32_t top = pack_bf16x2(lo, hi);
+                            if constexpr (kPrecise) {
+                                hl[q * 4 + i] = top;
+                                hl[kCW / 2 + q * 4 + i] = pack_bf16x2(lo - __uint_as_float(top << 16), hi - __uint_as_float(top & 0xffff0000u));
+                            } else {
+                                pk[(c * (kCW / 2) + q * 4 + i) >> 5][(c * (kCW / 2) + q * 4 + i) & 31] = top;
+                            }
                         }
                     }
+                    if constexpr (kPrecise) tmem_st<kCW>(tS + c * kCW, hl);      // over the chunk's own score columns (already in registers)
                 };
                 auto exp_pass = [&](auto rag) {
                     if (!loaded) load_chunk(0, sa, wa);
@@ -488,8 +511,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             l += tile_sum;
 
             // P over the first half of this thread's own score columns
+            if constexpr (!kPrecise) {
 #pragma unroll
-            for (int c = 0; c < kCols / 64; ++c) tmem_st32(tS + c * 32, pk[c]);
+                for (int c = 0; c < kCols / 64; ++c) tmem_st32(tS + c * 32, pk[c]);
+            }
             tmem_wait_st();
             tc_fence_before();
             // Warps of a tile can be one step apart (nothing in the speculative pass waits for the
@@ -568,6 +593,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         v.z = pack_bf16x2(__uint_as_float(o[8 * i + 4]) * inv_l, __uint_as_float(o[8 * i + 5]) * inv_l);
                         v.w = pack_bf16x2(__uint_as_float(o[8 * i + 6]) * inv_l, __uint_as_float(o[8 * i + 7]) * inv_l);
                         dst[i] = v;
+                    }
+                    if (p.out_f32 != nullptr) {
+                        float4* dst32 = (float4*)(p.out_f32 + ((size_t)(node0 + q) * p.n_heads + h) * D + hf * kOC + c * kOP);
+#pragma unroll
+                        for (int i = 0; i < kOP / 4; ++i)
+                            dst32[i] = make_float4(__uint_as_float(o[4 * i]) * inv_l, __uint_as_float(o[4 * i + 1]) * inv_l,
+                                                   __uint_as_float(o[4 * i + 2]) * inv_l, __uint_as_float(o[4 * i + 3]) * inv_l);
                     }
                 }
             }
@@ -683,6 +715,10 @@ gt_status launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtenso
                      const FwdParams& p, const gt_batch* batch, int grid_z, cudaStream_t s, int grid_y = 0)
 {
     auto kern = p.n_buckets <= 32 ? attn_fwd_kernel<D, kPartial, true> : attn_fwd_kernel<D, kPartial, false>;
+    if constexpr (!kPartial) {
+        if (p.out_f32 != nullptr)
+            kern = p.n_buckets <= 32 ? attn_fwd_kernel<D, false, true, true> : attn_fwd_kernel<D, false, false, true>;
+    }
     GT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<D>::kDynamic));
     dim3 grid((unsigned)p.n_heads, (unsigned)(grid_y > 0 ? grid_y : (batch->max_seqlen + kRowsPerCta - 1) / kRowsPerCta), (unsigned)grid_z);
     kern<<<grid, kFwdThreads, FwdSmem<D>::kDynamic, s>>>(tq, tk, tv, tspd, p);
@@ -717,9 +753,20 @@ extern "C" gt_status gt_biased_attn_fwd(const void* q, const void* k, const void
                                         void* out, float* lse,
                                         void* workspace, size_t workspace_bytes, void* stream)
 {
+    return gt_biased_attn_fwd_ex(q, k, v, spd, spd_offsets, bias, batch, n_heads, head_dim, max_dist, out, lse, nullptr,
+                                 workspace, workspace_bytes, stream);
+}
+
+extern "C" gt_status gt_biased_attn_fwd_ex(const void* q, const void* k, const void* v,
+                                           const uint8_t* spd, const int64_t* spd_offsets, const float* bias,
+                                           const gt_batch* batch, int32_t n_heads, int32_t head_dim, int32_t max_dist,
+                                           void* out, float* lse, float* out_f32,
+                                           void* workspace, size_t workspace_bytes, void* stream)
+{
     using namespace gt;
     gt_status st = check_fwd_args(q, k, v, spd, spd_offsets, bias, batch, n_heads, head_dim, max_dist, out, lse);
     if (st != GT_OK) return st;
+    if (out_f32 != nullptr && misaligned16(out_f32)) return GT_ERR_INVALID_ARG;
     if (workspace == nullptr || workspace_bytes < kHeaderBytes || misaligned16(workspace)) return GT_ERR_WORKSPACE;
     if (sm_count() <= 0) return GT_ERR_NO_DEVICE;
     CUtensorMap tq, tk, tv;
@@ -735,6 +782,7 @@ extern "C" gt_status gt_biased_attn_fwd(const void* q, const void* k, const void
     p.cu_seqlens = batch->n_graphs > 1 ? batch->cu_seqlens : nullptr;
     p.bias = bias;
     p.out = (__nv_bfloat16*)out;
+    p.out_f32 = out_f32;
     p.lse = lse;
     p.status = (uint32_t*)workspace;
     p.n_total = batch->n_total;

@@ -255,6 +255,8 @@ struct DenseParams {
     int32_t n_max;
     int32_t n_pad;          // n_max rounded up to 32: pitch of the flag arrays
     int32_t n_groups;       // CTA groups that work on different column blocks at the same time (own state each)
+    uint32_t barrier_extra; // test hook: arrivals the grid barrier waits for beyond the thread blocks that exist (normally 0)
+    uint32_t barrier_limit; // polls of the barrier word before a thread block gives up
 };
 
 // item_start[v] = sum_{u<v} max(1, ceil(deg(u)/64)) for the vertices of one graph.  One block.
@@ -300,17 +302,18 @@ __global__ void spd_dense_item_rec_kernel(const int32_t* __restrict__ rp, const 
 
 // Grid barrier with a bounded wait (the kernel is launched cooperatively, so all CTAs are resident).
 // Returns false once any CTA has given up; every CTA then leaves the kernel.
-__device__ __forceinline__ bool dense_grid_sync(uint32_t* sync, uint32_t& epoch, uint32_t* status, uint32_t n_ctas)
+__device__ __forceinline__ bool dense_grid_sync(uint32_t* sync, uint32_t& epoch, uint32_t* status, uint32_t n_ctas,
+                                                uint32_t extra, uint32_t limit)
 {
     __shared__ uint32_t s_ok;
     ++epoch;
     __syncthreads();
     if (threadIdx.x == 0) {
-        const uint32_t target = epoch * n_ctas;
+        const uint32_t target = epoch * n_ctas + extra;
         __threadfence();
         atomicAdd(&sync[0], 1u);
         uint32_t ok = 0;
-        for (uint32_t it = 0; it < kGridWaitIterations; ++it) {
+        for (uint32_t it = 0; it < limit; ++it) {
             if (*(volatile uint32_t*)&sync[0] >= target) { ok = 1; break; }
             if (*(volatile uint32_t*)&sync[1]) break;
             __nanosleep(32);
@@ -504,7 +507,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
             if (lane < kDensePlanes) d.nonempty[(size_t)lane * d.n_pad + s] = (lane == 0 && mine) ? 1 : 0;
             if (lane == 0) d.row_done[s] = 0;
         }
-        if (!dense_grid_sync(d.sync, epoch, p.header, n_ctas)) return;
+        if (!dense_grid_sync(d.sync, epoch, p.header, n_ctas, d.barrier_extra, d.barrier_limit)) return;
 
         bool emitted = false;                  // the output pass of this column block has run
         for (int level = 1;; ++level) {
@@ -646,7 +649,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                 }
               }
             }
-            if (!dense_grid_sync(d.sync, epoch, p.header, n_ctas)) return;
+            if (!dense_grid_sync(d.sync, epoch, p.header, n_ctas, d.barrier_extra, d.barrier_limit)) return;
             const uint32_t any = *(volatile uint32_t*)&d.sync[2 + flag_idx];
             if (cta == 0 && threadIdx.x == 0) {                 // next written two levels from now
                 d.sync[2 + ((step + 2u) & 3u)] = 0u;
@@ -657,7 +660,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                 emit_rows(col0, level);
                 emitted = true;
                 // levels that follow blend into rows this pass wrote from other SMs
-                if (any && !dense_grid_sync(d.sync, epoch, p.header, n_ctas)) return;
+                if (any && !dense_grid_sync(d.sync, epoch, p.header, n_ctas, d.barrier_extra, d.barrier_limit)) return;
             }
             if (!any) break;
         }
@@ -665,6 +668,9 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
         // bit matrices until the barrier behind it
     }
 }
+
+// Test hook (gt_test_hook_barrier_overcount): consumed by the next bit-matrix build of this process.
+uint32_t g_barrier_overcount = 0;
 
 size_t spd_state_bytes(int32_t max_seqlen) { return (size_t)3 * (size_t)max_seqlen * sizeof(uint32_t); }
 constexpr size_t kSmemStateLimit = 200 * 1024;
@@ -793,6 +799,9 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
         d.n_max = batch->n_total;
         d.n_pad = (int32_t)align_up((size_t)batch->n_total, 32);
         d.n_groups = pl.dense_groups;
+        d.barrier_extra = g_barrier_overcount;
+        d.barrier_limit = g_barrier_overcount ? (1u << 17) : kGridWaitIterations;      // the hooked wait gives up within a second
+        g_barrier_overcount = 0;
         // accumulator rows, their counters and the barrier words start at zero
         GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[2], 0, pl.dense_off[4] - pl.dense_off[2], s));
         GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[7], 0, 256 * kDenseMaxGroups, s));
@@ -812,6 +821,11 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
     }
     GT_CUDA_TRY(cudaGetLastError());
     return GT_OK;
+}
+
+extern "C" void gt_test_hook_barrier_overcount(int32_t extra)
+{
+    gt::g_barrier_overcount = extra > 0 ? (uint32_t)extra : 0u;
 }
 
 // ------------------------------------------------------------------------------------------

@@ -42,6 +42,21 @@ def rel_l2(x: np.ndarray, r: np.ndarray) -> float:
     return float(np.linalg.norm((x - r).reshape(-1))) / (den if den > 0 else 1.0)
 
 
+def localized_rel_l2(x: np.ndarray, r: np.ndarray, block: int = 128) -> dict:
+    """Relative-L2 error of a [rows, H, d] gradient per head and per block of `block` consecutive rows
+    (each over all heads), worst of each: an error confined to one head, one tile of rows or one row cannot
+    hide in the norm of the whole tensor.  A block is measured against its own norm, but not below the
+    average block norm (a block of nearly zero gradient has no meaningful relative error)."""
+    n = x.shape[0]
+    per_head = max(rel_l2(x[:, h], r[:, h]) for h in range(x.shape[1]))
+    n_blocks = (n + block - 1) // block
+    err = np.array([np.linalg.norm((x[b * block:(b + 1) * block] - r[b * block:(b + 1) * block]).reshape(-1)) for b in range(n_blocks)])
+    ref = np.array([np.linalg.norm(r[b * block:(b + 1) * block].reshape(-1)) for b in range(n_blocks)])
+    floor = float(np.sqrt((ref ** 2).mean()))
+    den = np.maximum(ref, floor)
+    return {"head": per_head, "block": float((err / np.where(den > 0, den, 1.0)).max())}
+
+
 class DeviceCase:
     """A workload moved to the device, with the SPD either from the oracle (default, so that
     attention parity does not depend on the SPD kernel) or from gt_spd_build."""
@@ -69,6 +84,23 @@ class DeviceCase:
         ws = gt.gt_biased_attn_fwd(self.q, self.k, self.v, self.spd, self.bias, self.batch, self.w.max_dist, out, lse)
         gt.gt_check(ws)
         return out, lse
+
+    def forward_ex(self):
+        """Forward that also returns the fp32 output (before its rounding to bf16)."""
+        out = torch.full((self.T, self.H, self.d), float("nan"), dtype=torch.bfloat16, device=self.q.device)
+        out32 = torch.full((self.T, self.H, self.d), float("nan"), dtype=torch.float32, device=self.q.device)
+        lse = torch.full((self.H, self.T), float("nan"), dtype=torch.float32, device=self.q.device)
+        ws = gt.gt_biased_attn_fwd_ex(self.q, self.k, self.v, self.spd, self.bias, self.batch, self.w.max_dist, out, lse, out32)
+        gt.gt_check(ws)
+        return out, lse, out32
+
+    def backward_ex(self, out, lse, out32):
+        dq, dk, dv = (torch.full_like(self.q, float("nan")) for _ in range(3))
+        dbias = torch.full_like(self.bias, float("nan"))
+        ws = gt.gt_biased_attn_bwd_ex(self.q, self.k, self.v, out, self.dout, lse, self.spd, self.bias, self.batch,
+                                      self.w.max_dist, dq, dk, dv, dbias, out32)
+        gt.gt_check(ws)
+        return dq, dk, dv, dbias
 
     def forward_chunked(self, n_chunks, want_chunk_lse=False):
         out = torch.full((self.T, self.H, self.d), float("nan"), dtype=torch.bfloat16, device=self.q.device)

@@ -72,12 +72,103 @@ def test_named_workloads(name):
     check(wl.make_workload(name))
 
 
-def test_large_state_in_global_memory_matches_and_is_deterministic():
-    """n above the shared-memory state limit exercises the workspace-resident state."""
+def test_single_graph_beyond_the_shared_memory_state_matches_and_is_deterministic():
+    """A single graph above the shared-memory state limit (17 066 nodes) takes the bit-matrix build."""
     w = wl.Workload("pl20k", wl.pack_graphs([wl.chung_lu_power_law(20000, 8.0, 2.1, 3)]), 1, 32, 10)
     a = check(w)
     b = gpu_spd(w).cpu().numpy()
     np.testing.assert_array_equal(a, b)
+
+
+def test_packed_batch_with_a_graph_beyond_the_shared_memory_state():
+    """A packed batch that contains a graph above the shared-memory limit runs the multi-source BFS with its
+    frontier / next / visited words in the workspace (atomics and plain loads on the same L2-resident words).
+    Directed, with a hub of several thousand out-edges, vertices without out-edges and isolated vertices;
+    two tiny graphs ride along.  Bit-exact against the oracle, twice."""
+    n = 18000
+    rng = np.random.Generator(np.random.PCG64(77))
+    m = 2 * n
+    src = np.concatenate([rng.integers(0, n - 300, m), np.full(4000, 11)])
+    dst = np.concatenate([rng.integers(0, n - 150, m), rng.choice(n - 150, 4000, replace=False)])
+    big = wl.csr_from_edges(n, src, dst, symmetric=False)
+    mid = wl.random_directed(300, 2.0, 5)
+    tiny = wl.random_directed(5, 1.5, 6)
+    w = wl.Workload("packed_big", wl.pack_graphs([big, mid, tiny]), 1, 32, 9)
+    from gpu_util import device_batch
+    from paper_2609_34420_b200 import binding as gt
+    assert gt.gt_spd_build_workspace(device_batch(w.batch), int(w.batch.col_idx.size), 9) > 12 * n    # per-CTA state slices
+    a = check(w)
+    b = gpu_spd(w).cpu().numpy()
+    np.testing.assert_array_equal(a, b)
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    """Device-timeout path end to end: the test hook makes the grid barrier of the next bit-matrix build wait
+    for a thread block that does not exist; the bounded wait gives up, every thread block returns (the kernel
+    has no asynchronous copies in flight), gt_check reports GT_ERR_DEVICE_TIMEOUT and clears the status word,
+    and the same workspace then serves a normal, bit-exact build."""
+    from gpu_util import device_batch, device_csr
+    from paper_2609_34420_b200 import binding as gt
+    w = wl.Workload("pl18k", wl.pack_graphs([wl.chung_lu_power_law(18000, 6.0, 2.1, 9)]), 1, 32, 8)
+    bt = device_batch(w.batch)
+    rp, ci = device_csr(w.batch)
+    out = torch.empty(w.batch.spd_bytes, dtype=torch.uint8, device="cuda")
+    ws = gt._workspace(gt.gt_spd_build_workspace(bt, int(ci.numel()), w.max_dist), "cuda")
+    gt.gt_test_hook_barrier_overcount(1)
+    gt.gt_spd_build(rp, ci, bt, w.max_dist, out, ws)
+    with pytest.raises(gt.GtError) as e:
+        gt.gt_check(ws)
+    assert e.value.status == 5                      # GT_ERR_DEVICE_TIMEOUT
+    gt.gt_check(ws)                                 # cleared by the report
+    gt.gt_spd_build(rp, ci, bt, w.max_dist, out, ws)
+    gt.gt_check(ws)
+    exp = ospd.spd_packed(w.batch.row_ptr, w.batch.col_idx, w.batch.cu_seqlens, w.max_dist)
+    np.testing.assert_array_equal(out.cpu().numpy(), exp)
+
+
+def test_spd_validate_counts_entries_that_name_no_bucket():
+    from gpu_util import device_batch
+    from paper_2609_34420_b200 import binding as gt
+    w = wl.small_workload([5, 33, 1, 64, 200, 16, 2, 97], 1, 32, 6, seed=4, avg_degree=1.7)
+    b = w.batch
+    bt = device_batch(b)
+    spd = ospd.spd_packed(b.row_ptr, b.col_idx, b.cu_seqlens, w.max_dist).copy()
+    good = torch.from_numpy(spd).cuda()
+    ws = gt.gt_spd_validate(good, bt, w.max_dist)
+    gt.gt_check(ws)                                 # padding bytes (255) are outside the valid region
+    assert gt.gt_spd_validate_count(ws) == 0
+    # plant invalid bytes inside valid regions: first and last valid byte of a row, a one-node graph, a tail word
+    planted = 0
+    for g, (i, j) in ((4, (0, 0)), (4, (199, 199)), (2, (0, 0)), (7, (96, 93)), (1, (32, 32)), (4, (17, 130))):
+        n_g = int(b.cu_seqlens[g + 1] - b.cu_seqlens[g])
+        ld = (n_g + 15) // 16 * 16
+        spd[int(b.spd_offsets[g]) + i * ld + j] = w.max_dist + 2 + planted      # >= n_buckets
+        planted += 1
+    bad = torch.from_numpy(spd).cuda()
+    ws = gt.gt_spd_validate(bad, bt, w.max_dist)
+    with pytest.raises(gt.GtError) as e:
+        gt.gt_check(ws)
+    assert e.value.status == 7                      # GT_ERR_BAD_SPD
+    assert gt.gt_spd_validate_count(ws) == planted
+
+
+def test_a_workspace_whose_header_was_not_zeroed_is_reported_not_trusted():
+    """The first 256 bytes of a workspace must be zero when it is first handed over; a dirty header shows up as
+    an error from gt_check (which clears it), never as a silently accepted status."""
+    from gpu_util import device_batch, device_csr
+    from paper_2609_34420_b200 import binding as gt
+    w = wl.small_workload([40], 1, 32, 5, seed=0)
+    bt = device_batch(w.batch)
+    rp, ci = device_csr(w.batch)
+    out = torch.zeros(w.batch.spd_bytes, dtype=torch.uint8, device="cuda")
+    ws = torch.full((max(gt.gt_spd_build_workspace(bt, int(ci.numel()), 5), 256),), 0xFF, dtype=torch.uint8, device="cuda")
+    with pytest.raises(gt.GtError):
+        gt.gt_check(ws)
+    gt.gt_check(ws)                                 # the report cleared the status word
+    ws[:256].zero_()
+    gt.gt_spd_build(rp, ci, bt, 5, out, ws)
+    gt.gt_check(ws)
+    np.testing.assert_array_equal(out.cpu().numpy(), ospd.spd_packed(w.batch.row_ptr, w.batch.col_idx, w.batch.cu_seqlens, 5))
 
 
 def test_invalid_arguments_are_rejected_without_launch():

@@ -1,12 +1,13 @@
 """gt_spd_build_static: the SPD build for callers that are not allowed to allocate device memory
 (its scratch is an array built into the library).  Collected last on purpose.
 
-The result must be bit-identical to gt_spd_build's on the same inputs, also on the second of two
-calls in a row (the built-in array still holds the first call's leftovers then)."""
+The result must be bit-identical to gt_spd_build's on the same inputs and to the BFS oracle's, also on
+the second of two calls in a row (the built-in array still holds the first call's leftovers then)."""
 import numpy as np
 import pytest
 import torch
 
+from oracle import spd as ospd
 from paper_2609_34420_b200 import binding as gt
 from paper_2609_34420_b200 import workloads as wl
 
@@ -30,11 +31,13 @@ def test_static_scratch_build_matches_workspace_build_twice_in_a_row(make):
     rp, ci = device_csr(w.batch)
     assert gt.gt_spd_build_workspace(bt, int(ci.numel()), w.max_dist) <= gt.gt_spd_build_static_limit()
     ref = reference_build(w, bt, rp, ci)
+    exp = ospd.spd_packed(w.batch.row_ptr, w.batch.col_idx, w.batch.cu_seqlens, w.max_dist)
     for _ in range(2):
         out = torch.full_like(ref, 0x55)
         gt.gt_spd_build_static(rp, ci, bt, w.max_dist, out)
         torch.cuda.synchronize()
         assert torch.equal(out, ref)
+        assert np.array_equal(out.cpu().numpy(), exp)
 
 
 def test_batches_beyond_the_built_in_array_are_refused():
