@@ -54,7 +54,7 @@ constexpr int kHalf = 64;                   // queries per TMEM stage
 constexpr int kStages = 2;
 constexpr int kBwdThreads = 768;
 constexpr int kSoftmaxThreads = 512;
-constexpr int kMaxPrivateBinBuckets = 27;   // 2 KB of shared memory per bucket
+constexpr int kMaxPrivateBinBuckets = 26;   // 2 KB of shared memory per bucket, between the 128 KB mark and the last two buffers
 constexpr int kExtCols = 16;                // bf16 per (query, head) row of folded terms
 constexpr int kExtTileBytes = kTile * kExtCols * 2;
 
@@ -100,6 +100,14 @@ enum BwdBarrier {
 };
 enum BwdNamedBarrier { kNbFlush = 1, kNbDqStaged = 4, kNbDqStagingFree = 5 };
 
+// Shared-memory map.  The bias-gradient bins start at the ABSOLUTE shared address 128 KB: a thread's bin column
+// then lies at 128K + 4 * (softmax thread index) < 128K + 2048, an address whose bits 11..15 are zero, so the
+// address of its bin b is  column | (b << 11)  -- one logic instruction on the shifted bucket byte instead of a
+// mask and an add.  The window of a thread block starts at address 1024 (the first KB is reserved), which the
+// kernel checks; everything that must sit below the bins fills [1 KB, 128 KB), the rest follows the bins.
+constexpr uint32_t kBinsAbsAddr = 128u * 1024u;
+constexpr uint32_t kSmemWindowBase = 1024u;
+
 template <int D>
 struct BwdSmem {
     static constexpr int kRowBytes = D * 2;
@@ -113,13 +121,16 @@ struct BwdSmem {
     static constexpr int kDo = kQ + kTileBytes;                     // [kStages] at stride kStageBytes
     static constexpr int kExt = kQ + kStages * kStageBytes;         // [kStages] per-query rows
     static constexpr int kSpd = kExt + kStages * kExtTileBytes;     // one tile: refilled while the threads work from registers
-    static constexpr int kStg = kSpd + kSpdBytes;                   // dQ staging: 128 rows x 32 floats
-    static constexpr int kDs = kStg + 16384;                        // 2 atoms x 128 rows x 128 B
-    static constexpr int kBias = kDs + 32768;
+    static constexpr int kBias = kSpd + kSpdBytes;
     static constexpr int kBars = kBias + 256 * 4;
     static constexpr int kMisc = kBars + kNumBwdBarriers * 8;
-    static constexpr int kBins = (kMisc + 16 + 127) & ~127;         // [n_bins][512] float (private) or [nb][32]
-    static size_t dynamic_bytes(int bin_floats) { return (size_t)kBins + (size_t)bin_floats * 4 + 1024; }
+    static constexpr int kLowEnd = kMisc + 16;
+    static constexpr int kBins = (int)(kBinsAbsAddr - kSmemWindowBase);    // [n_bins][512] float (private) or [nb][32]
+    static_assert(kLowEnd <= kBins, "the buffers below the bins must end before 128 KB");
+    // behind the bins (their size is a multiple of 1024 bytes): dQ staging (128 rows x 32 floats), then dS^T
+    // (2 atoms x 128 rows x 128 B)
+    static size_t stg_off(int bin_floats) { return (size_t)kBins + (((size_t)bin_floats * 4 + 1023) & ~(size_t)1023); }
+    static size_t dynamic_bytes(int bin_floats) { return stg_off(bin_floats) + 16384 + 32768; }
 };
 
 // register budget: the CTA is launched with 768 x 80 registers; after the re-split it holds
@@ -137,9 +148,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 {
     using L = BwdSmem<D>;
     extern __shared__ uint8_t smem_raw[];
-    // 1024-byte alignment by pointer arithmetic on the __shared__ array itself, so that every derived
-    // pointer keeps its shared address space (integer round trips would turn the accesses generic)
-    uint8_t* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    // pointers are derived from the __shared__ array itself, so that they keep the shared address space
+    uint8_t* smem = smem_raw;
+    if (smem_u32(smem_raw) != kSmemWindowBase) {      // the address arithmetic of the bins assumes this window base
+        if (threadIdx.x == 0 && atomicCAS(p.status, 0u, (uint32_t)GT_ERR_CUDA) == 0u) p.status[1] = 199;
+        return;
+    }
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -164,6 +178,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     auto bar = [&](int i) { return smem_u32(&bars[i]); };
     volatile uint32_t* abort_flag = &misc[1];
     const int n_bin_floats = kPrivateBins ? p.n_buckets * kSoftmaxThreads : p.n_buckets * 32;
+    uint8_t* const s_stg = smem + L::kBins + (((size_t)n_bin_floats * 4 + 1023) & ~(size_t)1023);
+    uint8_t* const s_ds = s_stg + 16384;
 
     if (tid == 0) {
         misc[1] = 0u;
@@ -322,7 +338,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             constexpr uint32_t idesc_dq = make_idesc_bf16(128, D, true, true);         // A and B MN-major
             const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
             const uint64_t desc_k = make_smem_desc(smem_u32(smem + L::kK), L::kRowBytes, 0);
-            const uint64_t da = make_smem_desc(smem_u32(smem + L::kDs), 128, 16384);
+            const uint64_t da = make_smem_desc(smem_u32(s_ds), 128, 16384);
             mbar_wait(bar(kBarKvFull), 0, abort_flag, p.status, 120);
             for (int i = 0; i < n_q; ++i) {
                 // dQ_i = dS K once both halves have stored dS^T(i) and the reducer has drained dQ_{i-1}
@@ -357,7 +373,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         // the thread's 32 bucket bytes: row r of the SPD^T tile, 16-byte chunks 2 grp and 2 grp + 1 (swizzled by r & 7)
         const uint32_t spd_off0 = r * 128 + (((2 * grp) ^ (r & 7)) << 4), spd_off1 = r * 128 + (((2 * grp + 1) ^ (r & 7)) << 4);
         const uint32_t bins_base = smem_u32(my_bins);
-        uint8_t* ds_row = smem + L::kDs + half * 16384 + r * 128;
+        uint8_t* ds_row = s_ds + half * 16384 + r * 128;
 
         // K (warps 4-7) and V (warps 8-11) rows -> tensor memory, where they stay as the A operands of
         // S^T = K Q^T and dP^T = V dO^T: one shared-memory read instead of one per query half tile
@@ -446,11 +462,13 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                     const int c = rnd * 16 + k;
                     unpack_f32x2(mul_f32x2(pack_f32x2(pr[c], pr[c + 1]), pack_u32x2(dp[k], dp[k + 1])), pr[c], pr[c + 1]);
                 }
-                // byte offset of bin b: b * stride * 4, formed by one funnel shift and one mask
+                // byte offset of bin b: b * stride * 4, formed by one funnel shift and one logic operation; with
+                // private bins that operation also ORs in the address of the thread's bin column (see the memory map)
                 constexpr int kLog = kPrivateBins ? 11 : 7;               // log2(kBinStride * 4)
                 auto bin_off = [&](int c) {
                     const int sh = 8 * (c & 3) - kLog;
-                    return (sh >= 0 ? (bw[c >> 2] >> (sh >= 0 ? sh : 0)) : (bw[c >> 2] << (sh < 0 ? -sh : 0))) & (0xffu << kLog);
+                    const uint32_t x = sh >= 0 ? (bw[c >> 2] >> (sh >= 0 ? sh : 0)) : (bw[c >> 2] << (sh < 0 ? -sh : 0));
+                    return kPrivateBins ? ((x & (0xffu << kLog)) | bins_base) : (x & (0xffu << kLog));
                 };
                 if (kPrivateBins) {
                     // read-modify-write of the thread's own bins, two elements at a time so that two loads are
@@ -460,12 +478,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                         const int c = rnd * 16 + k;
                         const uint32_t o0 = bin_off(c), o1 = bin_off(c + 1);
                         float v0, v1;
-                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v0) : "r"(bins_base + o0));
-                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v1) : "r"(bins_base + o1));
+                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v0) : "r"(o0));
+                        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v1) : "r"(o1));
                         v0 += pr[c];
                         v1 = (o1 == o0 ? v0 : v1) + pr[c + 1];
-                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(bins_base + o0), "f"(v0));
-                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(bins_base + o1), "f"(v1));
+                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(o0), "f"(v0));
+                        asm volatile("st.shared.f32 [%0], %1;" ::"r"(o1), "f"(v1));
                     }
                 } else {
 #pragma unroll
@@ -562,7 +580,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
-                uint8_t* stg = smem + ((kStgBufs == 2 && c == 1) ? L::kV : L::kStg);
+                uint8_t* stg = (kStgBufs == 2 && c == 1) ? smem + L::kV : s_stg;
                 uint32_t o[32];
                 tmem_ld32(tmem + kColDq + c * 32 + lane_off, o);
                 tmem_wait_ld();
