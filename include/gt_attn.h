@@ -328,6 +328,33 @@ gt_status gt_biased_attn_fwd_chunked(const void* q, const void* k, const void* v
                                      int32_t n_kv_chunks, float* lse_chunks,
                                      void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------------------
+ * gt_feature_attn_fwd / gt_feature_attn_bwd -- Eq. 1 with a FEATURE bias in place of the distance-bucket
+ * table.  The end-to-end model of the paper has an "attention bias dimension of 4" (Sec. "Experiments",
+ * end-to-end configuration): every ordered node pair carries four bias features and each head weights
+ * them.  The paper states the dimension only; the linear form is the reading taken here:
+ *     S_ij = (q_i . k_j)/sqrt(head_dim) + sum_c weights[h][c] * features[i][j][c]     (c = 0..3)
+ * features: uint8 [N, N, 4] (row i = query, column j = key, the four features of a pair in one 32-bit
+ * word, base pointer 4-byte aligned); weights: fp32 [n_heads, 4].  Forward results as for
+ * gt_biased_attn_fwd (out bf16 [N,H,d], lse fp32 [H,N]); the backward overwrites dq, dk, dv (bf16) and
+ *     dweights[h][c] = sum_ij dS_ij * features[i][j][c]           (fp32 [n_heads, 4]),
+ * a contraction instead of the bucket form's scatter.  The backward takes the forward's lse but not its output:
+ * the per-query term dout_i . out_i is recomputed in fp32 as sum_j P_ij (dout_i . v_j), because the features have
+ * a large common part and a term taken from the rounded bf16 output would leak it into dweights.  Single graph only (n_graphs == 1, else
+ * GT_ERR_UNSUPPORTED); head_dim in {32, 64}.  This variant is a correctness-first fp32 path on the CUDA
+ * cores (no tensor cores): it is meant for the model sizes the paper trains (1 024 - 8 192 nodes per
+ * batch), not for the 65 536-node benchmark.  The forward needs no workspace and has no device status.
+ * ------------------------------------------------------------------------------------- */
+gt_status gt_feature_attn_fwd(const void* q, const void* k, const void* v, const uint8_t* features, const float* weights,
+                              const gt_batch* batch, int32_t n_heads, int32_t head_dim,
+                              void* out, float* lse, void* stream);
+size_t gt_feature_attn_bwd_workspace(const gt_batch* batch, int32_t n_heads);
+gt_status gt_feature_attn_bwd(const void* q, const void* k, const void* v, const void* dout, const float* lse,
+                              const uint8_t* features, const float* weights,
+                              const gt_batch* batch, int32_t n_heads, int32_t head_dim,
+                              void* dq, void* dk, void* dv, float* dweights,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

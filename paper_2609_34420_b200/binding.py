@@ -30,7 +30,8 @@ EXPORTS = ("gt_status_string", "gt_check",
            "gt_biased_attn_bwd_chunked_workspace", "gt_biased_attn_bwd_chunked",
            "gt_biased_attn_fwd_step_workspace", "gt_biased_attn_fwd_step",
            "gt_biased_attn_bwd_step_context_bytes", "gt_biased_attn_bwd_step_prepare", "gt_biased_attn_bwd_step_prepare_ex",
-           "gt_biased_attn_bwd_step", "gt_biased_attn_bwd_step_finish")
+           "gt_biased_attn_bwd_step", "gt_biased_attn_bwd_step_finish",
+           "gt_feature_attn_fwd", "gt_feature_attn_bwd_workspace", "gt_feature_attn_bwd")
 
 
 class GtError(RuntimeError):
@@ -111,6 +112,12 @@ def lib() -> ctypes.CDLL:
         L.gt_biased_attn_bwd_chunked_workspace.argtypes = [bp, i32, i32, i32, i32]
         L.gt_biased_attn_bwd_chunked.restype = ctypes.c_int
         L.gt_biased_attn_bwd_chunked.argtypes = [vp] * 8 + [bp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.gt_feature_attn_fwd.restype = ctypes.c_int
+        L.gt_feature_attn_fwd.argtypes = [vp] * 5 + [bp, i32, i32, vp, vp, vp]
+        L.gt_feature_attn_bwd_workspace.restype = sz
+        L.gt_feature_attn_bwd_workspace.argtypes = [bp, i32]
+        L.gt_feature_attn_bwd.restype = ctypes.c_int
+        L.gt_feature_attn_bwd.argtypes = [vp] * 7 + [bp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
         _lib = L
     return _lib
 
@@ -385,3 +392,30 @@ def gt_biased_attn_bwd_step_finish(dq_acc, dk_acc, dv_acc, dbias_acc, batch: Bat
     st = lib().gt_biased_attn_bwd_step_finish(_ptr(dq_acc), _ptr(dk_acc), _ptr(dv_acc), _ptr(dbias_acc), ctypes.byref(b), H, d,
                                               int(max_dist), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dbias), _stream())
     _raise(st, "gt_biased_attn_bwd_step_finish")
+
+
+def gt_feature_attn_fwd(q, k, v, features, weights, batch: Batch, out, lse) -> None:
+    """Forward with the feature bias: features uint8 [N, N, 4], weights fp32 [H, 4]."""
+    _, H, d = q.shape
+    b = batch.c_struct()
+    st = lib().gt_feature_attn_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(features), _ptr(weights), ctypes.byref(b), H, d,
+                                   _ptr(out), _ptr(lse), _stream())
+    _raise(st, "gt_feature_attn_fwd")
+
+
+def gt_feature_attn_bwd_workspace(batch: Batch, n_heads: int) -> int:
+    b = batch.c_struct()
+    return int(lib().gt_feature_attn_bwd_workspace(ctypes.byref(b), n_heads))
+
+
+def gt_feature_attn_bwd(q, k, v, dout, lse, features, weights, batch: Batch, dq, dk, dv, dweights,
+                        workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    _, H, d = q.shape
+    if workspace is None:
+        workspace = _workspace(gt_feature_attn_bwd_workspace(batch, H), q.device)
+    b = batch.c_struct()
+    st = lib().gt_feature_attn_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(dout), _ptr(lse), _ptr(features), _ptr(weights),
+                                   ctypes.byref(b), H, d, _ptr(dq), _ptr(dk), _ptr(dv), _ptr(dweights),
+                                   _ptr(workspace), workspace.numel(), _stream())
+    _raise(st, "gt_feature_attn_bwd")
+    return workspace
