@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the biased graph-attention hot path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference] [--mode step|ring]
 
 One step = one pass of the whole hot path over one seeded synthetic batch:
 gt_spd_build -> gt_biased_attn_fwd -> gt_biased_attn_bwd -> gt_biased_attn_fwd_chunked.
@@ -9,6 +9,11 @@ The headline metric is forward+backward attention TFLOP/s (14*H*d*sum n_g^2 FLOP
 divided by the forward+backward time inside the step, CUDA events); the SPD build GB/s, the
 chunked forward and the whole-step time are reported beside it.  With N > 1 (torchrun) every
 rank processes its own batch: weak scaling over independent batches, no data-path collective.
+
+`--mode ring` (under torchrun with N > 1, or alone) measures graph-aware context parallelism instead: ONE
+graph, query rows and bias rows sharded over the ranks, K/V blocks (and in the backward their dK/dV sums)
+passed round the ring with torch.distributed P2P while every rank runs the caller-driven step kernels on
+the block it holds; strong scaling, whole-job FLOPs over the max-over-ranks time.
 
 `--impl reference` times the CPU oracle (fp64, host cores) on a bounded row sample of the
 same workload and prints the same JSON line with "impl": "reference".
@@ -484,6 +489,140 @@ def run_cuda(args) -> int:
     return 0
 
 
+# --------------------------------------------------------------------------------------
+# Context-parallel ring (one graph over all ranks): forward ring + backward ring per step
+# --------------------------------------------------------------------------------------
+def run_ring(args) -> int:
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_34420_b200 import binding as gt
+    from paper_2609_34420_b200 import dist_util, ring
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
+    rank, local_rank, world = dist_util.env_world()
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    dist_util.init_process_group("nccl")
+    gt.lib()
+    w = wl.make_workload(args.workload)                     # the SAME graph on every rank: it is one sharded problem
+    b, t = w.batch, w.tensors()
+    if b.n_graphs != 1:
+        raise SystemExit("--mode ring needs a single-graph workload")
+    T, H, d, D = b.n_total, w.n_heads, w.head_dim, w.max_dist
+    n_super = args.super_nodes if args.super_nodes >= 0 else (1024 if T >= 8192 else 16 * (T // 160))
+    layout = ring.RingLayout.even(T, n_super, world)
+    (a, e), (sa, sb) = layout.shards[rank], layout.super_range
+    share = max(y - x for x, y in layout.shards)
+
+    def dev_bf16(bits):
+        return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    batch = gt.Batch(T)
+    rp, ci = torch.from_numpy(b.row_ptr).to(dev), torch.from_numpy(b.col_idx).to(dev)
+    spd = torch.empty(b.spd_bytes, dtype=torch.uint8, device=dev)
+    gt.gt_check(gt.gt_spd_build(rp, ci, batch, D, spd))       # a rank reads only the rows of its queries (its bias shard)
+    q, k, v, do = dev_bf16(t.q), dev_bf16(t.k), dev_bf16(t.v), dev_bf16(t.dout)
+    bias = torch.from_numpy(t.bias).to(dev)
+    # what the rank owns: its regular K/V rows and a replica of the super nodes' rows; everything else arrives
+    k_full, v_full = torch.zeros_like(k), torch.zeros_like(v)
+    k_full[sa:sb], v_full[sa:sb] = k[sa:sb], v[sa:sb]
+
+    def block(x, with_super):
+        blk = torch.zeros((share + (n_super if with_super else 0), H, d), dtype=x.dtype, device=dev)
+        blk[: e - a] = x[a:e]
+        if with_super:
+            blk[share:] = x[sa:sb]
+        return blk
+
+    fwd_blocks, bwd_blocks = (block(k, True), block(v, True)), (block(k, False), block(v, False))
+    o_acc = torch.zeros(T, H, d, dtype=torch.float32, device=dev)
+    lse_acc = torch.empty(H, T, dtype=torch.float32, device=dev)
+    out = torch.zeros_like(q)
+    accs = [torch.zeros(T, H, d, dtype=torch.float32, device=dev) for _ in range(3)]
+    db_acc = torch.zeros(H, D + 2, dtype=torch.float64, device=dev)
+    ctx = gt._workspace(gt.gt_biased_attn_bwd_step_context_bytes(batch, H, d), dev)
+    ws_step = gt._workspace(gt.gt_biased_attn_fwd_step_workspace(batch, H, d), dev)
+    dq, dk, dv = (torch.zeros_like(q) for _ in range(3))
+    dbias = torch.zeros_like(bias)
+    fwd_step = ring.device_step(gt, q, k_full, v_full, spd, bias, batch, D, layout, o_acc, lse_acc, out, ws_step)
+    bwd_step = ring.device_bwd_step(gt, q, k_full, v_full, do, bias, batch, D, layout, accs[0], accs[1], accs[2], db_acc, ctx)
+    # replicated on every rank until the all-reduce: the super rows of dq, the super keys' dk / dv, dbias
+    replicated = [accs[0][sa:sb], accs[1][sa:sb], accs[2][sa:sb], db_acc] if n_super else [db_acc]
+
+    def one_pass():
+        o_acc.zero_()
+        lse_acc.fill_(float("-inf"))
+        for x in accs:
+            x.zero_()
+        db_acc.zero_()
+        dk_own, dv_own = ring.context_parallel_pass(
+            layout, fwd_blocks, fwd_step, bwd_blocks, bwd_step, replicated=replicated,
+            between=lambda: gt.gt_biased_attn_bwd_step_prepare(None, do, lse_acc, spd, batch, D, ctx, out_f32=o_acc),
+            rank=rank, world=world)
+        accs[1][a:e].copy_(dk_own[: e - a])                  # the sums of the rank's own keys are home again
+        accs[2][a:e].copy_(dv_own[: e - a])
+        gt.gt_biased_attn_bwd_step_finish(accs[0], accs[1], accs[2], db_acc, batch, D, dq, dk, dv, dbias)
+
+    for _ in range(max(args.warmup, 1)):
+        one_pass()
+    torch.cuda.synchronize()
+    gt.gt_check(ctx)
+    gt.gt_check(ws_step)
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid)) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dist_util.barrier(dev)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(args.steps):
+        one_pass()
+    e1.record()
+    torch.cuda.synchronize()
+    dist_util.barrier(dev)
+    clocks = sampler.stop() if sampler else None
+    gt.gt_check(ctx)
+    gt.gt_check(ws_step)
+    f_fwd, f_bwd = w.attn_flops()
+    ms, _ = dist_util.aggregate(e0.elapsed_time(e1) / args.steps, 0.0, dev)
+    value = (f_fwd + f_bwd) / (ms * 1e-3) / 1e12
+
+    # the rank's rows against the one-shot calls on the whole graph (every rank holds the full inputs here)
+    out_ref, dq_ref, dk_ref, dv_ref = (torch.empty_like(q) for _ in range(4))
+    lse_ref = torch.empty(H, T, dtype=torch.float32, device=dev)
+    dbias_ref = torch.empty_like(bias)
+    gt.gt_check(gt.gt_biased_attn_fwd(q, k, v, spd, bias, batch, D, out_ref, lse_ref))
+    gt.gt_check(gt.gt_biased_attn_bwd(q, k, v, out_ref, do, lse_ref, spd, bias, batch, D, dq_ref, dk_ref, dv_ref, dbias_ref))
+    rows = torch.cat([torch.arange(a, e, device=dev), torch.arange(sa, sb, device=dev)])
+    rel = lambda x, y: float(((x.float() - y.float()).norm() / y.float().norm()).item())
+    check = {"out": rel(out[rows], out_ref[rows]), "dq": rel(dq[rows], dq_ref[rows]), "dk": rel(dk[rows], dk_ref[rows]),
+             "dv": rel(dv[rows], dv_ref[rows]), "dbias": rel(dbias, dbias_ref)}
+    worst = torch.tensor([max(check.values())], dtype=torch.float64, device=dev)
+    if dist.is_initialized():
+        dist.all_reduce(worst, op=dist.ReduceOp.MAX)
+    if rank != 0:
+        return 0
+    peaks, peak_kind = load_peaks()
+    blk_bytes = 2 * (share + n_super) * H * d * 2                       # K and V block, bf16
+    bwd_bytes = 2 * share * H * d * 2 + 2 * share * H * d * 4           # K, V (bf16) and their dK, dV sums (fp32)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 1),
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "mode": "ring",
+        "config": {"workload": args.workload, "note": w.note, "n_total": T, "n_heads": H, "head_dim": d, "max_dist": D,
+                   "super_nodes": n_super, "parallelism": f"cp{world} (query rows and bias rows sharded, K/V blocks round the ring)",
+                   "step": "forward ring + backward ring + all-reduce of the replicated sums + final conversion",
+                   "l2": "inputs larger than L2 at the default workload: every rank streams its %.2f GB bias shard per pass" % (b.spd_bytes / world / 1e9)},
+        "p2p_bytes_per_rank_per_step": {"forward": (world - 1) * blk_bytes, "backward": (world - 1) * bwd_bytes + (2 * share * H * d * 4 if world > 1 else 0)},
+        "pct_of_bf16_peak": {"sustained": 100 * value / world / float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
+                             "burst": 100 * value / world / float(peaks["bf16_tflops"])},
+        "max_rel_l2_vs_one_shot": float(worst.item()), "rel_l2_vs_one_shot_rank0": check,
+        "gpu_launches": None, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    return 0
+
+
 def main() -> int:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -491,9 +630,13 @@ def main() -> int:
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(wl.WORKLOAD_NAMES) + ["tiny_er256_sparse"])
+    ap.add_argument("--mode", default="step", choices=["step", "ring"])
+    ap.add_argument("--super-nodes", type=int, default=-1, help="ring mode: replicated super nodes (default 1024 from 8192 nodes up)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.mode == "ring":
+        return run_ring(args)
     return run_cuda(args)
 
 

@@ -234,7 +234,7 @@ gt_status gt_biased_attn_bwd_ex(const void* q, const void* k, const void* v, con
  * combination.  After the last step o_acc is the attention output and lse_acc its LSE.
  * q, k, v, spd: the tensors of the whole single graph (n_graphs == 1), as for gt_biased_attn_fwd.
  * out: optional bf16 [N, H, d]; its rows [q_begin, q_end) receive bf16(o_acc) after the step.
- * A key range must start at a multiple of 16 (else GT_ERR_UNSUPPORTED); ranges of one row's steps
+ * A non-empty key range must start at a multiple of 16 (else GT_ERR_UNSUPPORTED); ranges of one row's steps
  * must not overlap (a key seen twice is counted twice).
  * ------------------------------------------------------------------------------------- */
 size_t gt_biased_attn_fwd_step_workspace(const gt_batch* batch, int32_t n_heads, int32_t head_dim);

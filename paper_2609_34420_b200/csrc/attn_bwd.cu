@@ -709,8 +709,14 @@ __global__ void bwd_preprocess_kernel(const __nv_bfloat16* __restrict__ out, con
         }
     }
     uint4 e0 = make_uint4(0u, 0u, 0u, 0u), e1 = make_uint4(0u, 0u, 0u, 0u);
-    split3_bf16(-lse[(size_t)h * n_total + t] * sqrt_d, e0.x, e0.y);
-    split3_bf16(-acc, e1.x, e1.y);
+    // A row whose forward state is not final on this rank (a ring step's context holds lse = -inf for the rows
+    // of other ranks) gets zero terms: the row may share a 128-row tile with rows that are used, where its columns
+    // are masked by assignment after the exponential, and a non-finite term would turn 0 * (dP - Delta) into NaN.
+    const float l = lse[(size_t)h * n_total + t];
+    if (isfinite(l) && isfinite(acc)) {
+        split3_bf16(-l * sqrt_d, e0.x, e0.y);
+        split3_bf16(-acc, e1.x, e1.y);
+    }
     ext[2 * idx] = e0;
     ext[2 * idx + 1] = e1;
 }

@@ -877,7 +877,7 @@ extern "C" gt_status gt_biased_attn_fwd_step(const void* q, const void* k, const
     if (q_begin < 0 || q_end > n || q_begin >= q_end) return GT_ERR_INVALID_ARG;
     if (kv_begin0 < 0 || kv_end0 > n || kv_begin0 > kv_end0 || kv_begin1 < 0 || kv_end1 > n || kv_begin1 > kv_end1) return GT_ERR_INVALID_ARG;
     // a key range starts at a multiple of 16: the SPD tile of a range is fetched by TMA from that column
-    if ((kv_begin0 & 15) || (kv_begin1 & 15)) return GT_ERR_UNSUPPORTED;
+    if ((kv_end0 > kv_begin0 && (kv_begin0 & 15)) || (kv_end1 > kv_begin1 && (kv_begin1 & 15))) return GT_ERR_UNSUPPORTED;
     const size_t need = gt_biased_attn_fwd_step_workspace(batch, n_heads, head_dim);
     if (workspace == nullptr || workspace_bytes < need || misaligned16(workspace)) return GT_ERR_WORKSPACE;
     if (sm_count() <= 0) return GT_ERR_NO_DEVICE;

@@ -127,8 +127,10 @@ def ring_backward(layout: RingLayout, k_own: torch.Tensor, v_own: torch.Tensor, 
     if rank is None:
         rank = dist.get_rank(group) if dist.is_initialized() else 0
     assert len(layout.shards) == world
-    cur = [k_own, v_own, torch.zeros_like(k_own), torch.zeros_like(v_own)]
-    bufs = [[torch.empty_like(k_own) for _ in range(4)] for _ in range(2)] if world > 1 else []
+    # the sums travel in fp32 when K/V are 16-bit tensors (they are unscaled partial sums over many query rows)
+    sum_dtype = torch.float32 if k_own.dtype in (torch.bfloat16, torch.float16) else k_own.dtype
+    cur = [k_own, v_own, torch.zeros_like(k_own, dtype=sum_dtype), torch.zeros_like(v_own, dtype=sum_dtype)]
+    bufs = [[torch.empty_like(cur[t]) for t in range(4)] for _ in range(2)] if world > 1 else []
     empty: Range = (0, 0)
     has_super = layout.super_range[1] > layout.super_range[0]
     for s in range(world):
@@ -145,3 +147,51 @@ def ring_backward(layout: RingLayout, k_own: torch.Tensor, v_own: torch.Tensor, 
                 r.wait()
             cur = [nxt[t] if t in which else cur[t] for t in range(4)]
     return cur[2], cur[3]
+
+
+def device_bwd_step(binding, q, k_full, v_full, dout, bias, batch, max_dist: int, layout: RingLayout,
+                    dq_acc, dk_acc, dv_acc, dbias_acc, context) -> BwdStepFn:
+    """Backward step function backed by `gt_biased_attn_bwd_step` (counterpart of `device_step`).
+
+    The C ABI addresses keys by global row: an arriving block's K/V rows are copied to their rows of the
+    full-length `k_full` / `v_full`, and the sums that travel with the block (`dk_blk`, `dv_blk`, unscaled
+    fp32) are copied to the same rows of the full-length accumulators `dk_acc` / `dv_acc` before the call and
+    back into the travelling buffers after it, all on the current stream.  The super nodes' K/V are the
+    rank's own replica (already in `k_full` / `v_full`); their dK/dV rows of the accumulators, the super
+    rows of `dq_acc` and `dbias_acc` are this rank's partial sums, which the caller all-reduces at the end.
+    `context` comes from `gt_biased_attn_bwd_step_prepare`."""
+
+    def step(q_range: Range, kv_range: Range, sup: Range, k_blk, v_blk, dk_blk, dv_blk, owner: int) -> None:
+        a, b = kv_range
+        if b > a:
+            k_full[a:b].copy_(k_blk[: b - a], non_blocking=True)
+            v_full[a:b].copy_(v_blk[: b - a], non_blocking=True)
+            dk_acc[a:b].copy_(dk_blk[: b - a], non_blocking=True)
+            dv_acc[a:b].copy_(dv_blk[: b - a], non_blocking=True)
+        binding.gt_biased_attn_bwd_step(q, k_full, v_full, dout, bias, batch, max_dist, q_range, kv_range, sup,
+                                        dq_acc, dk_acc, dv_acc, dbias_acc, context)
+        if b > a:
+            dk_blk[: b - a].copy_(dk_acc[a:b], non_blocking=True)
+            dv_blk[: b - a].copy_(dv_acc[a:b], non_blocking=True)
+
+    return step
+
+
+def context_parallel_pass(layout: RingLayout, fwd_blocks: Tuple[torch.Tensor, torch.Tensor], fwd_step: StepFn,
+                          bwd_blocks: Tuple[torch.Tensor, torch.Tensor], bwd_step: BwdStepFn,
+                          replicated: Sequence[torch.Tensor] = (), between: Optional[Callable[[], None]] = None,
+                          group: Optional[dist.ProcessGroup] = None, rank: Optional[int] = None,
+                          world: Optional[int] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """One forward + backward of graph-aware context parallelism on this rank: the forward ring (K/V blocks
+    with the super nodes attached), `between()` (e.g. the backward's prepare call, once the forward state is
+    final), the backward ring (regular K/V rows travelling with their dK/dV sums), then the all-reduce of
+    what is replicated on every rank (`replicated`: the super rows of dq, the super keys' dk / dv, dbias --
+    per-rank partial sums until here).  Returns the rank's own (dk, dv) sums as `ring_backward` does."""
+    ring_forward(layout, fwd_blocks[0], fwd_blocks[1], fwd_step, group, rank, world)
+    if between is not None:
+        between()
+    dk_own, dv_own = ring_backward(layout, bwd_blocks[0], bwd_blocks[1], bwd_step, group, rank, world)
+    if dist.is_initialized() and (world is None or world > 1):
+        for t in replicated:
+            dist.all_reduce(t, group=group)
+    return dk_own, dv_own

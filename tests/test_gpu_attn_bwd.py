@@ -265,3 +265,92 @@ def test_backward_ring_steps_reproduce_the_backward_and_the_block_oracle(n, n_su
     s_ = 1.0 / np.sqrt(float(d))
     for name, got, ref in (("dq", acc[0], o_dq), ("dk", acc[1], o_dk), ("dv", acc[2], o_dv), ("db", db_acc, o_db)):
         assert rel_l2(got.cpu().numpy().astype(np.float64), ref) <= GRAD_REL_L2, name
+
+
+def test_context_parallel_pass_with_the_device_steps_on_one_rank():
+    """World size 1: the forward and backward rings degenerate to the rank's own block, which exercises both
+    device step wrappers (block -> global rows copies, two-part key slices, travelling dK/dV sums, the fp32
+    carried output feeding the backward's per-query term) end to end against the one-shot calls; the
+    multi-rank schedule itself is tested on CPU ranks."""
+    from paper_2609_34420_b200 import binding as gt, ring
+    n, n_super, H, d = 900, 52, 2, 64
+    w = wl.small_workload([n], H, d, 6, seed=21, avg_degree=2.0, directed=True)
+    case = DeviceCase(w)
+    out_ref, lse_ref = case.forward()
+    ref = case.backward(out_ref, lse_ref)
+    dev = case.q.device
+    layout = ring.RingLayout.even(n, n_super, 1)
+    (a, b), (sa, sb) = layout.shards[0], layout.super_range
+    k_full, v_full = torch.zeros_like(case.k), torch.zeros_like(case.v)
+    o_acc = torch.zeros(n, H, d, dtype=torch.float32, device=dev)
+    lse_acc = torch.full((H, n), float("-inf"), dtype=torch.float32, device=dev)
+    out = torch.full_like(case.q, float("nan"))
+    fwd_blocks = (torch.cat([case.k[a:b], case.k[sa:sb]]), torch.cat([case.v[a:b], case.v[sa:sb]]))
+    fwd_step = ring.device_step(gt, case.q, k_full, v_full, case.spd, case.bias, case.batch, w.max_dist, layout, o_acc, lse_acc, out)
+    accs = [torch.zeros(n, H, d, dtype=torch.float32, device=dev) for _ in range(3)]
+    db_acc = torch.zeros(H, w.max_dist + 2, dtype=torch.float64, device=dev)
+    ctx = gt._workspace(gt.gt_biased_attn_bwd_step_context_bytes(case.batch, H, d), dev)
+    bwd_step = ring.device_bwd_step(gt, case.q, k_full, v_full, case.dout, case.bias, case.batch, w.max_dist, layout,
+                                    accs[0], accs[1], accs[2], db_acc, ctx)
+    prepare = lambda: gt.gt_biased_attn_bwd_step_prepare(None, case.dout, lse_acc, case.spd, case.batch, w.max_dist, ctx, out_f32=o_acc)
+    dk_own, dv_own = ring.context_parallel_pass(layout, fwd_blocks, fwd_step, (case.k[a:b].clone(), case.v[a:b].clone()), bwd_step,
+                                                between=prepare, rank=0, world=1)
+    gt.gt_check(ctx)
+    dq, dk, dv = (torch.full_like(case.q, float("nan")) for _ in range(3))
+    dbias = torch.full_like(case.bias, float("nan"))
+    gt.gt_biased_attn_bwd_step_finish(accs[0], accs[1], accs[2], db_acc, case.batch, w.max_dist, dq, dk, dv, dbias)
+    torch.cuda.synchronize()
+    assert rel_l2(to_f64(out), to_f64(out_ref)) <= CHUNK_REL_L2
+    assert torch.equal(dk_own, accs[1][a:b]) and torch.equal(dv_own, accs[2][a:b])      # the sums that came home
+    for name, got, want in zip(("dq", "dk", "dv"), (dq, dk, dv), ref):
+        assert rel_l2(to_f64(got), to_f64(want)) <= 2e-3, name       # Delta from the fp32 state here, from the bf16 out there
+    # against the oracle directly (exact output): the fp32 carried state keeps dBias within the bound
+    q64, k64, v64, do64, b64 = case.host_f64()
+    rdq, rdk, rdv, rdb = oattn.backward_single(q64, k64, v64, do64, np.asarray(case.spd_host).reshape(n, -1), b64)
+    for name, got, want in (("dq", dq, rdq), ("dk", dk, rdk), ("dv", dv, rdv), ("dbias", dbias, rdb)):
+        assert rel_l2(to_f64(got), want) <= GRAD_REL_L2, name
+
+
+@pytest.mark.parametrize("ranks,n_super", [(3, 40), (2, 0)])
+def test_ranks_that_only_hold_their_own_forward_state(ranks, n_super):
+    """What a real multi-rank pass looks like from one rank: its carried state (o_acc, lse_acc) is final for its
+    own query rows only (the other rows stay at lse = -inf), and the backward context is prepared from that.
+    The ranks are run one after the other on this GPU (their launches do not wait on one another); their sums
+    add up to the one-shot backward.  Shard boundaries fall inside 128-row tiles, so a tile mixes rows of two ranks."""
+    from paper_2609_34420_b200 import binding as gt, ring
+    n, H, d = 1000, 2, 64
+    w = wl.small_workload([n], H, d, 6, seed=33 + ranks, avg_degree=2.0, directed=True)
+    case = DeviceCase(w)
+    out_ref, lse_ref = case.forward()
+    ref = case.backward(out_ref, lse_ref)
+    dev = case.q.device
+    layout = ring.RingLayout.even(n, n_super, ranks)
+    sup = layout.super_range
+    accs = [torch.zeros(n, H, d, dtype=torch.float32, device=dev) for _ in range(3)]
+    db_acc = torch.zeros(H, w.max_dist + 2, dtype=torch.float64, device=dev)
+    for r in range(ranks):
+        o_acc = torch.zeros(n, H, d, dtype=torch.float32, device=dev)
+        lse_acc = torch.full((H, n), float("-inf"), dtype=torch.float32, device=dev)
+        q_ranges = [layout.shards[r]] + ([sup] if n_super else [])
+        for s_ in range(ranks):
+            owner = (r - s_) % ranks
+            for qr in q_ranges:
+                gt.gt_biased_attn_fwd_step(case.q, case.k, case.v, case.spd, case.bias, case.batch, w.max_dist, qr,
+                                           layout.shards[owner], sup if s_ == 0 else (0, 0), o_acc, lse_acc)
+        ctx = gt.gt_biased_attn_bwd_step_prepare(None, case.dout, lse_acc, case.spd, case.batch, w.max_dist, out_f32=o_acc)
+        for s_ in range(ranks):
+            owner = (r - s_) % ranks
+            gt.gt_biased_attn_bwd_step(case.q, case.k, case.v, case.dout, case.bias, case.batch, w.max_dist, layout.shards[r],
+                                       layout.shards[owner], sup if s_ == 0 else (0, 0), accs[0], accs[1], accs[2], db_acc, ctx)
+            if n_super and s_ == 0:      # the super nodes' query rows: at a block's home rank, their own keys on rank 0
+                gt.gt_biased_attn_bwd_step(case.q, case.k, case.v, case.dout, case.bias, case.batch, w.max_dist, sup,
+                                           layout.shards[owner], sup if r == 0 else (0, 0), accs[0], accs[1], accs[2], db_acc, ctx)
+        gt.gt_check(ctx)
+    dq, dk, dv = (torch.full_like(case.q, float("nan")) for _ in range(3))
+    dbias = torch.full_like(case.bias, float("nan"))
+    gt.gt_biased_attn_bwd_step_finish(accs[0], accs[1], accs[2], db_acc, case.batch, w.max_dist, dq, dk, dv, dbias)
+    torch.cuda.synchronize()
+    for name, got, want in zip(("dq", "dk", "dv", "dbias"), (dq, dk, dv, dbias), ref):
+        g = to_f64(got)
+        assert np.isfinite(g).all(), name
+        assert rel_l2(g, to_f64(want)) <= 5e-3, name

@@ -173,3 +173,104 @@ def test_three_rank_backward_ring_reproduces_the_backward():
         np.testing.assert_allclose(dk_sup * s_, rdk[sa:sb], rtol=1e-9, atol=1e-12)
         np.testing.assert_allclose(dv_sup, rdv[sa:sb], rtol=1e-9, atol=1e-12)
         np.testing.assert_allclose(db, rdb, rtol=1e-9, atol=1e-12)
+
+
+def _cp_worker(rank, world, port, out_q):
+    """Forward ring, then backward ring fed by the forward's carried state, then the all-reduce of the replicated
+    pieces: `ring.context_parallel_pass` end to end with oracle-backed step functions."""
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    import torch.distributed as dist
+    from oracle import attention as oattn
+    from paper_2609_34420_b200 import ring, workloads as wl
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    q, k, v, spd, bias = _case()
+    w = wl.small_workload([N], H, D_HEAD, MAX_DIST, seed=5, avg_degree=2.0, directed=True)
+    do = wl.bf16_bits_to_f64(w.tensors().dout)
+    layout = ring.RingLayout.even(N, N_SUPER, world)
+    a, b = layout.shards[rank]
+    share = max(e - s for s, e in layout.shards)
+    sa, sb = layout.super_range
+
+    def block(x, with_super):
+        blk = np.zeros((share + (N_SUPER if with_super else 0),) + x.shape[1:])
+        blk[: b - a] = x[a:b]
+        if with_super:
+            blk[share:] = x[sa:sb]
+        return torch.from_numpy(blk)
+
+    o = np.zeros((N, H, D_HEAD)); lse = np.full((H, N), -np.inf)
+
+    def fwd_step(q_range, kv_range, sup, k_blk, v_blk, owner):
+        ka, kb = kv_range
+        kk, vv = np.zeros_like(k), np.zeros_like(v)
+        kk[ka:kb] = k_blk.numpy()[: kb - ka]; vv[ka:kb] = v_blk.numpy()[: kb - ka]
+        kk[sa:sb] = k_blk.numpy()[share:]; vv[sa:sb] = v_blk.numpy()[share:]
+        rows = np.arange(*q_range); keys = np.concatenate([np.arange(ka, kb), np.arange(*sup)])
+        po, pl = oattn.attend_key_set(q, kk, vv, spd, bias, rows, keys)
+        o[rows], lse[:, rows] = oattn.merge_state(o[rows], lse[:, rows], po, pl)
+
+    dq = np.zeros_like(q); dk_sup = np.zeros((N_SUPER, H, D_HEAD)); dv_sup = np.zeros((N_SUPER, H, D_HEAD)); db = np.zeros_like(bias)
+
+    def bwd_step(q_range, kv_range, sup, k_blk, v_blk, dk_blk, dv_blk, owner):
+        ka, kb = kv_range
+        kk, vv = np.zeros_like(k), np.zeros_like(v)
+        kk[ka:kb] = k_blk.numpy()[: kb - ka]; vv[ka:kb] = v_blk.numpy()[: kb - ka]
+        kk[sa:sb] = k[sa:sb]; vv[sa:sb] = v[sa:sb]
+        rows = np.arange(*q_range); keys = np.concatenate([np.arange(ka, kb), np.arange(*sup)])
+        # the forward state of THIS rank (its rows only are final): what the backward of a rank may use
+        pq, pk, pv, pb = oattn.backward_block(q, kk, vv, do, o, lse, spd, bias, rows, keys)
+        dq[rows] += pq
+        dk_blk.numpy()[: kb - ka] += pk[: kb - ka]; dv_blk.numpy()[: kb - ka] += pv[: kb - ka]
+        if sup[1] > sup[0]:
+            dk_sup[:] += pk[kb - ka:]; dv_sup[:] += pv[kb - ka:]
+        db[:] += pb
+
+    red = [torch.from_numpy(x) for x in (dk_sup, dv_sup, db)]
+    dq_sup = torch.zeros(N_SUPER, H, D_HEAD, dtype=torch.float64)
+    done = []
+
+    def between():
+        done.append("forward state final")
+
+    dk_own, dv_own = ring.context_parallel_pass(layout, (block(k, True), block(v, True)), fwd_step,
+                                                (block(k, False), block(v, False)), bwd_step, replicated=red, between=between)
+    dq_sup += torch.from_numpy(dq[sa:sb]); dist.all_reduce(dq_sup)
+    out_q.put((rank, o[a:b], dq[a:b], dk_own.numpy()[: b - a], dv_own.numpy()[: b - a], dq_sup.numpy(), [t.numpy() for t in red], done))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_three_rank_forward_then_backward_pass_with_the_all_reduce_of_the_replicated_sums():
+    world = 3
+    ctx = mp.get_context("spawn")
+    out_q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_cp_worker, args=(r, world, port, out_q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted((out_q.get(timeout=180) for _ in range(world)), key=lambda r: r[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    from oracle import attention as oattn
+    from paper_2609_34420_b200 import ring, workloads as wl
+    q, k, v, spd, bias = _case()
+    w = wl.small_workload([N], H, D_HEAD, MAX_DIST, seed=5, avg_degree=2.0, directed=True)
+    do = wl.bf16_bits_to_f64(w.tensors().dout)
+    ro, _ = oattn.forward_single(q, k, v, spd, bias)
+    rdq, rdk, rdv, rdb = oattn.backward_single(q, k, v, do, spd, bias)
+    layout = ring.RingLayout.even(N, N_SUPER, world)
+    sa, sb = layout.super_range
+    s_ = 1.0 / np.sqrt(float(D_HEAD))
+    for rank, o_sh, dq_sh, dk_sh, dv_sh, dq_sup, (dk_sup, dv_sup, db), done in res:
+        a, b = layout.shards[rank]
+        assert done == ["forward state final"]
+        np.testing.assert_allclose(o_sh, ro[a:b], rtol=1e-10, atol=1e-13)
+        np.testing.assert_allclose(dq_sh * s_, rdq[a:b], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(dk_sh * s_, rdk[a:b], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(dv_sh, rdv[a:b], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(dq_sup * s_, rdq[sa:sb], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(dk_sup * s_, rdk[sa:sb], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(dv_sup, rdv[sa:sb], rtol=1e-9, atol=1e-12)
+        np.testing.assert_allclose(db, rdb, rtol=1e-9, atol=1e-12)
