@@ -41,11 +41,12 @@ UNIT = "TFLOP/s"
 DEFAULT_WORKLOAD = "powerlaw64k"
 ORACLE_SAMPLE_ROWS = 256
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the backward kernel, from the ncu
-# capture summarised in profiles/attn_bwd_kernel_powerlaw16k.md (16 384-node graph, scaled by N^2).
+# Measured DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture) per launch of the
+# backward kernel on a 16 384-node graph, divided by N^2: the traffic is dominated by the N^2 bias-index tiles
+# and the N^2/128 dQ reductions, so a launch at another size is estimated as this figure times sum n_g^2.
 BWD_KERNEL_DRAM_BYTES_PER_N2 = 1036.5e6 / (16384.0 ** 2)
-# the same for the forward kernel (profiles/attn_fwd_kernel_powerlaw16k.md) and for the bit-matrix SPD build
-# (profiles/spd_dense_kernel_pl24000.md: 24 000-node graph; its traffic grows with N^2 x levels, so this is an estimate)
+# The same for the forward kernel (16 384 nodes) and for the bit-matrix SPD build (24 000 nodes; its traffic
+# also grows with the number of BFS levels, so the scaled figure is an estimate).
 FWD_KERNEL_DRAM_BYTES_PER_N2 = 438.7e6 / (16384.0 ** 2)
 SPD_DENSE_DRAM_BYTES_PER_N2 = 2.71e9 / (24000.0 ** 2)
 
@@ -261,6 +262,23 @@ def run_cuda(args) -> int:
     total_ms = e0.elapsed_time(e1)
     ph = np.array([[m[j].elapsed_time(m[j + 1]) for j in range(4)] for m in marks])       # [K, 4]
     spd_ms, fwd_ms, bwd_ms, chk_ms = (float(x) for x in ph.mean(axis=0))
+    phase_names = ("spd_build", "fwd", "bwd", "fwd_chunked")
+    ph_median = {nm: float(x) for nm, x in zip(phase_names, np.median(ph, axis=0))}
+    ph_min = {nm: float(x) for nm, x in zip(phase_names, ph.min(axis=0))}
+    fb = ph[:, 1] + ph[:, 2]
+
+    # ---- input statistics (outside the timed region): degrees, and the bucket histogram of a row sample of the built matrix ----
+    deg = np.diff(b.row_ptr)
+    n0 = int(b.cu_seqlens[1])
+    ld0 = int(b.spd_ld[0])
+    row_idx = torch.arange(0, n0, max(1, n0 // 1024), device=dev)[:1024]          # rows spread over the whole graph
+    n_hist_rows = int(row_idx.numel())
+    sample = spd[: n0 * ld0].view(n0, ld0)[row_idx][:, :n0]
+    hist = torch.bincount(sample.reshape(-1).to(torch.int32), minlength=D + 2)[: D + 2].double()
+    hist = (hist / hist.sum()).cpu().numpy()
+    graph_stats = {"deg_min": int(deg.min()), "deg_mean": float(deg.mean()), "deg_max": int(deg.max()),
+                   "spd_bucket_fractions": {"rows_sampled": n_hist_rows, "of_graph": 0,
+                                            "fractions": [round(float(x), 5) for x in hist]}}
     f_fwd, f_bwd = w.attn_flops()
     ms_step, _ = dist_util.aggregate(total_ms / args.steps, 0.0, dev)
     fb_ms, flops_all = dist_util.aggregate(fwd_ms + bwd_ms, f_fwd + f_bwd, dev)
@@ -471,9 +489,13 @@ def run_cuda(args) -> int:
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": args.workload, "note": w.note, "n_total": T, "n_graphs": b.n_graphs, "n_heads": H,
                    "head_dim": d, "max_dist": D, "n_kv_chunks": n_chunks, "nnz": int(ci.numel()),
+                   "graph": graph_stats,
                    "step": "spd_build + fwd + bwd + chunked fwd", "parallelism": f"dp{world} (independent batches)",
                    "l2": "inputs larger than L2: the SPD matrix (%.2f GB) is rebuilt and re-streamed every step" % (b.spd_bytes / 1e9)},
         "phases_ms": {"spd_build": spd_ms, "fwd": fwd_ms, "bwd": bwd_ms, "fwd_chunked": chk_ms if single else None},
+        "phases_ms_median": ph_median, "phases_ms_min": ph_min,
+        "fwd_bwd_ms": {"mean": float(fb.mean()), "median": float(np.median(fb)), "min": float(fb.min()), "repetitions": int(len(fb)),
+                       "note": "rank 0; `value` uses the mean (max over ranks)"},
         "fwd_tflops": f_fwd / (fwd_ms * 1e-3) / 1e12, "bwd_tflops": bwd_tflops,
         "fwd_chunked_tflops": (f_fwd / (chk_ms * 1e-3) / 1e12) if single else None,
         "bwd_chunked": bwd_chunked, "fwd_ring_steps": fwd_ring, "bwd_ring_steps": bwd_ring,

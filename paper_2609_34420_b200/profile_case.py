@@ -3,8 +3,8 @@
     python -m paper_2609_34420_b200.profile_case WORKLOAD [REPS] [spd|fwd|bwd|chunked|all]
 
 WORKLOAD is one of the named workloads (tiny_er256, ba4096, powerlaw16k, powerlaw64k,
-varlen_rgg64) or plN for a power-law graph of N nodes (H=8, d=64, max_dist=24).  It is the small,
-self-contained target used for the ncu captures summarised under profiles/.
+varlen_rgg64) or plN for a power-law graph of N nodes (H=8, d=64, max_dist=24).  A small,
+self-contained timing command line for one entry point at a time.
 """
 from __future__ import annotations
 
