@@ -95,10 +95,12 @@ gt_status gt_check(void* workspace, void* stream);
  * distinct from unreachable pairs (bucket max_dist+1).  Bit-exact and deterministic.
  * Out-of-range col_idx entries are undefined behaviour.
  * Workspace: 256 bytes + 4(G+1) when every graph has at most 17 066 nodes; a single larger graph
- * needs about 15 KB per node for each of min(4, ceil(n/8192)) groups of thread blocks (fifteen bit
- * matrices of 1 KB rows per group; 3.9 GB at 65 536 nodes) plus 16 bytes per 32 edges, and a
- * device that supports cooperative launches; a batch that contains a larger graph needs 12 bytes
- * per node of the largest graph for each of up to 2 x (number of SMs) thread blocks.
+ * needs about 7 KB per node for each of min(4, ceil(n/8192)) groups of thread blocks (seven bit
+ * matrices of 1 KB rows per group: visited, and one frontier per level up to 5; later levels reuse two of
+ * them) plus 1 KB per 33 edges per group (rows for vertices with more than 32 out-edges) and 16 bytes per
+ * 32 edges -- 2.0 GB at 65 536 nodes with 786 000 edges -- and a device that supports cooperative
+ * launches; a batch that contains a larger graph needs 12 bytes per node of the largest graph for each
+ * of up to 2 x (number of SMs) thread blocks.
  * ------------------------------------------------------------------------------------- */
 size_t gt_spd_build_workspace(const gt_batch* batch, int64_t nnz, int32_t max_dist);
 gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx, int64_t nnz,

@@ -237,7 +237,7 @@ constexpr int kDenseVecs = kDenseRowWords / 128;         // 16-byte vectors per 
 constexpr int kDenseChunk = 32;                          // out-edges per work item
 constexpr int kDenseBatch = 4;                           // work items a warp takes at a time
 constexpr int kDenseMaxGroups = 4;                       // CTA groups working on different column blocks at once
-constexpr int kDenseHist = 12;                           // levels whose frontier matrices are kept for the output pass
+constexpr int kDenseHist = 5;                            // levels whose frontier matrices are kept for the output pass (later levels blend into written rows)
 constexpr int kDensePlanes = kDenseHist + 1;             // frontier matrices per group (level 0 .. kDenseHist)
 constexpr int kDenseFlagWords = 8192;                    // row flags of a level kept as a bitmap in shared memory (graphs up to 262 144 vertices)
 constexpr uint32_t kGridWaitIterations = 1u << 24;
@@ -245,7 +245,9 @@ constexpr uint32_t kGridWaitIterations = 1u << 24;
 struct DenseParams {
     uint32_t* vis;          // [n_max][kDenseRowWords]
     uint32_t* fr;           // [kDensePlanes][n_max][kDenseRowWords] frontier of level l in plane l (later levels: planes 0 / 1 in turn)
-    uint32_t* acc;          // [n_max][kDenseRowWords] accumulator rows of split vertices (all zero between uses)
+    uint32_t* acc;          // [acc_rows][kDenseRowWords] accumulator rows of split vertices (all zero between uses)
+    int32_t* acc_row;       // [n_max] accumulator row of a split vertex (vertices with more than kDenseChunk out-edges)
+    int32_t acc_rows;       // accumulator rows per CTA group
     uint32_t* acc_cnt;      // [n_max] finished chunks of a split vertex
     uint8_t* nonempty;      // [kDensePlanes][n_pad] the row of that plane is valid and has a bit set (rows without the flag are never read)
     uint8_t* row_done;      // [n_max] every valid target of the block is visited
@@ -259,34 +261,41 @@ struct DenseParams {
     uint32_t barrier_limit; // polls of the barrier word before a thread block gives up
 };
 
-// item_start[v] = sum_{u<v} max(1, ceil(deg(u)/64)) for the vertices of one graph.  One block.
-__global__ void spd_dense_items_kernel(const int32_t* __restrict__ rp, int32_t n, int32_t* __restrict__ item_start)
+// item_start[v] = sum_{u<v} max(1, ceil(deg(u)/32)) for the vertices of one graph, and acc_row[v] = number of split
+// vertices (more than one chunk) before v.  One block; both prefix sums ride in one 64-bit scan.
+__global__ void spd_dense_items_kernel(const int32_t* __restrict__ rp, int32_t n, int32_t* __restrict__ item_start,
+                                       int32_t* __restrict__ acc_row)
 {
-    __shared__ int32_t carry;
-    __shared__ int32_t part[1024];
-    if (threadIdx.x == 0) carry = 0;
+    __shared__ unsigned long long carry;
+    __shared__ unsigned long long part[1024];
+    if (threadIdx.x == 0) carry = 0ull;
     __syncthreads();
     for (int base = 0; base < n; base += blockDim.x) {
         const int v = base + threadIdx.x;
-        int32_t cnt = 0;
+        unsigned long long cnt = 0ull;
         if (v < n) {
             const int32_t deg = rp[v + 1] - rp[v];
-            cnt = deg <= kDenseChunk ? 1 : (deg + kDenseChunk - 1) / kDenseChunk;
+            const unsigned long long chunks = deg <= kDenseChunk ? 1 : (deg + kDenseChunk - 1) / kDenseChunk;
+            cnt = chunks | ((chunks > 1 ? 1ull : 0ull) << 32);
         }
         part[threadIdx.x] = cnt;
         __syncthreads();
         for (int off = 1; off < (int)blockDim.x; off <<= 1) {
-            int32_t add = threadIdx.x >= (unsigned)off ? part[threadIdx.x - off] : 0;
+            unsigned long long add = threadIdx.x >= (unsigned)off ? part[threadIdx.x - off] : 0ull;
             __syncthreads();
             part[threadIdx.x] += add;
             __syncthreads();
         }
-        if (v < n) item_start[v] = carry + part[threadIdx.x] - cnt;
+        if (v < n) {
+            const unsigned long long before = carry + part[threadIdx.x] - cnt;
+            item_start[v] = (int32_t)(before & 0xffffffffull);
+            acc_row[v] = (int32_t)(before >> 32);
+        }
         __syncthreads();
         if (threadIdx.x == blockDim.x - 1) carry += part[threadIdx.x];
         __syncthreads();
     }
-    if (threadIdx.x == 0) item_start[n] = carry;
+    if (threadIdx.x == 0) item_start[n] = (int32_t)(carry & 0xffffffffull);
 }
 
 __global__ void spd_dense_item_rec_kernel(const int32_t* __restrict__ rp, const int32_t* __restrict__ item_start, int32_t n,
@@ -370,7 +379,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
     const uint32_t n_ctas = ((uint32_t)gridDim.x - (uint32_t)grp + (uint32_t)d.n_groups - 1u) / (uint32_t)d.n_groups;
     {
         const size_t m = (size_t)grp * d.n_max;
-        d.vis += m * kDenseRowWords; d.fr += m * kDensePlanes * kDenseRowWords; d.acc += m * kDenseRowWords;
+        d.vis += m * kDenseRowWords; d.fr += m * kDensePlanes * kDenseRowWords; d.acc += (size_t)grp * d.acc_rows * kDenseRowWords;
         d.acc_cnt += m; d.nonempty += (size_t)grp * d.n_pad * kDensePlanes; d.row_done += m;
         d.sync += grp * 64;
     }
@@ -624,7 +633,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
                 if (n_chunks == 1) {
                     finalise(s, acc, col0, vis_row, next_row, ne_next, code, flag_idx, emitted);
                 } else {
-                    uint32_t* acc_row = d.acc + (size_t)s * kDenseRowWords;
+                    uint32_t* acc_row = d.acc + (size_t)d.acc_row[s] * kDenseRowWords;
 #pragma unroll
                     for (int q = 0; q < kDenseVecs; ++q)
 #pragma unroll
@@ -679,7 +688,8 @@ struct SpdPlan {
     bool smem_state;
     bool dense;                // single large graph: bit-matrix BFS (persistent cooperative kernel)
     int dense_groups;
-    size_t dense_off[9];       // vis, frontier planes, acc, acc_cnt, nonempty flags, row_done, item_start, sync, item_rec
+    size_t dense_off[10];      // vis, frontier planes, acc, acc_cnt, nonempty flags, row_done, item_start, sync, item_rec, acc_row
+    int32_t dense_acc_rows;    // accumulator rows per CTA group: a bound on the vertices with more than kDenseChunk out-edges
     int threads;
     int grid;
     size_t smem_bytes;
@@ -722,10 +732,12 @@ SpdPlan make_plan(const gt_batch* b, int64_t nnz)
             pl.dense_groups = n_col_blocks < kDenseMaxGroups ? n_col_blocks : kDenseMaxGroups;
             const size_t G = (size_t)pl.dense_groups;
             const size_t mat = align_up(G * n * kDenseRowWords * sizeof(uint32_t), 256);
+            const size_t split_bound = (size_t)(nnz > 0 ? nnz : 0) / (kDenseChunk + 1) + 1;
+            pl.dense_acc_rows = (int32_t)(split_bound < n ? split_bound : n);
             size_t off = pl.scratch_off;
             pl.dense_off[0] = off; off += mat;
             pl.dense_off[1] = off; off += mat * kDensePlanes;
-            pl.dense_off[2] = off; off += mat;
+            pl.dense_off[2] = off; off += align_up(G * (size_t)pl.dense_acc_rows * kDenseRowWords * sizeof(uint32_t), 256);
             pl.dense_off[3] = off; off += align_up(G * n * sizeof(uint32_t), 256);
             pl.dense_off[4] = off; off += align_up(G * align_up(n, 32) * kDensePlanes, 256);
             pl.dense_off[5] = off; off += align_up(G * n, 256);
@@ -733,6 +745,7 @@ SpdPlan make_plan(const gt_batch* b, int64_t nnz)
             pl.dense_off[7] = off; off += 256 * kDenseMaxGroups;
             // work items: one per vertex plus one per further chunk of out-edges
             pl.dense_off[8] = off; off += align_up((n + (size_t)(nnz > 0 ? nnz : 0) / kDenseChunk + 1) * sizeof(int4), 256);
+            pl.dense_off[9] = off; off += align_up(n * sizeof(int32_t), 256);
             pl.total_bytes = off;
         } else {
             cudaGetLastError();
@@ -796,6 +809,8 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
         d.item_start = (int32_t*)(ws + pl.dense_off[6]);
         d.sync = (uint32_t*)(ws + pl.dense_off[7]);
         d.item_rec = (int4*)(ws + pl.dense_off[8]);
+        d.acc_row = (int32_t*)(ws + pl.dense_off[9]);
+        d.acc_rows = pl.dense_acc_rows;
         d.n_max = batch->n_total;
         d.n_pad = (int32_t)align_up((size_t)batch->n_total, 32);
         d.n_groups = pl.dense_groups;
@@ -805,7 +820,7 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
         // accumulator rows, their counters and the barrier words start at zero
         GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[2], 0, pl.dense_off[4] - pl.dense_off[2], s));
         GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[7], 0, 256 * kDenseMaxGroups, s));
-        spd_dense_items_kernel<<<1, 1024, 0, s>>>(row_ptr, batch->n_total, d.item_start);
+        spd_dense_items_kernel<<<1, 1024, 0, s>>>(row_ptr, batch->n_total, d.item_start, d.acc_row);
         GT_CUDA_TRY(cudaGetLastError());
         spd_dense_item_rec_kernel<<<(unsigned)((batch->n_total + 255) / 256), 256, 0, s>>>(row_ptr, d.item_start, batch->n_total, d.item_rec);
         GT_CUDA_TRY(cudaGetLastError());

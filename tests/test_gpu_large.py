@@ -140,29 +140,34 @@ def test_bit_matrix_build_directed_ragged_with_hub_and_isolated_vertices():
     np.testing.assert_array_equal(got, exp)
 
 
-@pytest.mark.parametrize("chain", [6, 7])
-def test_bit_matrix_build_depth_around_the_kept_levels(chain):
-    """Chains of `chain` vertices hanging off one centre: the longest path has 2 * chain hops.  With 12
-    levels kept for the output pass, chain = 6 ends exactly there (the pass runs while the last level still
-    found pairs, the level after finds none) and chain = 7 adds two levels that blend into written rows.
-    Directed extras make the matrix asymmetric; a few vertices stay isolated."""
-    n_chains = 17200 // chain
-    n = 1 + n_chains * chain + 37               # 37 isolated vertices at the end
+@pytest.mark.parametrize("base,one_longer", [(2, False), (2, True), (3, False), (6, True)])
+def test_bit_matrix_build_depth_around_the_kept_levels(base, one_longer):
+    """Chains of `base` vertices hanging off one centre (one of them a vertex longer if asked): the longest path
+    has 2 * base (+ 1) hops.  The build keeps the frontiers of five levels for its output pass: 4 hops end before
+    that, 5 exactly there (the pass runs while the last level still found pairs, the level after finds none),
+    6 add one level and 13 add eight levels that blend into written rows.  Directed extras make the matrix
+    asymmetric; a few vertices stay isolated."""
+    n_chains = 17200 // base
+    lengths = [base] * n_chains
+    if one_longer:
+        lengths[n_chains // 2] += 1
+    firsts = 1 + np.concatenate([[0], np.cumsum(lengths)[:-1]])
+    n = 1 + int(np.sum(lengths)) + 37           # 37 isolated vertices at the end
     src, dst = [], []
-    for c in range(n_chains):
-        first = 1 + c * chain
-        src.append(0); dst.append(first)
-        for t in range(chain - 1):
-            src.append(first + t); dst.append(first + t + 1)
+    for first, length in zip(firsts, lengths):
+        src.append(0); dst.append(int(first))
+        for t in range(length - 1):
+            src.append(int(first) + t); dst.append(int(first) + t + 1)
     src, dst = np.array(src), np.array(dst)
     both_src, both_dst = np.concatenate([src, dst]), np.concatenate([dst, src])
-    # one-way shortcuts from chain ends back to the centre's first neighbour of the next chain
-    ends = 1 + np.arange(0, n_chains - 1, 97) * chain + (chain - 1)
-    both_src = np.concatenate([both_src, ends]); both_dst = np.concatenate([both_dst, ends + 1])
+    # one-way shortcuts from some chain ends to the first vertex of the next chain
+    pick = np.arange(0, n_chains - 1, 97)
+    ends = firsts[pick] + np.array(lengths)[pick] - 1
+    both_src = np.concatenate([both_src, ends]); both_dst = np.concatenate([both_dst, firsts[pick + 1]])
     csr = wl.csr_from_edges(n, both_src, both_dst, symmetric=False)
     w, got = _spd_of(csr, 24)
     exp = ospd.spd_matrix(w.batch.row_ptr, w.batch.col_idx, 24)
-    assert int(exp[exp <= 24].max()) == 2 * chain
+    assert int(exp[exp <= 24].max()) == 2 * base + (1 if one_longer else 0)
     np.testing.assert_array_equal(got, exp)
 
 
