@@ -246,6 +246,8 @@ def run_cuda(args) -> int:
     # ---- timed region ----
     sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid)) if rank == 0 else None
     marks = [[ev() for _ in range(5)] for _ in range(args.steps)]
+    kern_ev = [[ev() for _ in range(args.steps)] for _ in range(2)]       # around the backward's main kernel, recorded by the library
+    gt.gt_profile_bwd_kernel_events(kern_ev[0], kern_ev[1])
     e0, e1 = ev(), ev()
     dist_util.barrier(dev)
     torch.cuda.synchronize()
@@ -259,6 +261,8 @@ def run_cuda(args) -> int:
     for wsx in (ws_spd, ws_fwd, ws_bwd) + ((ws_chk,) if single else ()):
         gt.gt_check(wsx)
 
+    gt.gt_profile_bwd_kernel_events([], [])
+    bwd_kernel_ms = float(np.mean([a_.elapsed_time(b_) for a_, b_ in zip(kern_ev[0], kern_ev[1])]))
     total_ms = e0.elapsed_time(e1)
     ph = np.array([[m[j].elapsed_time(m[j + 1]) for j in range(4)] for m in marks])       # [K, 4]
     spd_ms, fwd_ms, bwd_ms, chk_ms = (float(x) for x in ph.mean(axis=0))
@@ -451,14 +455,18 @@ def run_cuda(args) -> int:
 
     peaks, peak_kind = load_peaks()
     bwd_tflops = f_bwd / (bwd_ms * 1e-3) / 1e12
+    bwd_kernel_tflops = f_bwd / (bwd_kernel_ms * 1e-3) / 1e12
     peak_tf = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
     sum_n2 = float(b.sum_n2)
     roofline = {
-        "kernel": "attn_bwd_kernel", "bound": "tensor", "achieved": bwd_tflops, "peak": peak_tf, "unit": "TFLOP/s",
-        "frac": bwd_tflops / peak_tf, "peak_kind": f"bf16_tflops_sustained of {peak_kind} (kernel timed inside a long step)",
-        "frac_of_burst_peak": bwd_tflops / float(peaks["bf16_tflops"]),
+        "kernel": "attn_bwd_kernel", "bound": "tensor", "achieved": bwd_kernel_tflops, "peak": peak_tf, "unit": "TFLOP/s",
+        "frac": bwd_kernel_tflops / peak_tf, "peak_kind": f"bf16_tflops_sustained of {peak_kind} (kernel timed inside a long step)",
+        "frac_of_burst_peak": bwd_kernel_tflops / float(peaks["bf16_tflops"]),
         "traffic": None if BWD_KERNEL_DRAM_BYTES_PER_N2 is None else BWD_KERNEL_DRAM_BYTES_PER_N2 * sum_n2,
-        "flops_per_launch": f_bwd, "ms_per_launch": bwd_ms,
+        "flops_per_launch": f_bwd, "ms_per_launch": bwd_kernel_ms,
+        "timing": "CUDA events recorded by the library around the kernel's launch inside every timed step (mean over the steps)",
+        "ms_per_call": bwd_ms, "frac_of_call": bwd_tflops / peak_tf,
+        "call_note": "gt_biased_attn_bwd also runs the SPD transpose, the per-query pre-pass, two zero fills and the final conversion",
     }
     fwd_tflops_ = f_fwd / (fwd_ms * 1e-3) / 1e12
     roofline_fwd = {

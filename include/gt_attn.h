@@ -223,6 +223,13 @@ gt_status gt_biased_attn_bwd_ex(const void* q, const void* k, const void* v, con
                                 void* dq, void* dk, void* dv, float* dbias, const float* out_f32,
                                 void* workspace, size_t workspace_bytes, void* stream);
 
+/* gt_profile_bwd_kernel_events -- measurement hook (no counterpart in the paper): `before` and `after` are host
+ * arrays of n caller-owned cudaEvent_t handles (passed as void*); the i-th of the next n calls of
+ * gt_biased_attn_bwd / _bwd_ex / _bwd_chunked records before[i] and after[i] on its stream around the launches of
+ * its main kernel (after the pre-passes, before the final conversion), so that a benchmark can report the kernel's
+ * own duration from inside its timed loop.  n = 0 or NULL arrays switch the hook off.  Not thread-safe. */
+void gt_profile_bwd_kernel_events(void** before, void** after, int32_t n);
+
 /* ---------------------------------------------------------------------------------------
  * gt_biased_attn_fwd_step -- one ring step of graph-aware context parallelism driven by the caller
  * (Sec. GA-CP, items 1-3): the query rows [q_begin, q_end) of a rank attend to ONE incoming key/value

@@ -25,7 +25,7 @@ EXPORTS = ("gt_status_string", "gt_check",
            "gt_spd_build_workspace", "gt_spd_build", "gt_spd_build_static_limit", "gt_spd_build_static",
            "gt_spd_validate_workspace", "gt_spd_validate", "gt_spd_validate_count", "gt_test_hook_barrier_overcount",
            "gt_biased_attn_fwd_workspace", "gt_biased_attn_fwd", "gt_biased_attn_fwd_ex",
-           "gt_biased_attn_bwd_workspace", "gt_biased_attn_bwd", "gt_biased_attn_bwd_ex",
+           "gt_biased_attn_bwd_workspace", "gt_biased_attn_bwd", "gt_biased_attn_bwd_ex", "gt_profile_bwd_kernel_events",
            "gt_biased_attn_fwd_chunked_workspace", "gt_biased_attn_fwd_chunked",
            "gt_biased_attn_bwd_chunked_workspace", "gt_biased_attn_bwd_chunked",
            "gt_biased_attn_fwd_step_workspace", "gt_biased_attn_fwd_step",
@@ -90,6 +90,8 @@ def lib() -> ctypes.CDLL:
         L.gt_biased_attn_bwd.argtypes = [vp] * 9 + [bp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
         L.gt_biased_attn_bwd_ex.restype = ctypes.c_int
         L.gt_biased_attn_bwd_ex.argtypes = [vp] * 9 + [bp, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.gt_profile_bwd_kernel_events.restype = None
+        L.gt_profile_bwd_kernel_events.argtypes = [vp, vp, i32]
         L.gt_biased_attn_fwd_chunked_workspace.restype = sz
         L.gt_biased_attn_fwd_chunked_workspace.argtypes = [bp, i32, i32, i32]
         L.gt_biased_attn_fwd_chunked.restype = ctypes.c_int
@@ -419,3 +421,23 @@ def gt_feature_attn_bwd(q, k, v, dout, lse, features, weights, batch: Batch, dq,
                                    _ptr(workspace), workspace.numel(), _stream())
     _raise(st, "gt_feature_attn_bwd")
     return workspace
+
+
+_profile_keepalive = None
+
+
+def gt_profile_bwd_kernel_events(before, after) -> None:
+    """Have the next ``len(before)`` backward calls record the given torch CUDA events (created with
+    ``enable_timing=True``) around their main kernel; pass empty lists to switch the hook off."""
+    global _profile_keepalive
+    n = len(before)
+    if n == 0:
+        lib().gt_profile_bwd_kernel_events(None, None, 0)
+        _profile_keepalive = None
+        return
+    for e in list(before) + list(after):
+        e.record()                                   # torch creates the CUDA event lazily, at its first record
+    arr_t = ctypes.c_void_p * n
+    a, b = arr_t(*[e.cuda_event for e in before]), arr_t(*[e.cuda_event for e in after])
+    _profile_keepalive = (a, b, list(before), list(after))
+    lib().gt_profile_bwd_kernel_events(a, b, n)

@@ -791,6 +791,24 @@ extern "C" size_t gt_biased_attn_bwd_workspace(const gt_batch* batch, int32_t n_
     return gt::bwd_workspace(batch, n_heads, head_dim, max_dist).total;
 }
 
+// Optional timing hook (gt_profile_bwd_kernel_events): pairs of caller-owned CUDA events recorded around the main
+// kernel launches of the next backward calls, so that a benchmark can time the kernel itself inside its own loop.
+namespace gt {
+namespace {
+cudaEvent_t* g_prof_before = nullptr;
+cudaEvent_t* g_prof_after = nullptr;
+int g_prof_n = 0, g_prof_next = 0;
+}  // namespace
+}  // namespace gt
+
+extern "C" void gt_profile_bwd_kernel_events(void** before, void** after, int32_t n)
+{
+    gt::g_prof_before = (cudaEvent_t*)before;
+    gt::g_prof_after = (cudaEvent_t*)after;
+    gt::g_prof_n = (before && after && n > 0) ? n : 0;
+    gt::g_prof_next = 0;
+}
+
 // Shared by the one-shot and the chunked entry point: pre-passes, one launch of the main kernel per key chunk
 // (the chunks run one after the other in stream order, like ring steps; dQ and dB accumulate across them,
 // dK and dV of a chunk's rows are complete when its launch ends), then the final conversion.
@@ -867,6 +885,8 @@ static gt_status gt_bwd_run(const void* q, const void* k, const void* v, const v
     const int32_t all_tiles = (batch->max_seqlen + kTile - 1) / kTile;
     const int32_t tiles_per_chunk = ((batch->max_seqlen + n_kv_chunks - 1) / n_kv_chunks + kTile - 1) / kTile;
     double* db_base = p.db_acc;
+    const int prof = g_prof_next < g_prof_n ? g_prof_next++ : -1;
+    if (prof >= 0) GT_CUDA_TRY(cudaEventRecord(g_prof_before[prof], s));
     for (int32_t c = 0; c < n_kv_chunks; ++c) {
         p.db_acc = db_base + (size_t)c * n_db;
         p.kv_row0 = n_kv_chunks == 1 ? 0 : c * tiles_per_chunk * kTile;
@@ -877,6 +897,7 @@ static gt_status gt_bwd_run(const void* q, const void* k, const void* v, const v
                             : launch_bwd<32>(tq, tk, tv, tdo, text, tspd, p, batch, s);
         if (st != GT_OK) return st;
     }
+    if (prof >= 0) GT_CUDA_TRY(cudaEventRecord(g_prof_after[prof], s));
     p.db_acc = db_base;
     const size_t n_vec4 = rows * head_dim / 4;
     const size_t n_fin = n_vec4 > (size_t)n_db ? n_vec4 : (size_t)n_db;
