@@ -94,7 +94,8 @@ gt_status gt_check(void* workspace, void* stream);
  * The traversal runs to exhaustion, so pairs farther than max_dist (bucket max_dist) stay
  * distinct from unreachable pairs (bucket max_dist+1).  Bit-exact and deterministic.
  * Out-of-range col_idx entries are undefined behaviour.
- * Workspace: 256 bytes + 4(G+1) when every graph has at most 17 066 nodes; a single larger graph
+ * Workspace: 256 bytes + 4(G+1) for a packed batch whose graphs have at most 17 066 nodes each and for a single
+ * graph below 14 500 nodes; a single larger graph (it takes a bit-matrix traversal, which is the faster one from there)
  * needs about 7 KB per node for each of min(4, ceil(n/8192)) groups of thread blocks (seven bit
  * matrices of 1 KB rows per group: visited, and one frontier per level up to 5; later levels reuse two of
  * them) plus 1 KB per 33 edges per group (rows for vertices with more than 32 out-edges) and 16 bytes per
@@ -121,8 +122,8 @@ gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx, int64_t n
  *
  * Same arguments, results and error codes as gt_spd_build, minus the workspace, with these rules:
  *  - Size limit: the batch must satisfy gt_spd_build_workspace(batch, nnz, max_dist) <=
- *    gt_spd_build_static_limit(); in practice every graph of the batch has at most 17 066 nodes
- *    (larger graphs keep their traversal state in the workspace and need far more).  Otherwise
+ *    gt_spd_build_static_limit(); in practice a packed batch whose graphs have at most 17 066 nodes each, or a
+ *    single graph below 14 500 nodes (larger ones keep their traversal state in the workspace and need far more).  Otherwise
  *    GT_ERR_WORKSPACE is returned and nothing is launched.
  *  - First call per device: the first call made with a given device current looks up the
  *    device address of the built-in array (a one-off set-up step).  Make that first call outside
@@ -157,7 +158,7 @@ gt_status gt_spd_validate_count(void* workspace, void* stream, int64_t* count_ho
  * gt_test_hook_barrier_overcount -- test hook of the device-timeout path (no counterpart in the
  * paper).  Every device-side wait of this library is bounded; one that runs out makes its kernel
  * return and gt_check() report GT_ERR_DEVICE_TIMEOUT.  After gt_test_hook_barrier_overcount(k), k > 0,
- * the NEXT bit-matrix build of this process (gt_spd_build on a single graph beyond 17 066 nodes) waits
+ * the NEXT bit-matrix build of this process (gt_spd_build on a single graph of 14 500 nodes or more) waits
  * at its grid barriers for k arrivals more than there are thread blocks, with a shortened limit, so the
  * wait runs out within a second; the kernel issues no asynchronous copies, so nothing is in flight when
  * it returns, the context stays usable and the next build is normal.  The output of the hooked build

@@ -73,11 +73,21 @@ def test_named_workloads(name):
 
 
 def test_single_graph_beyond_the_shared_memory_state_matches_and_is_deterministic():
-    """A single graph above the shared-memory state limit (17 066 nodes) takes the bit-matrix build."""
+    """A single graph of 14 500 nodes or more takes the bit-matrix build."""
     w = wl.Workload("pl20k", wl.pack_graphs([wl.chung_lu_power_law(20000, 8.0, 2.1, 3)]), 1, 32, 10)
     a = check(w)
     b = gpu_spd(w).cpu().numpy()
     np.testing.assert_array_equal(a, b)
+
+
+@pytest.mark.parametrize("n", [14499, 14500, 16001])
+def test_single_graphs_around_the_switch_to_the_bit_matrix_build(n):
+    """14 499 nodes: multi-source BFS with the state in shared memory; 14 500 and 16 001: bit-matrix build with a
+    ragged second column block.  Directed, so that the matrix is asymmetric."""
+    rng = np.random.Generator(np.random.PCG64(n))
+    m = 4 * n
+    csr = wl.csr_from_edges(n, rng.integers(0, n - 50, m), rng.integers(0, n - 20, m), symmetric=False)
+    check(wl.Workload("switch", wl.pack_graphs([csr]), 1, 32, 7))
 
 
 def test_packed_batch_with_a_graph_beyond_the_shared_memory_state():
