@@ -132,10 +132,27 @@ __global__ void __launch_bounds__(1024, kSmemState ? 1 : 2) spd_bfs_kernel(SpdPa
                     if (f) { e0 = rp[v]; e1 = rp[v + 1]; }
                 }
                 uint32_t uni = __reduce_or_sync(0xffffffffu, f);
-                while (uni) {                               // one source row at a time: coalesced run
-                    int b = __ffs(uni) - 1;
-                    uni &= uni - 1;
-                    if ((f >> b) & 1u) out0[(int64_t)b * ld + v] = code;
+                if (uni == 0u) continue;                    // no frontier vertex among these 32: nothing to emit or push
+                // Dense frontiers (small-world graphs: many lanes share a source bit): one source row at a time, so that a
+                // warp store fills a run of one row.  Thin frontiers (graphs of large diameter: a lane holds one or two
+                // bits, the warp many different ones): every lane walks its own bits, a few rounds instead of one per
+                // source that occurs in the warp.
+                const int own_rounds = (int)__reduce_max_sync(0xffffffffu, (unsigned)__popc(f));
+                if (__popc(uni) > 2 * own_rounds) {
+                    uint32_t mine = f;
+                    for (int k = 0; k < own_rounds; ++k) {
+                        if (mine) {
+                            const int b = __ffs(mine) - 1;
+                            mine &= mine - 1;
+                            out0[(int64_t)b * ld + v] = code;
+                        }
+                    }
+                } else {
+                    while (uni) {
+                        int b = __ffs(uni) - 1;
+                        uni &= uni - 1;
+                        if ((f >> b) & 1u) out0[(int64_t)b * ld + v] = code;
+                    }
                 }
                 const int deg = e1 - e0;
                 if (f && deg <= kWarpDegree) {
