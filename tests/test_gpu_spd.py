@@ -162,6 +162,23 @@ def test_spd_validate_counts_entries_that_name_no_bucket():
     assert gt.gt_spd_validate_count(ws) == planted
 
 
+def test_spd_validate_on_a_single_graph_built_on_the_gpu():
+    from gpu_util import device_batch
+    from paper_2609_34420_b200 import binding as gt
+    w = wl.make_workload("ba4096")
+    bt = device_batch(w.batch)
+    spd = gpu_spd(w)
+    ws = gt.gt_spd_validate(spd, bt, w.max_dist)
+    gt.gt_check(ws)
+    assert gt.gt_spd_validate_count(ws) == 0
+    ws = gt.gt_spd_validate(spd, bt, 3)             # declared with fewer buckets than the matrix holds: distances 4, 5 count
+    with pytest.raises(gt.GtError) as e:
+        gt.gt_check(ws)
+    assert e.value.status == 7
+    host = spd.cpu().numpy().reshape(4096, -1)[:, :4096]
+    assert gt.gt_spd_validate_count(ws) == int((host >= 5).sum())
+
+
 def test_a_workspace_whose_header_was_not_zeroed_is_reported_not_trusted():
     """The first 256 bytes of a workspace must be zero when it is first handed over; a dirty header shows up as
     an error from gt_check (which clears it), never as a silently accepted status."""
