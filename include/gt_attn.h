@@ -94,8 +94,9 @@ gt_status gt_check(void* workspace, void* stream);
  * The traversal runs to exhaustion, so pairs farther than max_dist (bucket max_dist) stay
  * distinct from unreachable pairs (bucket max_dist+1).  Bit-exact and deterministic.
  * Out-of-range col_idx entries are undefined behaviour.
- * Workspace: 256 bytes + 4(G+1) for a packed batch whose graphs have at most 17 066 nodes each and for a single
- * graph below 14 500 nodes; a single larger graph (it takes a bit-matrix traversal, which is the faster one from there)
+ * Workspace: about 4(G+1) + 4 n_total + 4 G + 1 KB for a packed batch whose graphs have at most 17 066 nodes each and
+ * for a single graph below 14 500 nodes (per-graph offsets, and the connected-component label of every node: the search
+ * of an undirected graph without a vertex of more than 64 out-edges stops at level max_dist); a single larger graph (it takes a bit-matrix traversal, which is the faster one from there)
  * needs about 7 KB per node for each of min(4, ceil(n/8192)) groups of thread blocks (seven bit
  * matrices of 1 KB rows per group: visited, and one frontier per level up to 5; later levels reuse two of
  * them) plus 1 KB per 33 edges per group (rows for vertices with more than 32 out-edges) and 16 bytes per

@@ -9,9 +9,10 @@
 // out-neighbours with a shared-memory OR (high-degree vertices are expanded by the whole
 // warp, the rest by their own lane); the newly reached (source, vertex) pairs are then
 // written to the output, lanes holding consecutive vertices so that one warp store fills a
-// contiguous run of one SPD row.  Every output byte is written exactly once (distances when
-// they are discovered, "unreachable" and row padding at the end), so the HBM traffic is the
-// matrix itself plus the CSR.  The frontier / next / visited words live in shared memory
+// contiguous run of one SPD row.  Distances below max_dist are written when they are discovered; at level
+// max_dist everything not reached yet is written as "max_dist or farther" in one pass of full runs, the later
+// levels only push, and "unreachable" (overwriting those bytes) and row padding follow at the end: every byte is
+// written once, unreachable pairs of graphs deeper than max_dist twice, so the HBM traffic is the matrix plus the CSR.  The frontier / next / visited words live in shared memory
 // when 12 bytes per vertex fit, otherwise in an L2-resident slice of the workspace (batches with a
 // graph beyond that size); a single graph beyond that size takes the bit-matrix build further down.
 #include "gt_common.cuh"
@@ -32,6 +33,8 @@ struct SpdParams {
     int32_t* batch_start;         // [G+1] prefix sum of ceil(n_g/32)
     uint32_t* scratch;            // global state slices (only when !kSmemState)
     size_t scratch_words_per_cta;
+    int32_t* comp;                // [n_total] connected component of a node (smallest local id in it); valid where sym[g] != 0
+    int32_t* sym;                 // [G] the graph is undirected (every edge has its reverse) and comp is filled in
     int32_t n_total;
     int32_t n_graphs;
     int32_t max_dist;
@@ -70,11 +73,68 @@ __global__ void spd_setup_kernel(SpdParams p)
     }
 }
 
+// Undirected graphs that are deeper than max_dist: beyond level max_dist only "reachable or not" is left to decide,
+// and in an undirected graph that is "same connected component or not".  One CTA per graph checks that every edge
+// has its reverse (graphs with a vertex of more than kMaxSymDegree out-edges are not examined: the check costs
+// deg^2 loads per vertex, and graphs with hubs are shallow anyway) and labels the components by min-label
+// propagation with pointer jumping in shared memory.  The BFS then stops at level max_dist for such a graph.
+constexpr int kMaxSymDegree = 64;
+constexpr int kCompThreads = 512;
+
+__global__ void __launch_bounds__(kCompThreads) spd_components_kernel(SpdParams p, int32_t max_labels)
+{
+    extern __shared__ int32_t lab[];
+    const int g = blockIdx.x;
+    const int32_t node0 = p.cu_seqlens ? p.cu_seqlens[g] : 0;
+    const int32_t n_g = p.cu_seqlens ? p.cu_seqlens[g + 1] - node0 : p.n_total;
+    const int32_t* rp = p.row_ptr + node0;
+    int bad = n_g > max_labels;
+    for (int v = threadIdx.x; v < n_g && !bad; v += blockDim.x)
+        if (rp[v + 1] - rp[v] > kMaxSymDegree) bad = 1;
+    if (__syncthreads_or(bad)) {
+        if (threadIdx.x == 0) p.sym[g] = 0;
+        return;
+    }
+    for (int v = threadIdx.x; v < n_g; v += blockDim.x) {
+        lab[v] = v;
+        for (int e = rp[v]; e < rp[v + 1] && !bad; ++e) {
+            const int w = p.col_idx[e] - node0;
+            bool found = false;
+            for (int e2 = rp[w]; e2 < rp[w + 1]; ++e2) found |= (p.col_idx[e2] - node0 == v);
+            if (!found) bad = 1;
+        }
+    }
+    if (__syncthreads_or(bad)) {
+        if (threadIdx.x == 0) p.sym[g] = 0;
+        return;
+    }
+    // Labels are local vertex ids and only ever decrease; lab[v] always names a vertex of v's component.  Only the
+    // owner of v writes lab[v]; reads of other entries may see the old or the new value, both are valid labels.
+    for (;;) {
+        int changed = 0;
+        for (int v = threadIdx.x; v < n_g; v += blockDim.x) {
+            const int old = lab[v];
+            int m = old;
+            for (int e = rp[v]; e < rp[v + 1]; ++e) m = min(m, lab[p.col_idx[e] - node0]);
+            if (m < old) { lab[v] = m; changed = 1; }
+        }
+        __syncthreads();
+        for (int it = 0; it < 3; ++it) {
+            for (int v = threadIdx.x; v < n_g; v += blockDim.x) lab[v] = lab[lab[v]];
+            __syncthreads();
+        }
+        if (!__syncthreads_or(changed)) break;
+    }
+    for (int v = threadIdx.x; v < n_g; v += blockDim.x) p.comp[node0 + v] = lab[v];
+    if (threadIdx.x == 0) p.sym[g] = 1;
+}
+
 template <bool kSmemState>
 __global__ void __launch_bounds__(1024, kSmemState ? 1 : 2) spd_bfs_kernel(SpdParams p)
 {
     extern __shared__ uint32_t smem_words[];
     __shared__ int32_t s_batch;
+    __shared__ int32_t s_src_comp[kSrcPerBatch];
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -111,6 +171,9 @@ __global__ void __launch_bounds__(1024, kSmemState ? 1 : 2) spd_bfs_kernel(SpdPa
         uint32_t* nxt = cur + n_g;
         uint32_t* vis = nxt + n_g;
 
+        const bool undirected = p.sym[g] != 0;
+        const int32_t* comp = p.comp + node0;
+        if (undirected && threadIdx.x < n_src) s_src_comp[threadIdx.x] = comp[s0 + threadIdx.x];
         for (int v = threadIdx.x; v < n_g; v += blockDim.x) {
             uint32_t f = (v >= s0 && v < s0 + n_src) ? (1u << (v - s0)) : 0u;
             cur[v] = f;
@@ -120,8 +183,45 @@ __global__ void __launch_bounds__(1024, kSmemState ? 1 : 2) spd_bfs_kernel(SpdPa
         __syncthreads();
 
         const int32_t* rp = p.row_ptr + node0;
+        bool done_early = false;
         for (int level = 0;; ++level) {
             const uint8_t code = (uint8_t)min(level, p.max_dist);
+            // From level max_dist on every newly reached pair gets the same code, so the levels are no longer told apart:
+            // all pairs not reached before this level are written now, a run of one row per warp store, as "max_dist or
+            // farther"; the remaining levels only push, and the pairs they never reach are overwritten at the end.
+            const bool emit = level < p.max_dist;
+            if (level == p.max_dist) {
+                if (undirected) {
+                    // the rest of the block at once: same component = "max_dist or farther", else unreachable; row padding
+                    for (int vb = warp * 32; vb < (int)ld; vb += n_warps * 32) {
+                        const int v = vb + lane;
+                        uint32_t m = 0u;
+                        int32_t cv = -1;
+                        if (v < n_g) { m = (~vis[v] | cur[v]) & src_mask; cv = comp[v]; }
+                        else if (v < ld) m = src_mask;
+                        uint32_t uni = __reduce_or_sync(0xffffffffu, m);
+                        while (uni) {
+                            const int b = __ffs(uni) - 1;
+                            uni &= uni - 1;
+                            if ((m >> b) & 1u)
+                                out0[(int64_t)b * ld + v] = v >= n_g ? (uint8_t)255 : (s_src_comp[b] == cv ? code : (uint8_t)(p.max_dist + 1));
+                        }
+                    }
+                    done_early = true;
+                    break;
+                }
+                for (int vb = warp * 32; vb < n_g; vb += n_warps * 32) {
+                    const int v = vb + lane;
+                    uint32_t m = 0u;
+                    if (v < n_g) m = (~vis[v] | cur[v]) & src_mask;
+                    uint32_t uni = __reduce_or_sync(0xffffffffu, m);
+                    while (uni) {
+                        const int b = __ffs(uni) - 1;
+                        uni &= uni - 1;
+                        if ((m >> b) & 1u) out0[(int64_t)b * ld + v] = code;
+                    }
+                }                       // (the final pass, which overwrites some of these bytes, is behind this level's barriers)
+            }
             // ---- emit newly reached pairs and push the frontier ----
             for (int vb = warp * 32; vb < n_g; vb += n_warps * 32) {
                 const int v = vb + lane;
@@ -138,7 +238,8 @@ __global__ void __launch_bounds__(1024, kSmemState ? 1 : 2) spd_bfs_kernel(SpdPa
                 // bits, the warp many different ones): every lane walks its own bits, a few rounds instead of one per
                 // source that occurs in the warp.
                 const int own_rounds = (int)__reduce_max_sync(0xffffffffu, (unsigned)__popc(f));
-                if (__popc(uni) > 2 * own_rounds) {
+                if (!emit) {
+                } else if (__popc(uni) > 2 * own_rounds) {
                     uint32_t mine = f;
                     for (int k = 0; k < own_rounds; ++k) {
                         if (mine) {
@@ -212,7 +313,7 @@ __global__ void __launch_bounds__(1024, kSmemState ? 1 : 2) spd_bfs_kernel(SpdPa
 
         // ---- unreachable pairs and row padding ----
         const uint8_t unreach = (uint8_t)(p.max_dist + 1);
-        for (int vb = warp * 32; vb < (int)ld; vb += n_warps * 32) {
+        for (int vb = warp * 32; vb < (int)ld && !done_early; vb += n_warps * 32) {
             const int v = vb + lane;
             uint32_t m = 0u;
             uint8_t val = unreach;
@@ -698,6 +799,8 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
 // Test hook (gt_test_hook_barrier_overcount): consumed by the next bit-matrix build of this process.
 uint32_t g_barrier_overcount = 0;
 
+// labels of the component pre-pass: one shared-memory word per vertex of the largest graph, at most 200 KB (larger graphs skip it)
+int32_t b_max_labels(int32_t max_seqlen) { return max_seqlen < 50 * 1024 ? max_seqlen : 50 * 1024; }
 size_t spd_state_bytes(int32_t max_seqlen) { return (size_t)3 * (size_t)max_seqlen * sizeof(uint32_t); }
 constexpr size_t kSmemStateLimit = 200 * 1024;
 constexpr int32_t kDenseMinNodes = 14500;
@@ -711,7 +814,7 @@ struct SpdPlan {
     int threads;
     int grid;
     size_t smem_bytes;
-    size_t batch_start_off, scratch_off, scratch_words_per_cta, total_bytes;
+    size_t batch_start_off, scratch_off, scratch_words_per_cta, comp_off, sym_off, total_bytes;
 };
 
 SpdPlan make_plan(const gt_batch* b, int64_t nnz)
@@ -735,7 +838,9 @@ SpdPlan make_plan(const gt_batch* b, int64_t nnz)
     pl.batch_start_off = kHeaderBytes;
     pl.scratch_off = align_up(pl.batch_start_off + sizeof(int32_t) * ((size_t)b->n_graphs + 1), 256);
     pl.scratch_words_per_cta = pl.smem_state ? 0 : align_up((size_t)3 * b->max_seqlen, 64);
-    pl.total_bytes = pl.scratch_off + pl.scratch_words_per_cta * sizeof(uint32_t) * (size_t)pl.grid;
+    pl.comp_off = align_up(pl.scratch_off + pl.scratch_words_per_cta * sizeof(uint32_t) * (size_t)pl.grid, 256);
+    pl.sym_off = align_up(pl.comp_off + sizeof(int32_t) * (size_t)b->n_total, 256);
+    pl.total_bytes = pl.sym_off + sizeof(int32_t) * (size_t)b->n_graphs;
     pl.dense = false;
     // A single graph takes the bit-matrix build from kDenseMinNodes up: measured on power-law graphs of average degree 12 it
     // overtakes the multi-source BFS between 14 000 and 15 000 nodes (16 384 nodes: 0.98 against 1.65 ms), before the BFS
@@ -848,6 +953,16 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
         void* args[] = {(void*)&p, (void*)&d};
         GT_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)spd_dense_kernel, dim3((unsigned)pl.grid), dim3((unsigned)pl.threads), args, 0, s));
         return GT_OK;
+    }
+    {
+        p.comp = (int32_t*)(ws + pl.comp_off);
+        p.sym = (int32_t*)(ws + pl.sym_off);
+        const int32_t max_labels = b_max_labels(batch->max_seqlen);
+        const size_t lab_bytes = sizeof(int32_t) * (size_t)max_labels;
+        if (lab_bytes > 48 * 1024)
+            GT_CUDA_TRY(cudaFuncSetAttribute(spd_components_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lab_bytes));
+        spd_components_kernel<<<(unsigned)batch->n_graphs, kCompThreads, lab_bytes, s>>>(p, max_labels);
+        GT_CUDA_TRY(cudaGetLastError());
     }
     if (pl.smem_state) {
         GT_CUDA_TRY(cudaFuncSetAttribute(spd_bfs_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem_bytes));

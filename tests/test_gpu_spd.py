@@ -53,6 +53,60 @@ def test_directed_cycle():
     np.testing.assert_array_equal(got, (j - i) % n)
 
 
+def _csr(n, src, dst):
+    """CSR exactly as given (no symmetrisation, duplicates and self loops kept)."""
+    src, dst = np.asarray(src, np.int64), np.asarray(dst, np.int64)
+    order = np.lexsort((dst, src))
+    rp = np.zeros(n + 1, np.int32)
+    np.add.at(rp, src + 1, 1)
+    return np.cumsum(rp).astype(np.int32), dst[order].astype(np.int32)
+
+
+def _both_ways(edges):
+    e = np.array(edges, np.int64).reshape(-1, 2)
+    return np.concatenate([e[:, 0], e[:, 1]]), np.concatenate([e[:, 1], e[:, 0]])
+
+
+def test_undirected_graphs_deeper_than_max_dist_stop_at_the_clip_level():
+    """Beyond level max_dist an undirected graph only needs "same component or not".  One packed batch with: three
+    paths of different lengths in one graph (far pairs, unreachable pairs), a grid, the same paths with duplicate
+    edges and self loops, a directed chain (no reverse edges: the full search), the paths with ONE reverse edge
+    missing (must not be taken for undirected: nodes behind the one-way edge reach forward only), and a deep
+    graph with a hub of 80 leaves (beyond the degree up to which the reverse edges are checked)."""
+    D = 6
+    paths = [(i, i + 1) for i in range(0, 149)] + [(i, i + 1) for i in range(150, 199)] + [(i, i + 1) for i in range(200, 229)]
+    g_paths = _csr(230, *_both_ways(paths))
+    side = 23
+    grid = [(r * side + c, r * side + c + 1) for r in range(side) for c in range(side - 1)] + \
+           [(r * side + c, (r + 1) * side + c) for r in range(side - 1) for c in range(side)]
+    g_grid = _csr(side * side, *_both_ways(grid))
+    s, d = _both_ways(paths + paths[:40])
+    g_dups = _csr(230, np.concatenate([s, np.arange(0, 230, 7)]), np.concatenate([d, np.arange(0, 230, 7)]))
+    g_chain = _csr(120, np.arange(119), np.arange(1, 120))
+    s, d = _both_ways(paths)
+    keep = ~((s == 60) & (d == 59))
+    g_oneway = _csr(230, s[keep], d[keep])
+    hub = [(i, i + 1) for i in range(0, 99)] + [(50, 100 + j) for j in range(80)]
+    g_hub = _csr(180, *_both_ways(hub))
+    w = wl.Workload("deep", wl.pack_graphs([g_paths, g_grid, g_dups, g_chain, g_oneway, g_hub]), 1, 32, D)
+    got = check(w)
+    b = w.batch
+    first = got[: b.spd_offsets[1]].reshape(230, -1)[:, :230]
+    i, j = np.indices((230, 230))
+    block = lambda x: np.where(x < 150, 0, np.where(x < 200, 1, 2))
+    np.testing.assert_array_equal(first, np.where(block(i) == block(j), np.minimum(np.abs(i - j), D), D + 1))
+    a = b.spd_offsets[4]
+    oneway = got[a: a + 230 * 240].reshape(230, 240)[:, :230]
+    assert oneway[70, 10] == D + 1 and oneway[10, 70] == D and oneway[61, 60] == 1 and oneway[60, 59] == D + 1
+
+
+@pytest.mark.parametrize("n,D", [(3000, 3), (5000, 12)])
+def test_deep_undirected_single_graph(n, D):
+    """Random geometric graph near its connectivity threshold: many levels, several components."""
+    w = wl.Workload("rgg", wl.pack_graphs([wl.random_geometric(n, 5.0, 11)]), 1, 32, D)
+    check(w)
+
+
 def test_star_hub_uses_warp_expansion():
     n = 600                                     # hub degree 599 > the per-lane expansion limit
     w = closed_form_workload(n, [(0, j) for j in range(1, n)], D=4)
