@@ -257,16 +257,25 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
                 } else {
                     // packed batch (per-graph pitch): cp.async in the layout of the TMA 128-byte swizzle,
                     // 16-byte chunk c of row r at chunk c ^ (r & 7)
+                    // (a lane copies chunk cc of rows lr, lr + 4, ...: the swizzle depends on the parity of the round only)
                     const int32_t q0 = q_lo + i * kTile;
                     const uint32_t dst0 = smem_u32(smem + L::kSpd);
-#pragma unroll 4
-                    for (int it = 0; it < (kTile * 8) / 32; ++it) {
-                        const int c = it * 32 + lane;
-                        const int r = c >> 3, cc = c & 7;
-                        const int64_t col = (int64_t)q0 + cc * 16;
-                        const bool valid = (kv0 + r < n_g) && (col < ld);
-                        const uint8_t* src = valid ? spd_g + (int64_t)(kv0 + r) * ld + col : spd_g;
-                        cp_async_16(dst0 + r * 128 + ((cc ^ (r & 7)) << 4), src, valid ? 16u : 0u);
+                    const int cc = lane & 7, lr = lane >> 3;
+                    const uint32_t dst_even = dst0 + (uint32_t)(lr * 128 + ((cc ^ lr) << 4)), dst_odd = dst0 + (uint32_t)(lr * 128 + ((cc ^ (4 + lr)) << 4));
+                    const uint32_t step = 4u * (uint32_t)ld;
+                    const uint8_t* src = spd_g + (int64_t)(kv0 + lr) * ld + q0 + cc * 16;
+                    const int32_t lim = ((int64_t)q0 + cc * 16 < ld) ? n_g - kv0 - lr : 0;       // rounds 4 it < lim are in range
+                    if (kv0 + kTile <= n_g && (int64_t)q0 + kTile <= ld) {
+#pragma unroll 8
+                        for (int it = 0; it < kTile / 4; ++it) {
+                            cp_async_16(((it & 1) ? dst_odd : dst_even) + it * 512, src + (uint64_t)step * (uint32_t)it, 16u);
+                        }
+                    } else {
+#pragma unroll 8
+                        for (int it = 0; it < kTile / 4; ++it) {
+                            const bool valid = 4 * it < lim;
+                            cp_async_16(((it & 1) ? dst_odd : dst_even) + it * 512, valid ? src + (uint64_t)step * (uint32_t)it : spd_g, valid ? 16u : 0u);
+                        }
                     }
                     cp_async_mbar_arrive_noinc(bar(kBarSpdFull));
                 }

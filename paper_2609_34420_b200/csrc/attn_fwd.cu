@@ -307,20 +307,31 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             }
         } else if (!p.spd_tma) {
             // ---- warp 2: SPD tile loader for packed batches ----
+            // A lane copies 16-byte chunk cc of rows lr, lr + 4, ...; the 128-byte swizzle (chunk c of row r at c ^ (r & 7))
+            // depends on the parity of the round only, so both shared-memory offsets and the source pointer are
+            // formed once and a copy costs the instruction itself plus one multiply-add for its address.
+            const int cc = lane & 7, lr = lane >> 3;
+            const uint32_t dst_even = (uint32_t)(lr * 128 + ((cc ^ lr) << 4)), dst_odd = (uint32_t)(lr * 128 + ((cc ^ (4 + lr)) << 4));
+            const uint8_t* lane_src = spd_g + (int64_t)(q0 + lr) * ld + cc * 16;
+            const uint32_t step = 4u * (uint32_t)ld;      // every copy's address is base + (constant round) * step: no dependent chain
+            const int32_t rows_valid = min(kRowsPerCta, n_g - q0);
             for (int j = 0; j < n_kv; ++j) {
                 const int s2 = j % kSpdStages;
                 mbar_wait(bar(kBarSpdEmpty + s2), ((j / kSpdStages) & 1) ^ 1, abort_flag, p.status, 30);
                 const int32_t kv0 = kv_begin + j * kKvTile;
                 const uint32_t dst0 = smem_u32(smem + L::kSpd + s2 * L::kSpdTileBytes);
-                const int cc = lane & 7;
-                const int64_t col = (int64_t)kv0 + cc * 16;
-                const bool col_ok = col < ld;
-#pragma unroll 4
-                for (int i = 0; i < 64; ++i) {
-                    const int r = i * 4 + (lane >> 3);
-                    const bool valid = col_ok && (q0 + r < n_g);
-                    const uint8_t* src = valid ? spd_g + (int64_t)(q0 + r) * ld + col : spd_g;
-                    cp_async_16(dst0 + r * 128 + ((cc ^ (r & 7)) << 4), src, valid ? 16u : 0u);
+                const uint8_t* src = lane_src + kv0;
+                if (rows_valid == kRowsPerCta && (int64_t)kv0 + kKvTile <= ld) {
+#pragma unroll 16
+                    for (int i = 0; i < kRowsPerCta / 4; ++i)
+                        cp_async_16(dst0 + i * 512 + ((i & 1) ? dst_odd : dst_even), src + (uint64_t)step * (uint32_t)i, 16u);
+                } else {
+                    const int32_t lim = ((int64_t)kv0 + cc * 16 < ld) ? rows_valid - lr : 0;     // rounds 4 i < lim are in range
+#pragma unroll 8
+                    for (int i = 0; i < kRowsPerCta / 4; ++i) {
+                        const bool valid = 4 * i < lim;
+                        cp_async_16(dst0 + i * 512 + ((i & 1) ? dst_odd : dst_even), valid ? src + (uint64_t)step * (uint32_t)i : spd_g, valid ? 16u : 0u);
+                    }
                 }
                 cp_async_mbar_arrive_noinc(bar(kBarSpdFull + s2));
             }
