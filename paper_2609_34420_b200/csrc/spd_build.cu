@@ -81,26 +81,43 @@ __global__ void spd_setup_kernel(SpdParams p)
 constexpr int kMaxSymDegree = 64;
 constexpr int kCompThreads = 512;
 
-__global__ void __launch_bounds__(kCompThreads) spd_components_kernel(SpdParams p, int32_t max_labels)
+__global__ void __launch_bounds__(kCompThreads) spd_components_kernel(SpdParams p, int32_t smem_words)
 {
-    extern __shared__ int32_t lab[];
+    extern __shared__ int32_t comp_smem[];
     const int g = blockIdx.x;
     const int32_t node0 = p.cu_seqlens ? p.cu_seqlens[g] : 0;
     const int32_t n_g = p.cu_seqlens ? p.cu_seqlens[g + 1] - node0 : p.n_total;
-    const int32_t* rp = p.row_ptr + node0;
-    int bad = n_g > max_labels;
+    const int32_t* grp = p.row_ptr + node0;
+    const int32_t e_base = grp[0];
+    const int64_t nnz_g = (int64_t)grp[n_g] - e_base;
+    int bad = n_g > smem_words;
     for (int v = threadIdx.x; v < n_g && !bad; v += blockDim.x)
-        if (rp[v + 1] - rp[v] > kMaxSymDegree) bad = 1;
+        if (grp[v + 1] - grp[v] > kMaxSymDegree) bad = 1;
     if (__syncthreads_or(bad)) {
         if (threadIdx.x == 0) p.sym[g] = 0;
         return;
     }
-    for (int v = threadIdx.x; v < n_g; v += blockDim.x) {
-        lab[v] = v;
+    // labels, and the graph's CSR with local ids when it fits next to them (it is walked deg times per vertex by the
+    // reverse-edge check and once per round of the labelling)
+    int32_t* lab = comp_smem;
+    const bool staged = (int64_t)2 * n_g + 1 + nnz_g <= (int64_t)smem_words;
+    const int32_t* rp = grp;
+    const int32_t* ci = p.col_idx;
+    int32_t sub = node0;                        // subtracted from a column index to make it local
+    if (staged) {
+        int32_t* srp = comp_smem + n_g;
+        int32_t* sci = srp + n_g + 1;
+        for (int v = threadIdx.x; v <= n_g; v += blockDim.x) srp[v] = grp[v] - e_base;
+        for (int e = threadIdx.x; e < (int)nnz_g; e += blockDim.x) sci[e] = p.col_idx[e_base + e] - node0;
+        rp = srp; ci = sci; sub = 0;
+    }
+    for (int v = threadIdx.x; v < n_g; v += blockDim.x) lab[v] = v;
+    __syncthreads();
+    for (int v = threadIdx.x; v < n_g && !bad; v += blockDim.x) {
         for (int e = rp[v]; e < rp[v + 1] && !bad; ++e) {
-            const int w = p.col_idx[e] - node0;
+            const int w = ci[e] - sub;
             bool found = false;
-            for (int e2 = rp[w]; e2 < rp[w + 1]; ++e2) found |= (p.col_idx[e2] - node0 == v);
+            for (int e2 = rp[w]; e2 < rp[w + 1]; ++e2) found |= (ci[e2] - sub == v);
             if (!found) bad = 1;
         }
     }
@@ -110,18 +127,15 @@ __global__ void __launch_bounds__(kCompThreads) spd_components_kernel(SpdParams 
     }
     // Labels are local vertex ids and only ever decrease; lab[v] always names a vertex of v's component.  Only the
     // owner of v writes lab[v]; reads of other entries may see the old or the new value, both are valid labels.
+    // A round with no change by any thread read stable values, so it proves the fixed point: one label per component.
     for (;;) {
         int changed = 0;
         for (int v = threadIdx.x; v < n_g; v += blockDim.x) {
             const int old = lab[v];
             int m = old;
-            for (int e = rp[v]; e < rp[v + 1]; ++e) m = min(m, lab[p.col_idx[e] - node0]);
+            for (int e = rp[v]; e < rp[v + 1]; ++e) m = min(m, lab[ci[e] - sub]);
+            m = lab[lab[lab[m]]];               // pointer jumping: the label's own label, three steps
             if (m < old) { lab[v] = m; changed = 1; }
-        }
-        __syncthreads();
-        for (int it = 0; it < 3; ++it) {
-            for (int v = threadIdx.x; v < n_g; v += blockDim.x) lab[v] = lab[lab[v]];
-            __syncthreads();
         }
         if (!__syncthreads_or(changed)) break;
     }
@@ -799,8 +813,7 @@ __global__ void __launch_bounds__(512, 2) spd_dense_kernel(SpdParams p, DensePar
 // Test hook (gt_test_hook_barrier_overcount): consumed by the next bit-matrix build of this process.
 uint32_t g_barrier_overcount = 0;
 
-// labels of the component pre-pass: one shared-memory word per vertex of the largest graph, at most 200 KB (larger graphs skip it)
-int32_t b_max_labels(int32_t max_seqlen) { return max_seqlen < 50 * 1024 ? max_seqlen : 50 * 1024; }
+constexpr size_t kCompSmemBytes = 200 * 1024;     // shared memory of the component pre-pass (graphs whose labels do not fit skip it)
 size_t spd_state_bytes(int32_t max_seqlen) { return (size_t)3 * (size_t)max_seqlen * sizeof(uint32_t); }
 constexpr size_t kSmemStateLimit = 200 * 1024;
 constexpr int32_t kDenseMinNodes = 14500;
@@ -957,8 +970,10 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
     {
         p.comp = (int32_t*)(ws + pl.comp_off);
         p.sym = (int32_t*)(ws + pl.sym_off);
-        const int32_t max_labels = b_max_labels(batch->max_seqlen);
-        const size_t lab_bytes = sizeof(int32_t) * (size_t)max_labels;
+        // room for the labels of the largest graph and, if it is not much more, for a graph's CSR beside them
+        const size_t want = sizeof(int32_t) * ((size_t)batch->max_seqlen * (2 + 16) + 1);
+        const size_t lab_bytes = want < kCompSmemBytes ? want : kCompSmemBytes;
+        const int32_t max_labels = (int32_t)(lab_bytes / sizeof(int32_t));
         if (lab_bytes > 48 * 1024)
             GT_CUDA_TRY(cudaFuncSetAttribute(spd_components_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lab_bytes));
         spd_components_kernel<<<(unsigned)batch->n_graphs, kCompThreads, lab_bytes, s>>>(p, max_labels);
