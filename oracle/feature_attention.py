@@ -23,6 +23,15 @@ memory.  One graph per call (a packed batch is a loop over graphs with dW summed
 Pinned by tests against torch autograd in fp64 through an einsum-built dense bias, central finite
 differences on W, the reduction to the bucket form when f is the one-hot code of a distance matrix, and
 the identity sum_c dW[h,c] * u[c] = 0 when every pair's features satisfy f . u = const.
+
+Categorical features (few distinct feature vectors, as structural encodings are): the feature form IS a bucket
+form.  With the distinct 4-vectors numbered c = 0..n_codes-1,
+
+    b_attn[h,i,j] = table[h, code[i,j]],  table[h,c] = sum_x W[h,x] * vec[c,x],   dW[h,x] = sum_c dTable[h,c] * vec[c,x]
+
+exactly (same sums, regrouped).  encode_features / code_table / weights_gradient_from_table write that out; they
+are pinned by the round trip vec[code] == f, by table[code] == feature_bias, and by dW through the codes equalling
+backward_feature's dW.
 """
 from __future__ import annotations
 
@@ -80,3 +89,25 @@ def backward_feature(q: np.ndarray, k: np.ndarray, v: np.ndarray, dout: np.ndarr
             dk[:, h, :] += (ds.T @ q[r0:r1, h, :]) * inv_sqrt_d
             dw[h] += np.tensordot(ds, ff, axes=([0, 1], [0, 1]))
     return dq, dk, dv, dw
+
+
+def encode_features(f: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """f uint8 [n,n,4] -> (code int64 [n,n], vec uint8 [n_codes,4]).  Codes number the distinct feature vectors in
+    ascending order of the 32-bit word f0 + 256 f1 + 65536 f2 + 16777216 f3."""
+    n = f.shape[0]
+    assert f.shape == (n, n, 4) and f.dtype == np.uint8
+    word = (f[..., 0].astype(np.uint32) | (f[..., 1].astype(np.uint32) << 8) |
+            (f[..., 2].astype(np.uint32) << 16) | (f[..., 3].astype(np.uint32) << 24))
+    distinct, inverse = np.unique(word.reshape(-1), return_inverse=True)
+    vec = np.stack([(distinct >> (8 * x)) & 0xff for x in range(4)], axis=1).astype(np.uint8)
+    return inverse.reshape(n, n).astype(np.int64), vec
+
+
+def code_table(w: np.ndarray, vec: np.ndarray) -> np.ndarray:
+    """table[h,c] = sum_x w[h,x] * vec[c,x]; w fp64 [H,4], vec uint8 [n_codes,4]."""
+    return w @ vec.astype(np.float64).T
+
+
+def weights_gradient_from_table(dtable: np.ndarray, vec: np.ndarray) -> np.ndarray:
+    """dW[h,x] = sum_c dtable[h,c] * vec[c,x]."""
+    return dtable @ vec.astype(np.float64)

@@ -105,3 +105,46 @@ def test_transposed_features_are_not_interchangeable():
     o, _ = ofeat.forward_feature(q, k, v, f, w)
     ot, _ = ofeat.forward_feature(q, k, v, np.ascontiguousarray(f.transpose(1, 0, 2)), w)
     assert np.abs(o - ot).max() > 1e-3
+
+
+def categorical_features(n, n_vec, seed):
+    rng = np.random.Generator(np.random.PCG64(seed))
+    vec = rng.integers(0, 256, size=(n_vec, 4), dtype=np.uint8)
+    return vec[rng.integers(0, n_vec, size=(n, n))]
+
+
+def test_codes_round_trip_and_are_numbered_by_ascending_word():
+    f = categorical_features(37, 9, 3)
+    code, vec = ofeat.encode_features(f)
+    np.testing.assert_array_equal(vec[code], f)
+    word = vec.astype(np.uint64) @ np.array([1, 256, 65536, 16777216], dtype=np.uint64)
+    assert (np.diff(word.astype(np.int64)) > 0).all() and len(vec) <= 9
+    # a hand-made case: three distinct vectors, the order decided by the LAST feature first
+    g = np.zeros((2, 2, 4), np.uint8)
+    g[0, 0] = (9, 0, 0, 0); g[0, 1] = (0, 0, 0, 1); g[1, 0] = (0, 1, 0, 0); g[1, 1] = (9, 0, 0, 0)
+    code, vec = ofeat.encode_features(g)
+    np.testing.assert_array_equal(code, [[0, 2], [1, 0]])
+    np.testing.assert_array_equal(vec, [[9, 0, 0, 0], [0, 1, 0, 0], [0, 0, 0, 1]])
+
+
+def test_the_code_form_is_the_feature_form_regrouped():
+    """table[code] is the feature bias, and dW through the codes (the bucket oracle's scatter, then the contraction
+    with the vectors) is backward_feature's dW."""
+    from oracle import attention as oattn
+    n, H, d = 41, 3, 8
+    rng = np.random.Generator(np.random.PCG64(5))
+    q, k, v, do = (rng.standard_normal((n, H, d)) for _ in range(4))
+    w = rng.standard_normal((H, 4)) * 0.02
+    f = categorical_features(n, 11, 8)
+    code, vec = ofeat.encode_features(f)
+    table = ofeat.code_table(w, vec)
+    for h in range(H):
+        np.testing.assert_allclose(table[h][code], ofeat.feature_bias(f, w[h]), rtol=0, atol=1e-12)
+    o1, l1 = ofeat.forward_feature(q, k, v, f, w)
+    o2, l2 = oattn.forward_single(q, k, v, code, table)
+    np.testing.assert_allclose(o2, o1, atol=1e-12)
+    np.testing.assert_allclose(l2, l1, atol=1e-12)
+    dq1, dk1, dv1, dw1 = ofeat.backward_feature(q, k, v, do, f, w)
+    dq2, dk2, dv2, dt = oattn.backward_single(q, k, v, do, code, table)
+    np.testing.assert_allclose(dq2, dq1, atol=1e-11)
+    np.testing.assert_allclose(ofeat.weights_gradient_from_table(dt, vec), dw1, atol=1e-9)
