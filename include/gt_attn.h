@@ -366,6 +366,38 @@ gt_status gt_feature_attn_bwd(const void* q, const void* k, const void* v, const
                               void* dq, void* dk, void* dv, float* dweights,
                               void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------------------
+ * gt_feature_encode, gt_feature_code_table, gt_feature_code_dweights -- the feature bias above through the
+ * tensor-core kernels of the bucket form, for CATEGORICAL features: when the node pairs of a graph carry at most 256
+ * distinct feature vectors, numbering them c = 0..n_codes-1 gives, exactly (the same sums regrouped),
+ *     sum_x weights[h][x] features[i][j][x] = table[h][code[i][j]],   table[h][c] = sum_x weights[h][x] vectors[c][x],
+ *     dweights[h][x] = sum_c dtable[h][c] vectors[c][x],
+ * so gt_biased_attn_fwd / gt_biased_attn_bwd (and their _ex, chunked and step forms) run on `codes` in place of the
+ * SPD matrix, with max_dist = max(n_codes, 3) - 2 and `table` / `dtable` in place of bias / dbias.
+ *
+ * gt_feature_encode (once per batch, like gt_spd_build): features uint8 [N,N,4] (device, 4-byte aligned) -> codes
+ * (device uint8, N rows of pitch N rounded up to 16, padding 255: the SPD layout of a single graph) and vectors
+ * (device uint32 [256]: vectors[c] = features of code c as f0 + 256 f1 + 65536 f2 + 16777216 f3, zero beyond
+ * n_codes).  Codes follow the ascending order of that word, so the result is deterministic.  Single graph only
+ * (else GT_ERR_UNSUPPORTED).  With more than 256 distinct vectors the status word of `workspace` is set to
+ * GT_ERR_UNSUPPORTED (reported by gt_check), `codes` is left unwritten and the caller falls back to
+ * gt_feature_attn_fwd / _bwd.  Workspace: gt_feature_encode_workspace() bytes (about 41 KB), header zeroed by the
+ * caller before first use.  gt_feature_encode_count synchronises the stream and returns the number of distinct
+ * vectors found (it can exceed 256 when the encoding was given up).
+ *
+ * gt_feature_code_table: weights fp32 [n_heads,4] -> table fp32 [n_heads, n_codes] (1 <= n_codes <= 256; codes beyond
+ * the ones found get 0).  gt_feature_code_dweights: dtable fp32 [n_heads, n_codes] -> dweights fp32 [n_heads,4]
+ * (overwritten; fp64 sums).  Both take device pointers, launch one small kernel on `stream` and keep no state.
+ * ------------------------------------------------------------------------------------- */
+size_t gt_feature_encode_workspace(void);
+gt_status gt_feature_encode(const uint8_t* features, const gt_batch* batch, uint8_t* codes, uint32_t* vectors,
+                            void* workspace, size_t workspace_bytes, void* stream);
+gt_status gt_feature_encode_count(void* workspace, void* stream, int32_t* n_codes_host);
+gt_status gt_feature_code_table(const float* weights, const uint32_t* vectors, int32_t n_heads, int32_t n_codes,
+                                float* table, void* stream);
+gt_status gt_feature_code_dweights(const float* dtable, const uint32_t* vectors, int32_t n_heads, int32_t n_codes,
+                                   float* dweights, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -31,7 +31,9 @@ EXPORTS = ("gt_status_string", "gt_check",
            "gt_biased_attn_fwd_step_workspace", "gt_biased_attn_fwd_step",
            "gt_biased_attn_bwd_step_context_bytes", "gt_biased_attn_bwd_step_prepare", "gt_biased_attn_bwd_step_prepare_ex",
            "gt_biased_attn_bwd_step", "gt_biased_attn_bwd_step_finish",
-           "gt_feature_attn_fwd", "gt_feature_attn_bwd_workspace", "gt_feature_attn_bwd")
+           "gt_feature_attn_fwd", "gt_feature_attn_bwd_workspace", "gt_feature_attn_bwd",
+           "gt_feature_encode_workspace", "gt_feature_encode", "gt_feature_encode_count",
+           "gt_feature_code_table", "gt_feature_code_dweights")
 
 
 class GtError(RuntimeError):
@@ -120,6 +122,16 @@ def lib() -> ctypes.CDLL:
         L.gt_feature_attn_bwd_workspace.argtypes = [bp, i32]
         L.gt_feature_attn_bwd.restype = ctypes.c_int
         L.gt_feature_attn_bwd.argtypes = [vp] * 7 + [bp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.gt_feature_encode_workspace.restype = sz
+        L.gt_feature_encode_workspace.argtypes = []
+        L.gt_feature_encode.restype = ctypes.c_int
+        L.gt_feature_encode.argtypes = [vp, bp, vp, vp, vp, sz, vp]
+        L.gt_feature_encode_count.restype = ctypes.c_int
+        L.gt_feature_encode_count.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32)]
+        L.gt_feature_code_table.restype = ctypes.c_int
+        L.gt_feature_code_table.argtypes = [vp, vp, i32, i32, vp, vp]
+        L.gt_feature_code_dweights.restype = ctypes.c_int
+        L.gt_feature_code_dweights.argtypes = [vp, vp, i32, i32, vp, vp]
         _lib = L
     return _lib
 
@@ -441,3 +453,32 @@ def gt_profile_bwd_kernel_events(before, after) -> None:
     a, b = arr_t(*[e.cuda_event for e in before]), arr_t(*[e.cuda_event for e in after])
     _profile_keepalive = (a, b, list(before), list(after))
     lib().gt_profile_bwd_kernel_events(a, b, n)
+
+
+def gt_feature_encode(features, batch: Batch, codes, vectors, workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Categorical features uint8 [N, N, 4] -> codes (uint8, N rows of pitch N rounded up to 16) and vectors (int32/uint32 [256])."""
+    if workspace is None:
+        workspace = _workspace(int(lib().gt_feature_encode_workspace()), features.device)
+    b = batch.c_struct()
+    st = lib().gt_feature_encode(_ptr(features), ctypes.byref(b), _ptr(codes), _ptr(vectors), _ptr(workspace),
+                                 workspace.numel(), _stream())
+    _raise(st, "gt_feature_encode")
+    return workspace
+
+
+def gt_feature_encode_count(workspace: torch.Tensor) -> int:
+    """Synchronises; the number of distinct feature vectors the last gt_feature_encode on this workspace found."""
+    c = ctypes.c_int32(0)
+    _raise(lib().gt_feature_encode_count(_ptr(workspace), _stream(), ctypes.byref(c)), "gt_feature_encode_count")
+    return int(c.value)
+
+
+def gt_feature_code_table(weights, vectors, table) -> None:
+    H, n_codes = table.shape
+    _raise(lib().gt_feature_code_table(_ptr(weights), _ptr(vectors), H, n_codes, _ptr(table), _stream()), "gt_feature_code_table")
+
+
+def gt_feature_code_dweights(dtable, vectors, dweights) -> None:
+    H, n_codes = dtable.shape
+    _raise(lib().gt_feature_code_dweights(_ptr(dtable), _ptr(vectors), H, n_codes, _ptr(dweights), _stream()),
+           "gt_feature_code_dweights")

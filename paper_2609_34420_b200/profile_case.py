@@ -1,10 +1,13 @@
 """Run the hot path a few times on one named workload and print CUDA-event timings.
 
     python -m paper_2609_34420_b200.profile_case WORKLOAD [REPS] [spd|fwd|bwd|chunked|all]
+    python -m paper_2609_34420_b200.profile_case featN [REPS] [VECTORS]
 
 WORKLOAD is one of the named workloads (tiny_er256, ba4096, powerlaw16k, powerlaw64k,
 varlen_rgg64) or plN for a power-law graph of N nodes (H=8, d=64, max_dist=24).  A small,
-self-contained timing command line for one entry point at a time.
+self-contained timing command line for one entry point at a time.  featN times the feature-bias
+variant on N nodes (H=8, d=64) with VECTORS distinct feature vectors (default 12): the fp32 path on
+the CUDA cores, and the code matrix through the tensor-core kernels of the bucket form.
 """
 from __future__ import annotations
 
@@ -16,9 +19,71 @@ from . import binding as gt
 from . import workloads as wl
 
 
+def timed_ms(fn, reps):
+    fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def feature_case(n: int, reps: int, n_vec: int) -> int:
+    H, d = 8, 64
+    dev = torch.device("cuda", 0)
+    g = torch.Generator(device=dev).manual_seed(1)
+    q, k, v, do = (torch.randn(n, H, d, device=dev, generator=g).bfloat16() for _ in range(4))
+    wt = torch.randn(H, 4, device=dev, generator=g) * 0.01
+    vec = torch.randint(0, 256, (n_vec, 4), device=dev, generator=g, dtype=torch.uint8)
+    feat = vec[torch.randint(0, n_vec, (n, n), device=dev, generator=g)].contiguous()
+    batch = gt.Batch(n)
+    out, dq, dk, dv = (torch.empty_like(q) for _ in range(4))
+    lse, dw = torch.empty(H, n, device=dev), torch.empty_like(wt)
+    f_fwd, f_bwd = 4.0 * H * d * n * n, 10.0 * H * d * n * n
+    ms = timed_ms(lambda: gt.gt_feature_attn_fwd(q, k, v, feat, wt, batch, out, lse), reps)
+    print(f"feature fwd (CUDA cores) {ms:.3f} ms  {f_fwd / ms / 1e9:.1f} TFLOP/s")
+    ws_b = gt.gt_feature_attn_bwd(q, k, v, do, lse, feat, wt, batch, dq, dk, dv, dw)
+    ms = timed_ms(lambda: gt.gt_feature_attn_bwd(q, k, v, do, lse, feat, wt, batch, dq, dk, dv, dw, ws_b), reps)
+    print(f"feature bwd (CUDA cores) {ms:.3f} ms  {f_bwd / ms / 1e9:.1f} TFLOP/s")
+    gt.gt_check(ws_b)
+    ld = (n + 15) // 16 * 16
+    codes = torch.empty(n * ld, dtype=torch.uint8, device=dev)
+    vectors = torch.empty(256, dtype=torch.int32, device=dev)
+    ws_e = gt.gt_feature_encode(feat, batch, codes, vectors)
+    gt.gt_check(ws_e)
+    width = max(gt.gt_feature_encode_count(ws_e), 3)
+    ms = timed_ms(lambda: gt.gt_feature_encode(feat, batch, codes, vectors, ws_e), reps)
+    print(f"feature encode {ms:.3f} ms  {n * n * 5 / ms / 1e6:.1f} GB/s  ({width} codes)")
+    table, dtable = torch.empty(H, width, device=dev), torch.empty(H, width, device=dev)
+    out32 = torch.empty(n, H, d, device=dev)
+
+    def fwd(ws=None):
+        gt.gt_feature_code_table(wt, vectors, table)
+        return gt.gt_biased_attn_fwd_ex(q, k, v, codes, table, batch, width - 2, out, lse, out32, ws)
+
+    def bwd(ws=None):
+        ws = gt.gt_biased_attn_bwd_ex(q, k, v, out, do, lse, codes, table, batch, width - 2, dq, dk, dv, dtable, out32, ws)
+        gt.gt_feature_code_dweights(dtable, vectors, dw)
+        return ws
+
+    ws_f, ws_bb = fwd(), bwd()
+    ms = timed_ms(lambda: fwd(ws_f), reps)
+    print(f"feature fwd (codes, fp32 output too) {ms:.3f} ms  {f_fwd / ms / 1e9:.1f} TFLOP/s")
+    ms = timed_ms(lambda: bwd(ws_bb), reps)
+    print(f"feature bwd (codes) {ms:.3f} ms  {f_bwd / ms / 1e9:.1f} TFLOP/s")
+    gt.gt_check(ws_f)
+    gt.gt_check(ws_bb)
+    return 0
+
+
 def main(argv) -> int:
     name = argv[1] if len(argv) > 1 else "powerlaw16k"
     reps = int(argv[2]) if len(argv) > 2 else 1
+    if name.startswith("feat") and name[4:].isdigit():
+        return feature_case(int(name[4:]), reps, int(argv[3]) if len(argv) > 3 else 12)
     what = argv[3] if len(argv) > 3 else "all"
     if name.startswith("pl") and name[2:].isdigit():
         w = wl.Workload(name, wl.pack_graphs([wl.chung_lu_power_law(int(name[2:]), 12.0, 2.1, 0)]), 8, 64, 24)
@@ -46,15 +111,7 @@ def main(argv) -> int:
         gt.gt_check(ws)
 
     def timed(fn):
-        fn()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(reps):
-            fn()
-        e1.record()
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / reps
+        return timed_ms(fn, reps)
 
     f_fwd, f_bwd = w.attn_flops()
     if what in ("all", "spd"):
