@@ -44,10 +44,10 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # Measured DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture) per launch of the
 # backward kernel on a 16 384-node graph, divided by N^2: the traffic is dominated by the N^2 bias-index tiles
 # and the N^2/128 dQ reductions, so a launch at another size is estimated as this figure times sum n_g^2.
-BWD_KERNEL_DRAM_BYTES_PER_N2 = 1044.0e6 / (16384.0 ** 2)
+BWD_KERNEL_DRAM_BYTES_PER_N2 = 1037.7e6 / (16384.0 ** 2)
 # The same for the forward kernel (16 384 nodes) and for the bit-matrix SPD build (24 000 nodes; its traffic
 # also grows with the number of BFS levels, so the scaled figure is an estimate).
-FWD_KERNEL_DRAM_BYTES_PER_N2 = 440.4e6 / (16384.0 ** 2)
+FWD_KERNEL_DRAM_BYTES_PER_N2 = 438.1e6 / (16384.0 ** 2)
 SPD_DENSE_DRAM_BYTES_PER_N2 = 2.749e9 / (24000.0 ** 2)
 
 
