@@ -38,6 +38,7 @@ struct SpdParams {
     int32_t n_total;
     int32_t n_graphs;
     int32_t max_dist;
+    int32_t src_per_batch;        // sources a CTA advances at once: 32, or fewer (16, 8) when that still leaves CTA slots idle
 };
 
 // batch_start[g] = sum_{g'<g} ceil(n_g'/32); header[3] = total.  One block.
@@ -52,7 +53,7 @@ __global__ void spd_setup_kernel(SpdParams p)
         int32_t cnt = 0;
         if (g < p.n_graphs) {
             int32_t n_g = p.cu_seqlens ? p.cu_seqlens[g + 1] - p.cu_seqlens[g] : p.n_total;
-            cnt = (n_g + kSrcPerBatch - 1) / kSrcPerBatch;
+            cnt = (n_g + p.src_per_batch - 1) / p.src_per_batch;
         }
         part[threadIdx.x] = cnt;
         __syncthreads();
@@ -176,8 +177,8 @@ __global__ void __launch_bounds__(1024, kSmemState ? 1 : 2) spd_bfs_kernel(SpdPa
         const int32_t n_g = p.cu_seqlens ? p.cu_seqlens[g + 1] - node0 : p.n_total;
         const int64_t ld = (int64_t)((n_g + 15) & ~15);
         uint8_t* spd_g = p.spd + (p.spd_offsets ? p.spd_offsets[g] : 0);
-        const int32_t s0 = (batch - p.batch_start[g]) * kSrcPerBatch;
-        const int32_t n_src = min(kSrcPerBatch, n_g - s0);
+        const int32_t s0 = (batch - p.batch_start[g]) * p.src_per_batch;
+        const int32_t n_src = min(p.src_per_batch, n_g - s0);
         const uint32_t src_mask = n_src == 32 ? 0xffffffffu : ((1u << n_src) - 1u);
         uint8_t* out0 = spd_g + (int64_t)s0 * ld;        // row of source bit 0
 
@@ -826,6 +827,7 @@ struct SpdPlan {
     int32_t dense_acc_rows;    // accumulator rows per CTA group: a bound on the vertices with more than kDenseChunk out-edges
     int threads;
     int grid;
+    int src_per_batch;
     size_t smem_bytes;
     size_t batch_start_off, scratch_off, scratch_words_per_cta, comp_off, sym_off, total_bytes;
 };
@@ -836,7 +838,6 @@ SpdPlan make_plan(const gt_batch* b, int64_t nnz)
     size_t state = spd_state_bytes(b->max_seqlen);
     pl.smem_state = state <= kSmemStateLimit;
     pl.threads = b->max_seqlen <= 1024 ? 256 : (b->max_seqlen <= 4096 ? 512 : 1024);
-    long max_batches = ((long)b->n_total + kSrcPerBatch - 1) / kSrcPerBatch + b->n_graphs;
     int sms = sm_count();
     int per_sm = 1;
     if (pl.smem_state) {
@@ -846,6 +847,13 @@ SpdPlan make_plan(const gt_batch* b, int64_t nnz)
     }
     if (!pl.smem_state) per_sm = 2;      // state in L2: two CTAs per SM keep more loads in flight
     long want = (long)sms * per_sm;
+    // A batch's time is mostly the latency of its levels, so while there are fewer batches than SMs, narrower batches
+    // (less to emit and push per batch, more of them at once) end sooner.
+    pl.src_per_batch = kSrcPerBatch;
+    if (pl.smem_state)
+        while (pl.src_per_batch > 8 && ((long)b->n_total + pl.src_per_batch - 1) / pl.src_per_batch + b->n_graphs <= (long)sms)
+            pl.src_per_batch /= 2;
+    long max_batches = ((long)b->n_total + pl.src_per_batch - 1) / pl.src_per_batch + b->n_graphs;
     pl.grid = (int)(max_batches < want ? max_batches : want);
     pl.smem_bytes = pl.smem_state ? state : 0;
     pl.batch_start_off = kHeaderBytes;
@@ -933,6 +941,7 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
     p.n_total = batch->n_total;
     p.n_graphs = batch->n_graphs;
     p.max_dist = max_dist;
+    p.src_per_batch = pl.src_per_batch;
 
     GT_CUDA_TRY(cudaMemsetAsync(ws + 8, 0, 8, s));     // work counter and item count
     spd_setup_kernel<<<1, 1024, 0, s>>>(p);
