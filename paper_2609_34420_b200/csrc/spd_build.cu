@@ -395,40 +395,61 @@ struct DenseParams {
 };
 
 // item_start[v] = sum_{u<v} max(1, ceil(deg(u)/32)) for the vertices of one graph, and acc_row[v] = number of split
-// vertices (more than one chunk) before v.  One block; both prefix sums ride in one 64-bit scan.
-__global__ void spd_dense_items_kernel(const int32_t* __restrict__ rp, int32_t n, int32_t* __restrict__ item_start,
-                                       int32_t* __restrict__ acc_row)
+// vertices (more than one chunk) before v.  One block of 1024 threads; both prefix sums ride in one 64-bit value.  A thread
+// owns a run of consecutive vertices: it adds its run, the block scans the 1024 run totals once (warp shuffles), and the
+// thread walks its run again to write the prefixes (a scan step per 1024 vertices took 146 us at 65 536 vertices).
+__device__ __forceinline__ unsigned long long dense_item_count(int32_t deg)
 {
-    __shared__ unsigned long long carry;
-    __shared__ unsigned long long part[1024];
-    if (threadIdx.x == 0) carry = 0ull;
-    __syncthreads();
-    for (int base = 0; base < n; base += blockDim.x) {
-        const int v = base + threadIdx.x;
-        unsigned long long cnt = 0ull;
-        if (v < n) {
-            const int32_t deg = rp[v + 1] - rp[v];
-            const unsigned long long chunks = deg <= kDenseChunk ? 1 : (deg + kDenseChunk - 1) / kDenseChunk;
-            cnt = chunks | ((chunks > 1 ? 1ull : 0ull) << 32);
+    const unsigned long long chunks = deg <= kDenseChunk ? 1 : (deg + kDenseChunk - 1) / kDenseChunk;
+    return chunks | ((chunks > 1 ? 1ull : 0ull) << 32);
+}
+
+__global__ void __launch_bounds__(1024) spd_dense_items_kernel(const int32_t* __restrict__ rp, int32_t n, int32_t* __restrict__ item_start,
+                                                               int32_t* __restrict__ acc_row)
+{
+    __shared__ unsigned long long warp_total[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int per = (n + 1023) / 1024;
+    const int v0 = min(n, (int)threadIdx.x * per), v1 = min(n, v0 + per);
+    unsigned long long mine = 0ull;
+    {
+        int32_t prev = v0 < v1 ? rp[v0] : 0;
+#pragma unroll 8
+        for (int v = v0; v < v1; ++v) {
+            const int32_t next = rp[v + 1];
+            mine += dense_item_count(next - prev);
+            prev = next;
         }
-        part[threadIdx.x] = cnt;
-        __syncthreads();
-        for (int off = 1; off < (int)blockDim.x; off <<= 1) {
-            unsigned long long add = threadIdx.x >= (unsigned)off ? part[threadIdx.x - off] : 0ull;
-            __syncthreads();
-            part[threadIdx.x] += add;
-            __syncthreads();
-        }
-        if (v < n) {
-            const unsigned long long before = carry + part[threadIdx.x] - cnt;
-            item_start[v] = (int32_t)(before & 0xffffffffull);
-            acc_row[v] = (int32_t)(before >> 32);
-        }
-        __syncthreads();
-        if (threadIdx.x == blockDim.x - 1) carry += part[threadIdx.x];
-        __syncthreads();
     }
-    if (threadIdx.x == 0) item_start[n] = (int32_t)(carry & 0xffffffffull);
+    unsigned long long incl = mine;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += up;
+    }
+    if (lane == 31) warp_total[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        unsigned long long t = warp_total[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned long long up = __shfl_up_sync(0xffffffffu, t, off);
+            if (lane >= off) t += up;
+        }
+        warp_total[lane] = t;                   // inclusive totals of the warps
+    }
+    __syncthreads();
+    unsigned long long before = incl - mine + (warp > 0 ? warp_total[warp - 1] : 0ull);
+    int32_t prev = v0 < v1 ? rp[v0] : 0;
+#pragma unroll 8
+    for (int v = v0; v < v1; ++v) {
+        const int32_t next = rp[v + 1];
+        item_start[v] = (int32_t)(before & 0xffffffffull);
+        acc_row[v] = (int32_t)(before >> 32);
+        before += dense_item_count(next - prev);
+        prev = next;
+    }
+    if (threadIdx.x == 1023) item_start[n] = (int32_t)(warp_total[31] & 0xffffffffull);
 }
 
 __global__ void spd_dense_item_rec_kernel(const int32_t* __restrict__ rp, const int32_t* __restrict__ item_start, int32_t n,
