@@ -100,9 +100,10 @@ def test_undirected_graphs_deeper_than_max_dist_stop_at_the_clip_level():
     assert oneway[70, 10] == D + 1 and oneway[10, 70] == D and oneway[61, 60] == 1 and oneway[60, 59] == D + 1
 
 
-@pytest.mark.parametrize("n,D", [(3000, 3), (5000, 12)])
+@pytest.mark.parametrize("n,D", [(3000, 3), (5000, 12), (12000, 6)])
 def test_deep_undirected_single_graph(n, D):
-    """Random geometric graph near its connectivity threshold: many levels, several components."""
+    """Random geometric graph near its connectivity threshold: many levels, several components.  (At 12 000 nodes the
+    graph's CSR no longer fits beside the labels in the component pre-pass's shared memory and is read in place.)"""
     w = wl.Workload("rgg", wl.pack_graphs([wl.random_geometric(n, 5.0, 11)]), 1, 32, D)
     check(w)
 
