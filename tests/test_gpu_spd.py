@@ -167,6 +167,14 @@ def test_packed_batch_with_a_graph_beyond_the_shared_memory_state():
     np.testing.assert_array_equal(a, b)
 
 
+def test_packed_batch_with_a_deep_undirected_graph_beyond_the_shared_memory_state():
+    """The same kernel variant (state in the workspace) where the search stops at level max_dist: a random geometric
+    graph of 18 000 nodes (dozens of levels deep, several components) next to a small directed graph."""
+    big = wl.random_geometric(18000, 5.5, 21)
+    small = wl.random_directed(200, 2.0, 3)
+    check(wl.Workload("packed_deep", wl.pack_graphs([big, small]), 1, 32, 7))
+
+
 def test_a_bounded_wait_that_runs_out_is_reported_and_the_context_stays_usable():
     """Device-timeout path end to end: the test hook makes the grid barrier of the next bit-matrix build wait
     for a thread block that does not exist; the bounded wait gives up, every thread block returns (the kernel
