@@ -77,8 +77,8 @@ __global__ void spd_setup_kernel(SpdParams p)
 // Undirected graphs that are deeper than max_dist: beyond level max_dist only "reachable or not" is left to decide,
 // and in an undirected graph that is "same connected component or not".  One CTA per graph checks that every edge
 // has its reverse (graphs with a vertex of more than kMaxSymDegree out-edges are not examined: the check costs
-// deg^2 loads per vertex, and graphs with hubs are shallow anyway) and labels the components by min-label
-// propagation with pointer jumping in shared memory.  The BFS then stops at level max_dist for such a graph.
+// deg^2 loads per vertex, and graphs with hubs are shallow anyway) and labels the components (hooking and pointer
+// jumping in shared memory).  The BFS then stops at level max_dist for such a graph.
 constexpr int kMaxSymDegree = 64;
 constexpr int kCompThreads = 512;
 
@@ -126,17 +126,29 @@ __global__ void __launch_bounds__(kCompThreads) spd_components_kernel(SpdParams 
         if (threadIdx.x == 0) p.sym[g] = 0;
         return;
     }
-    // Labels are local vertex ids and only ever decrease; lab[v] always names a vertex of v's component.  Only the
-    // owner of v writes lab[v]; reads of other entries may see the old or the new value, both are valid labels.
-    // A round with no change by any thread read stable values, so it proves the fixed point: one label per component.
+    // Components by hooking and pointer jumping: lab[] is a forest of pointers to smaller ids (lab[x] <= x always, so
+    // no cycles).  A round hooks the tree of every edge's larger-labelled end below the other end's label (atomicMin on
+    // the ROOT's pointer, so whole trees merge at once: about log n rounds, where passing labels from vertex to vertex
+    // took one round per hop of the graph's diameter), then every vertex follows its pointers to the root.  A round in
+    // which no hook succeeds has the same root at both ends of every edge: one label, the smallest id, per component.
     for (;;) {
         int changed = 0;
         for (int v = threadIdx.x; v < n_g; v += blockDim.x) {
-            const int old = lab[v];
-            int m = old;
-            for (int e = rp[v]; e < rp[v + 1]; ++e) m = min(m, lab[ci[e] - sub]);
-            m = lab[lab[lab[m]]];               // pointer jumping: the label's own label, three steps
-            if (m < old) { lab[v] = m; changed = 1; }
+            const int pv = lab[v];
+            for (int e = rp[v]; e < rp[v + 1]; ++e) {
+                const int pu = lab[ci[e] - sub];
+                if (pu < pv && pu < atomicMin(&lab[pv], pu)) changed = 1;
+            }
+        }
+        __syncthreads();
+        for (int v = threadIdx.x; v < n_g; v += blockDim.x) {
+            int r = lab[v];
+            for (int hop = 0; hop < n_g; ++hop) {
+                const int up = lab[r];
+                if (up == r) break;
+                r = up;
+            }
+            lab[v] = r;
         }
         if (!__syncthreads_or(changed)) break;
     }
