@@ -407,39 +407,46 @@ struct DenseParams {
 };
 
 // item_start[v] = sum_{u<v} max(1, ceil(deg(u)/32)) for the vertices of one graph, and acc_row[v] = number of split
-// vertices (more than one chunk) before v.  One block of 1024 threads; both prefix sums ride in one 64-bit value.  A thread
-// owns a run of consecutive vertices: it adds its run, the block scans the 1024 run totals once (warp shuffles), and the
-// thread walks its run again to write the prefixes (a scan step per 1024 vertices took 146 us at 65 536 vertices).
+// vertices (more than one chunk) before v; both prefix sums ride in one 64-bit value.  Two small kernels over blocks of
+// 4 096 vertices (a thread owns four consecutive ones): the first leaves every block's total, the second adds the totals of
+// the blocks before its own and scans its block with warp shuffles.  (One thread block for the whole graph took 0.1 ms at
+// 65 536 vertices.)
+constexpr int kScanRun = 4;
+constexpr int kScanBlock = 1024 * kScanRun;
+
 __device__ __forceinline__ unsigned long long dense_item_count(int32_t deg)
 {
     const unsigned long long chunks = deg <= kDenseChunk ? 1 : (deg + kDenseChunk - 1) / kDenseChunk;
     return chunks | ((chunks > 1 ? 1ull : 0ull) << 32);
 }
 
-__global__ void __launch_bounds__(1024) spd_dense_items_kernel(const int32_t* __restrict__ rp, int32_t n, int32_t* __restrict__ item_start,
-                                                               int32_t* __restrict__ acc_row)
+// counts of the calling thread's run of vertices; returns their sum
+__device__ __forceinline__ unsigned long long dense_run_counts(const int32_t* __restrict__ rp, int32_t n, unsigned long long (&c)[kScanRun])
+{
+    const int v0 = (int)blockIdx.x * kScanBlock + (int)threadIdx.x * kScanRun;
+    int32_t r[kScanRun + 1];
+#pragma unroll
+    for (int k = 0; k <= kScanRun; ++k) r[k] = rp[min(v0 + k, n)];
+    unsigned long long sum = 0ull;
+#pragma unroll
+    for (int k = 0; k < kScanRun; ++k) {
+        c[k] = v0 + k < n ? dense_item_count(r[k + 1] - r[k]) : 0ull;
+        sum += c[k];
+    }
+    return sum;
+}
+
+// inclusive scan of one value per thread over a block of 1024 threads; *total = sum over the block
+__device__ __forceinline__ unsigned long long block_scan_1024(unsigned long long x, unsigned long long* total)
 {
     __shared__ unsigned long long warp_total[32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int per = (n + 1023) / 1024;
-    const int v0 = min(n, (int)threadIdx.x * per), v1 = min(n, v0 + per);
-    unsigned long long mine = 0ull;
-    {
-        int32_t prev = v0 < v1 ? rp[v0] : 0;
-#pragma unroll 8
-        for (int v = v0; v < v1; ++v) {
-            const int32_t next = rp[v + 1];
-            mine += dense_item_count(next - prev);
-            prev = next;
-        }
-    }
-    unsigned long long incl = mine;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
-        const unsigned long long up = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += up;
+        const unsigned long long up = __shfl_up_sync(0xffffffffu, x, off);
+        if (lane >= off) x += up;
     }
-    if (lane == 31) warp_total[warp] = incl;
+    if (lane == 31) warp_total[warp] = x;
     __syncthreads();
     if (warp == 0) {
         unsigned long long t = warp_total[lane];
@@ -448,20 +455,47 @@ __global__ void __launch_bounds__(1024) spd_dense_items_kernel(const int32_t* __
             const unsigned long long up = __shfl_up_sync(0xffffffffu, t, off);
             if (lane >= off) t += up;
         }
-        warp_total[lane] = t;                   // inclusive totals of the warps
+        warp_total[lane] = t;
     }
     __syncthreads();
-    unsigned long long before = incl - mine + (warp > 0 ? warp_total[warp - 1] : 0ull);
-    int32_t prev = v0 < v1 ? rp[v0] : 0;
-#pragma unroll 8
-    for (int v = v0; v < v1; ++v) {
-        const int32_t next = rp[v + 1];
-        item_start[v] = (int32_t)(before & 0xffffffffull);
-        acc_row[v] = (int32_t)(before >> 32);
-        before += dense_item_count(next - prev);
-        prev = next;
+    *total = warp_total[31];
+    return x + (warp > 0 ? warp_total[warp - 1] : 0ull);
+}
+
+__global__ void __launch_bounds__(1024) spd_dense_items_total_kernel(const int32_t* __restrict__ rp, int32_t n,
+                                                                     unsigned long long* __restrict__ block_total)
+{
+    unsigned long long c[kScanRun], total;
+    block_scan_1024(dense_run_counts(rp, n, c), &total);
+    if (threadIdx.x == 0) block_total[blockIdx.x] = total;
+}
+
+__global__ void __launch_bounds__(1024) spd_dense_items_kernel(const int32_t* __restrict__ rp, int32_t n,
+                                                               const unsigned long long* __restrict__ block_total,
+                                                               int32_t* __restrict__ item_start, int32_t* __restrict__ acc_row)
+{
+    __shared__ unsigned long long s_before;
+    if (threadIdx.x < 32) {                      // totals of the blocks before this one (at most a few hundred)
+        unsigned long long b = 0ull;
+        for (int i = threadIdx.x; i < (int)blockIdx.x; i += 32) b += block_total[i];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) b += __shfl_xor_sync(0xffffffffu, b, off);
+        if (threadIdx.x == 0) s_before = b;
     }
-    if (threadIdx.x == 1023) item_start[n] = (int32_t)(warp_total[31] & 0xffffffffull);
+    unsigned long long c[kScanRun], total;
+    const unsigned long long mine = dense_run_counts(rp, n, c);
+    const unsigned long long incl = block_scan_1024(mine, &total);       // (its barriers also publish s_before)
+    unsigned long long before = s_before + incl - mine;
+    const int v0 = (int)blockIdx.x * kScanBlock + (int)threadIdx.x * kScanRun;
+#pragma unroll
+    for (int k = 0; k < kScanRun; ++k) {
+        if (v0 + k < n) {
+            item_start[v0 + k] = (int32_t)(before & 0xffffffffull);
+            acc_row[v0 + k] = (int32_t)(before >> 32);
+        }
+        before += c[k];
+    }
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == 0) item_start[n] = (int32_t)((s_before + total) & 0xffffffffull);
 }
 
 __global__ void spd_dense_item_rec_kernel(const int32_t* __restrict__ rp, const int32_t* __restrict__ item_start, int32_t n,
@@ -1001,7 +1035,14 @@ extern "C" gt_status gt_spd_build(const int32_t* row_ptr, const int32_t* col_idx
         // accumulator rows, their counters and the barrier words start at zero
         GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[2], 0, pl.dense_off[4] - pl.dense_off[2], s));
         GT_CUDA_TRY(cudaMemsetAsync(ws + pl.dense_off[7], 0, 256 * kDenseMaxGroups, s));
-        spd_dense_items_kernel<<<1, 1024, 0, s>>>(row_ptr, batch->n_total, d.item_start, d.acc_row);
+        {
+            // the block totals borrow the start of the item records, which are written afterwards
+            const unsigned scan_blocks = (unsigned)((batch->n_total + kScanBlock - 1) / kScanBlock);
+            unsigned long long* block_total = (unsigned long long*)(ws + pl.dense_off[8]);
+            spd_dense_items_total_kernel<<<scan_blocks, 1024, 0, s>>>(row_ptr, batch->n_total, block_total);
+            GT_CUDA_TRY(cudaGetLastError());
+            spd_dense_items_kernel<<<scan_blocks, 1024, 0, s>>>(row_ptr, batch->n_total, block_total, d.item_start, d.acc_row);
+        }
         GT_CUDA_TRY(cudaGetLastError());
         spd_dense_item_rec_kernel<<<(unsigned)((batch->n_total + 255) / 256), 256, 0, s>>>(row_ptr, d.item_start, batch->n_total, d.item_rec);
         GT_CUDA_TRY(cudaGetLastError());
