@@ -232,10 +232,10 @@ def run_cuda(args) -> int:
         if marks is not None:
             marks[4].record()
 
-    # spd: setup + BFS, or for a single graph beyond the shared-memory state setup + item scan + item table +
-    # bit-matrix BFS; fwd; bwd: transpose, pre-pass, main, finalize; chunked: partial + merge
+    # spd: setup + component pre-pass + BFS, or for a single graph beyond the shared-memory state setup + two item-scan
+    # kernels + item table + bit-matrix BFS; fwd; bwd: transpose, pre-pass, main, finalize; chunked: partial + merge
     dense_spd = single and b.max_seqlen >= 14500          # the library's switch to the bit-matrix build
-    kernels_per_step = (4 if dense_spd else 2) + 1 + 4 + (2 if single else 0)
+    kernels_per_step = (5 if dense_spd else 3) + 1 + 4 + (2 if single else 0)
 
     for _ in range(max(args.warmup, 0)):
         step()
