@@ -385,6 +385,19 @@ def run_cuda(args) -> int:
                     "note": "outside the timed step; includes the prepare pass (SPD transpose) and the final conversion"}
         del accs, ctx, dq_r, dk_r, dv_r
 
+    # ---- outside the timed step: the feature-bias variant (four uint8 features per pair) on 8 192 nodes ----
+    feature_bias = None
+    if rank == 0 and single:
+        from paper_2609_34420_b200.profile_case import feature_timings
+        ft = feature_timings(8192, 3, 12)
+        tf = lambda flops, ms: flops / (ms * 1e-3) / 1e12
+        feature_bias = {"n": ft["n"], "distinct_feature_vectors": ft["codes"], "encode_ms": ft["encode_ms"],
+                        "fwd_ms": ft["codes_fwd_ms"], "fwd_tflops": tf(ft["fwd_flops"], ft["codes_fwd_ms"]),
+                        "bwd_ms": ft["codes_bwd_ms"], "bwd_tflops": tf(ft["bwd_flops"], ft["codes_bwd_ms"]),
+                        "fp32_path_fwd_ms": ft["fp32_fwd_ms"], "fp32_path_bwd_ms": ft["fp32_bwd_ms"],
+                        "note": "outside the timed step; categorical features as a code matrix through the tensor-core kernels "
+                                "(forward with the fp32 output), next to the fp32 path on the CUDA cores that serves any features"}
+
     # ---- end to end through the C ABI with host buffers (pinned), copies inside the timed region ----
     host_in = {name: x.cpu().pin_memory() for name, x in
                (("q", q), ("k", k), ("v", v), ("do", do), ("bias", bias), ("rp", rp), ("ci", ci))}
@@ -506,7 +519,7 @@ def run_cuda(args) -> int:
                        "note": "rank 0; `value` uses the mean (max over ranks)"},
         "fwd_tflops": f_fwd / (fwd_ms * 1e-3) / 1e12, "bwd_tflops": bwd_tflops,
         "fwd_chunked_tflops": (f_fwd / (chk_ms * 1e-3) / 1e12) if single else None,
-        "bwd_chunked": bwd_chunked, "fwd_ring_steps": fwd_ring, "bwd_ring_steps": bwd_ring,
+        "bwd_chunked": bwd_chunked, "fwd_ring_steps": fwd_ring, "bwd_ring_steps": bwd_ring, "feature_bias": feature_bias,
         "spd_build_gbs": roofline_spd["achieved"],
         "pct_of_bf16_peak": {"burst": 100 * value / world / float(peaks["bf16_tflops"]),
                              "sustained": 100 * value / world / peak_tf, "nominal_2250": 100 * value / world / 2250.0},

@@ -31,9 +31,10 @@ def timed_ms(fn, reps):
     return e0.elapsed_time(e1) / reps
 
 
-def feature_case(n: int, reps: int, n_vec: int) -> int:
+def feature_timings(n: int, reps: int, n_vec: int, cuda_core_path: bool = True) -> dict:
+    """CUDA-event timings (ms) of the feature-bias variant on n nodes, H=8, d=64, n_vec distinct feature vectors."""
     H, d = 8, 64
-    dev = torch.device("cuda", 0)
+    dev = torch.device("cuda", torch.cuda.current_device())
     g = torch.Generator(device=dev).manual_seed(1)
     q, k, v, do = (torch.randn(n, H, d, device=dev, generator=g).bfloat16() for _ in range(4))
     wt = torch.randn(H, 4, device=dev, generator=g) * 0.01
@@ -42,21 +43,20 @@ def feature_case(n: int, reps: int, n_vec: int) -> int:
     batch = gt.Batch(n)
     out, dq, dk, dv = (torch.empty_like(q) for _ in range(4))
     lse, dw = torch.empty(H, n, device=dev), torch.empty_like(wt)
-    f_fwd, f_bwd = 4.0 * H * d * n * n, 10.0 * H * d * n * n
-    ms = timed_ms(lambda: gt.gt_feature_attn_fwd(q, k, v, feat, wt, batch, out, lse), reps)
-    print(f"feature fwd (CUDA cores) {ms:.3f} ms  {f_fwd / ms / 1e9:.1f} TFLOP/s")
-    ws_b = gt.gt_feature_attn_bwd(q, k, v, do, lse, feat, wt, batch, dq, dk, dv, dw)
-    ms = timed_ms(lambda: gt.gt_feature_attn_bwd(q, k, v, do, lse, feat, wt, batch, dq, dk, dv, dw, ws_b), reps)
-    print(f"feature bwd (CUDA cores) {ms:.3f} ms  {f_bwd / ms / 1e9:.1f} TFLOP/s")
-    gt.gt_check(ws_b)
+    res = {"n": n, "n_heads": H, "head_dim": d, "fwd_flops": 4.0 * H * d * n * n, "bwd_flops": 10.0 * H * d * n * n}
+    if cuda_core_path:
+        res["fp32_fwd_ms"] = timed_ms(lambda: gt.gt_feature_attn_fwd(q, k, v, feat, wt, batch, out, lse), reps)
+        ws_b = gt.gt_feature_attn_bwd(q, k, v, do, lse, feat, wt, batch, dq, dk, dv, dw)
+        res["fp32_bwd_ms"] = timed_ms(lambda: gt.gt_feature_attn_bwd(q, k, v, do, lse, feat, wt, batch, dq, dk, dv, dw, ws_b), reps)
+        gt.gt_check(ws_b)
     ld = (n + 15) // 16 * 16
     codes = torch.empty(n * ld, dtype=torch.uint8, device=dev)
     vectors = torch.empty(256, dtype=torch.int32, device=dev)
     ws_e = gt.gt_feature_encode(feat, batch, codes, vectors)
     gt.gt_check(ws_e)
     width = max(gt.gt_feature_encode_count(ws_e), 3)
-    ms = timed_ms(lambda: gt.gt_feature_encode(feat, batch, codes, vectors, ws_e), reps)
-    print(f"feature encode {ms:.3f} ms  {n * n * 5 / ms / 1e6:.1f} GB/s  ({width} codes)")
+    res["codes"] = width
+    res["encode_ms"] = timed_ms(lambda: gt.gt_feature_encode(feat, batch, codes, vectors, ws_e), reps)
     table, dtable = torch.empty(H, width, device=dev), torch.empty(H, width, device=dev)
     out32 = torch.empty(n, H, d, device=dev)
 
@@ -70,12 +70,21 @@ def feature_case(n: int, reps: int, n_vec: int) -> int:
         return ws
 
     ws_f, ws_bb = fwd(), bwd()
-    ms = timed_ms(lambda: fwd(ws_f), reps)
-    print(f"feature fwd (codes, fp32 output too) {ms:.3f} ms  {f_fwd / ms / 1e9:.1f} TFLOP/s")
-    ms = timed_ms(lambda: bwd(ws_bb), reps)
-    print(f"feature bwd (codes) {ms:.3f} ms  {f_bwd / ms / 1e9:.1f} TFLOP/s")
+    res["codes_fwd_ms"] = timed_ms(lambda: fwd(ws_f), reps)
+    res["codes_bwd_ms"] = timed_ms(lambda: bwd(ws_bb), reps)
     gt.gt_check(ws_f)
     gt.gt_check(ws_bb)
+    return res
+
+
+def feature_case(n: int, reps: int, n_vec: int) -> int:
+    r = feature_timings(n, reps, n_vec)
+    tf = lambda flops, ms: flops / ms / 1e9
+    print(f"feature fwd (CUDA cores) {r['fp32_fwd_ms']:.3f} ms  {tf(r['fwd_flops'], r['fp32_fwd_ms']):.1f} TFLOP/s")
+    print(f"feature bwd (CUDA cores) {r['fp32_bwd_ms']:.3f} ms  {tf(r['bwd_flops'], r['fp32_bwd_ms']):.1f} TFLOP/s")
+    print(f"feature encode {r['encode_ms']:.3f} ms  {n * n * 5 / r['encode_ms'] / 1e6:.1f} GB/s  ({r['codes']} codes)")
+    print(f"feature fwd (codes, fp32 output too) {r['codes_fwd_ms']:.3f} ms  {tf(r['fwd_flops'], r['codes_fwd_ms']):.1f} TFLOP/s")
+    print(f"feature bwd (codes) {r['codes_bwd_ms']:.3f} ms  {tf(r['bwd_flops'], r['codes_bwd_ms']):.1f} TFLOP/s")
     return 0
 
 
