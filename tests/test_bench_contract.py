@@ -30,3 +30,29 @@ def test_rank_zero_prints_one_line_with_the_contract_keys():
 def test_other_ranks_exit_without_work():
     r = run({"RANK": "1", "LOCAL_RANK": "1", "WORLD_SIZE": "2"}, "--gpus", "2", "--steps", "1", "--warmup", "0")
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+import pytest
+
+
+@pytest.mark.gpu
+def test_cuda_arm_prints_the_contract_line_on_a_small_workload():
+    """The same script's own arm on config 2 (4 096 nodes): schema of the line, not its numbers."""
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--workload", "ba4096", "--steps", "3", "--warmup", "3"],
+                       capture_output=True, text=True, cwd=ROOT, timeout=900)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.strip()]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                "vs_baseline", "dtype", "data", "config", "roofline", "cpu_baseline", "e2e", "gpu_launches", "clocks"):
+        assert key in d, key
+    assert d["n_gpus"] == 1 and d["steps"] == 3 and d["warmup"] == 3 and d["dtype"] == "bf16" and d["data"] == "synthetic"
+    assert d["config"]["workload"] == "ba4096" and d["value"] > 0 and d["gpu_launches"] > 0
+    roof = d["roofline"]
+    assert roof["bound"] == "tensor" and roof["unit"] == "TFLOP/s" and 0 < roof["frac"] < 1.2
+    assert abs(roof["frac"] - roof["achieved"] / roof["peak"]) < 1e-9
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["value"] > 0
+    assert d["e2e"]["value"] > 0 and d["e2e"]["h2d_bytes_per_step"] > 0 and d["e2e"]["d2h_bytes_per_step"] > 0
+    assert d["e2e"]["value"] < d["value"]            # copies inside the timed region: never the device-timed number again
+    assert "sm_mhz" in d["clocks"] and "reasons" in d["clocks"]
